@@ -1,0 +1,223 @@
+"""fp64 CPU oracle for the SSD hot path -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper around ``ssd_oracle.c`` (plain C, double precision, written
+from the paper).  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this package; the CUDA library never does, and this
+package never imports the CUDA library.  bf16 tensors travel as numpy ``uint16``
+bit patterns.
+
+Every function cites the passage of the paper it follows in ``ssd_oracle.c``.
+Parity status: all functions are pinned by ``tests/test_oracle_pins.py``
+(closed forms, brute force, special cases, a library routine); none is
+"parity unpinned".
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ssd_oracle.c")
+_LIB = os.path.join(_HERE, "libssd_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over independent pairs)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        )
+    return _LIB
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def _p(a, ty):
+    return a.ctypes.data_as(C.POINTER(ty))
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(_LIB)
+        u16p, f64p, i32p, u8p = (C.POINTER(C.c_uint16), C.POINTER(C.c_double),
+                                 C.POINTER(C.c_int32), C.POINTER(C.c_uint8))
+        L.ssd_oracle_attention_row.argtypes = [u16p, u16p, C.c_int, C.c_int, C.c_double, f64p]
+        L.ssd_oracle_attention_row.restype = None
+        L.ssd_oracle_sparsity_sum.argtypes = [u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                              C.c_double]
+        L.ssd_oracle_sparsity_sum.restype = C.c_double
+        L.ssd_oracle_sparsity.argtypes = [u16p, u16p] + [C.c_int] * 7 + [C.c_double, f64p]
+        L.ssd_oracle_sparsity.restype = None
+        L.ssd_oracle_labels.argtypes = [f64p, C.c_int, C.c_double, u8p]
+        L.ssd_oracle_labels.restype = None
+        L.ssd_oracle_scores.argtypes = [u16p, u16p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double,
+                                        f64p, f64p]
+        L.ssd_oracle_scores.restype = None
+        L.ssd_oracle_topm.argtypes = [f64p, C.c_int, C.c_int, i32p]
+        L.ssd_oracle_topm.restype = C.c_int
+        L.ssd_oracle_retained_set.argtypes = [C.c_int] * 5 + [i32p, C.c_int, i32p]
+        L.ssd_oracle_retained_set.restype = C.c_int
+        L.ssd_oracle_attend.argtypes = [u16p, u16p, u16p, C.c_int, i32p, C.c_int, C.c_double, f64p,
+                                        f64p]
+        L.ssd_oracle_attend.restype = None
+        L.ssd_oracle_select_batch.argtypes = [u16p, u16p, u8p, C.c_long] + [C.c_int] * 7 + [
+            C.c_double, f64p, i32p, i32p]
+        L.ssd_oracle_select_batch.restype = None
+        L.ssd_oracle_decode_batch.argtypes = [u16p, u16p, u16p, u8p, i32p, i32p, C.c_long] + [
+            C.c_int] * 7 + [C.c_double, C.c_int, f64p]
+        L.ssd_oracle_decode_batch.restype = None
+        L.ssd_oracle_threads.argtypes = []
+        L.ssd_oracle_threads.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def threads() -> int:
+    return int(lib().ssd_oracle_threads())
+
+
+def default_scale(D: int) -> float:
+    return 1.0 / float(np.sqrt(np.float64(D)))
+
+
+def attention_row(q, K, scale=None):
+    """a = softmax(scale * K q) over all rows of K.  q [D], K [n_ctx, D] (uint16 bf16)."""
+    q, K = _u16(q), _u16(K)
+    n, D = K.shape
+    out = np.empty(n, np.float64)
+    lib().ssd_oracle_attention_row(_p(q, C.c_uint16), _p(K, C.c_uint16), n, D,
+                                   default_scale(D) if scale is None else scale, _p(out, C.c_double))
+    return out
+
+
+def sparsity(Q_cal, K_cal, L, w, scale=None):
+    """s[l,h] of Sec. 3.3.  Q_cal [layers,P,H,N,D], K_cal [layers,P,H,L+N,D] -> [layers,H]."""
+    Q_cal, K_cal = _u16(Q_cal), _u16(K_cal)
+    nl, P, H, N, D = Q_cal.shape
+    assert K_cal.shape == (nl, P, H, L + N, D), (K_cal.shape, (nl, P, H, L + N, D))
+    s = np.empty((nl, H), np.float64)
+    lib().ssd_oracle_sparsity(_p(Q_cal, C.c_uint16), _p(K_cal, C.c_uint16), nl, P, H, L, N, D, w,
+                              default_scale(D) if scale is None else scale, _p(s, C.c_double))
+    return s
+
+
+def sparsity_sum(Q, K, L, w, scale=None):
+    """Inner sum over t of the ratio for one (layer, head, prompt).  Q [N,D], K [L+N,D]."""
+    Q, K = _u16(Q), _u16(K)
+    N, D = Q.shape
+    assert K.shape == (L + N, D)
+    return float(lib().ssd_oracle_sparsity_sum(_p(Q, C.c_uint16), _p(K, C.c_uint16), L, N, D, w,
+                                               default_scale(D) if scale is None else scale))
+
+
+def labels(s, tau):
+    """1 = Semantic iff s > tau (equality is Spatial)."""
+    s = np.ascontiguousarray(s, np.float64)
+    out = np.empty(s.shape, np.uint8)
+    lib().ssd_oracle_labels(_p(s, C.c_double), s.size, float(tau), _p(out, C.c_uint8))
+    return out
+
+
+def scores(Q_obs, K, L, n0, scale=None, return_prompt_mass=False):
+    """Accumulated post-softmax score per image token.  Q_obs [n_obs,D], K [L+n0,D] -> [n0]."""
+    Q_obs, K = _u16(Q_obs), _u16(K)
+    n_obs, D = Q_obs.shape
+    assert K.shape[0] >= L + n0 and K.shape[1] == D
+    sc = np.empty(n0, np.float64)
+    pm = C.c_double(0.0)
+    lib().ssd_oracle_scores(_p(Q_obs, C.c_uint16), _p(K, C.c_uint16), L, n0, n_obs, D,
+                            default_scale(D) if scale is None else scale, _p(sc, C.c_double),
+                            C.byref(pm))
+    return (sc, pm.value) if return_prompt_mass else sc
+
+
+def topm(score, n_cand, M):
+    """Indices (ascending) of the min(M, n_cand) largest of score[:n_cand]; ties -> lowest index."""
+    score = np.ascontiguousarray(score, np.float64)
+    assert score.size >= n_cand
+    idx = np.empty(max(M, 1), np.int32)
+    c = lib().ssd_oracle_topm(_p(score, C.c_double), int(n_cand), int(M), _p(idx, C.c_int32))
+    return idx[:c].copy()
+
+
+def retained_set(is_semantic, L, t, W, R, top_idx=None):
+    """Absolute positions a head holds after image token t-1 was appended (ascending)."""
+    top = np.ascontiguousarray(top_idx if top_idx is not None else np.zeros(0), np.int32)
+    pos = np.empty(L + t + top.size + 1, np.int32)
+    n = lib().ssd_oracle_retained_set(int(bool(is_semantic)), L, t, W, R, _p(top, C.c_int32),
+                                      top.size, _p(pos, C.c_int32))
+    return pos[:n].copy()
+
+
+def attend(q, K_hist, V_hist, pos, scale=None, return_weights=False):
+    """softmax attention of q over the given positions of the full history -> out [D] fp64."""
+    q, K_hist, V_hist = _u16(q), _u16(K_hist), _u16(V_hist)
+    pos = np.ascontiguousarray(pos, np.int32)
+    D = q.shape[0]
+    out = np.empty(D, np.float64)
+    wts = np.empty(max(pos.size, 1), np.float64)
+    lib().ssd_oracle_attend(_p(q, C.c_uint16), _p(K_hist, C.c_uint16), _p(V_hist, C.c_uint16), D,
+                            _p(pos, C.c_int32), pos.size,
+                            default_scale(D) if scale is None else scale, _p(out, C.c_double),
+                            _p(wts, C.c_double))
+    return (out, wts[:pos.size]) if return_weights else out
+
+
+def select_batch(Q_obs, K, is_semantic, L, n0, M, R, scale=None):
+    """Scores and top-M for many pairs.
+
+    Q_obs [..., n_obs, D], K [..., L+n_keys, D] (n_keys >= n0), is_semantic [...] uint8.
+    Returns (score [..., n0] fp64, idx [..., M] int32 padded with -1, cnt [...] int32).
+    """
+    Q_obs, K = _u16(Q_obs), _u16(K)
+    lead = Q_obs.shape[:-2]
+    n_obs, D = Q_obs.shape[-2:]
+    n_keys = K.shape[-2] - L
+    assert K.shape[:-2] == lead and n_keys >= n0
+    sem = np.ascontiguousarray(np.broadcast_to(is_semantic, lead), np.uint8)
+    n_pairs = int(np.prod(lead)) if lead else 1
+    sc = np.zeros(lead + (max(n0, 0),), np.float64)
+    idx = np.full(lead + (M,), -1, np.int32)
+    cnt = np.zeros(lead, np.int32)
+    lib().ssd_oracle_select_batch(_p(Q_obs, C.c_uint16), _p(K, C.c_uint16), _p(sem, C.c_uint8),
+                                  n_pairs, L, n_keys, n0, n_obs, D, M, R,
+                                  default_scale(D) if scale is None else scale, _p(sc, C.c_double),
+                                  _p(idx, C.c_int32), _p(cnt, C.c_int32))
+    return sc, idx, cnt
+
+
+def decode_batch(q, K_hist, V_hist, is_semantic, idx, cnt, L, t, W, M, R, scale=None, full=False):
+    """Decode attention at image step t for many pairs -> out [..., D] fp64.
+
+    q [..., D]; K_hist, V_hist [..., L+n_keys, D] with n_keys >= t; idx [..., M], cnt [...].
+    """
+    q, K_hist, V_hist = _u16(q), _u16(K_hist), _u16(V_hist)
+    lead = q.shape[:-1]
+    D = q.shape[-1]
+    n_keys = K_hist.shape[-2] - L
+    assert K_hist.shape[:-2] == lead and V_hist.shape == K_hist.shape and n_keys >= t
+    sem = np.ascontiguousarray(np.broadcast_to(is_semantic, lead), np.uint8)
+    n_pairs = int(np.prod(lead)) if lead else 1
+    if idx is None:
+        idx = np.full(lead + (M,), -1, np.int32)
+        cnt = np.zeros(lead, np.int32)
+    idx = np.ascontiguousarray(idx, np.int32)
+    cnt = np.ascontiguousarray(cnt, np.int32)
+    assert idx.shape == lead + (M,) and cnt.shape == lead
+    out = np.empty(lead + (D,), np.float64)
+    lib().ssd_oracle_decode_batch(_p(q, C.c_uint16), _p(K_hist, C.c_uint16), _p(V_hist, C.c_uint16),
+                                  _p(sem, C.c_uint8), _p(idx, C.c_int32), _p(cnt, C.c_int32), n_pairs,
+                                  L, n_keys, t, D, W, M, R,
+                                  default_scale(D) if scale is None else scale, int(bool(full)),
+                                  _p(out, C.c_double))
+    return out
