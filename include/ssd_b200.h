@@ -1,0 +1,161 @@
+/*
+ * ssd_b200.h -- C ABI of the SSD head-decoupled compressed KV cache for single-token
+ * decode attention on NVIDIA B200 (sm_100a).
+ *
+ * The method (paper: "SSD: Spatial-Semantic Head Decoupling for Efficient Autoregressive
+ * Image Generation") splits attention heads into spatial-locality heads, which keep a short
+ * window of the most recent visual tokens, and semantic-sink heads, which keep the top-M
+ * visual tokens by accumulated attention score plus a small reserved recent window
+ * (Sec. 3.3, Algorithm 1).  This library holds that cache and runs attention over it.
+ *
+ * Conventions
+ *  - All tensors are bf16, row-major, innermost dimension head_dim (= 128).
+ *  - Pointers named *_host are host memory; every other data pointer is DEVICE memory owned
+ *    by the caller.  The library allocates no device memory: the caller hands one device
+ *    buffer to ssd_cache_create and it is carved up internally.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
+ *    on it and return; exceptions are noted per function.  One cache must be driven from one
+ *    stream at a time (launches that overlap on the GPU would race on its scratch areas).
+ *  - L = prompt_len prompt tokens are retained whole by every head.  Image token j (0-based)
+ *    has absolute position L + j; image step t = j + 1.
+ *  - All sequences advance in lock step: every call acts on all n_seqs sequences of a layer.
+ *  - Every function returns an ssd_status (0 = SSD_OK, negative = error) unless noted; all
+ *    argument checking happens on the host before anything is launched.
+ */
+#ifndef SSD_B200_H
+#define SSD_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ssd_cache ssd_cache; /* opaque; created by ssd_cache_create, owned by the library */
+
+typedef struct ssd_config {
+  int32_t n_layers;
+  int32_t n_seqs;           /* sequences (a classifier-free-guidance pair is two) */
+  int32_t n_heads;          /* multi-head attention: kv heads == query heads; <= 128 */
+  int32_t head_dim;         /* must be 128 */
+  int32_t prompt_len;       /* L >= 0 */
+  int32_t max_image_tokens; /* N = h*w of the token grid */
+  int32_t window;           /* W >= 1: ring slots of a spatial head, newest token included */
+  int32_t sink_budget;      /* M >= 0: top-M static slots of a semantic head */
+  int32_t sink_recent;      /* R >= 1: ring slots of a semantic head, newest token included */
+  int32_t cls_window;       /* w of the sparsity metric (Sec. 3.3; the paper uses 32) */
+  float tau;                /* a head is semantic iff its sparsity s > tau (Sec. 3.3) */
+  float softmax_scale;      /* 0 selects 1/sqrt(head_dim) */
+} ssd_config;
+
+enum ssd_status {
+  SSD_OK = 0,
+  SSD_ERR_INVALID_ARG = -1, /* null pointer, out-of-range size or layer */
+  SSD_ERR_BAD_STATE = -2,   /* call order violated (e.g. compress before labels exist) */
+  SSD_ERR_OVERFLOW = -3,    /* append beyond max_image_tokens (cf. Algorithm 2, buffer overflow) */
+  SSD_ERR_NO_MEM = -4,      /* caller's device buffer too small for the layout */
+  SSD_ERR_CUDA = -5         /* a CUDA runtime call or launch failed */
+};
+
+/* Human-readable name of a status code (static storage; never NULL). */
+const char *ssd_status_string(int status);
+
+/* Device bytes ssd_cache_create needs.  n_sink_heads_total = number of (layer, head) entries
+ * that will be labelled semantic; pass -1 for the worst case over all labelings.  Returns 0 on
+ * an invalid config. */
+size_t ssd_cache_required_bytes(const ssd_config *cfg, int32_t n_sink_heads_total);
+
+/* Create a cache over caller-owned device memory [dev_mem, dev_mem + dev_bytes) (256-byte
+ * aligned).  Validates the config, lays out tables and scratch at the front of the buffer and
+ * clears them (synchronously, on the default stream).  Head labels do not exist yet: call
+ * ssd_classify_heads or ssd_set_head_labels next.  The buffer must outlive the cache. */
+int ssd_cache_create(const ssd_config *cfg, void *dev_mem, size_t dev_bytes, ssd_cache **out);
+
+/* Release the host object.  The device buffer stays with the caller.  NULL is accepted. */
+int ssd_cache_free(ssd_cache *cache);
+
+/* Head classification (Sec. 3.3): sparsity s[l,h] = mean over calibration sequences p and image
+ * steps t of (attention mass on visual tokens older than the newest cls_window) / (mass on all
+ * visual tokens so far); label = s > tau.
+ *   q_cal [n_layers, n_cal_seqs, n_heads, n_img, head_dim]   queries of image steps 1..n_img
+ *   k_cal [n_layers, n_cal_seqs, n_heads, prompt_len + n_img, head_dim]
+ *   s_out_host      [n_layers * n_heads] float  (may be NULL)
+ *   labels_out_host [n_layers * n_heads] uint8, 1 = semantic (may be NULL)
+ * Installs the labels in the cache (fixing the per-head layout) and SYNCHRONISES the stream.
+ * SSD_ERR_NO_MEM if the resulting layout does not fit the buffer. */
+int ssd_classify_heads(ssd_cache *cache, const void *q_cal, const void *k_cal, int32_t n_cal_seqs,
+                       int32_t n_img, float *s_out_host, uint8_t *labels_out_host, void *stream);
+
+/* The same measurement without installing labels: writes, per (layer, head), the sum over the
+ * given calibration sequences and steps of the ratio above (double, [n_layers * n_heads]).  A
+ * caller that shards calibration sequences over several GPUs adds these sums across ranks,
+ * divides by (total sequences * n_img) and calls ssd_set_head_labels.  Synchronises the stream. */
+int ssd_classify_partial(ssd_cache *cache, const void *q_cal, const void *k_cal, int32_t n_cal_seqs,
+                         int32_t n_img, double *ratio_sums_host, void *stream);
+
+/* Install head labels directly ([n_layers * n_heads] uint8, 1 = semantic): by-construction or
+ * random partitions (Sec. 4.4 ablation).  Resets every layer to the empty state. */
+int ssd_set_head_labels(ssd_cache *cache, const uint8_t *labels_host);
+
+/* Bulk-load one layer from an uncompressed cache holding the prompt and n0 image tokens, and
+ * compress it (Algorithm 1; Algorithm 2's prefill split when n0 == 0).
+ *   q_obs  [n_seqs, n_heads, n_obs, head_dim]  queries of image steps n0-n_obs+1 .. n0
+ *   k_full, v_full [n_seqs, n_heads, prompt_len + n0, head_dim]
+ * Semantic heads: score[j] = sum over the observed steps of the post-softmax attention on image
+ * token j (causal, softmax over prompt + image tokens); keep the min(M, n0-R) best-scoring
+ * tokens among j in [0, n0-R) (ties: lowest j), stored in ascending j, plus the R newest tokens.
+ * Spatial heads: keep the W newest tokens.  Every head keeps the whole prompt.
+ * 0 <= n0 <= max_image_tokens; 0 <= n_obs <= n0 (q_obs may be NULL when n_obs == 0 or the layer
+ * has no semantic head).  Replaces the layer's previous contents.  Asynchronous. */
+int ssd_compress(ssd_cache *cache, int32_t layer, const void *q_obs, const void *k_full,
+                 const void *v_full, int32_t n0, int32_t n_obs, void *stream);
+
+/* Append the newest token's K/V for every (sequence, head) of a layer: written into the head's
+ * ring, overwriting (evicting) the oldest ring entry once the ring is full (Algorithm 1, Append).
+ *   k_new, v_new [n_seqs, n_heads, head_dim]
+ * SSD_ERR_OVERFLOW once max_image_tokens tokens are held.  Asynchronous. */
+int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new, void *stream);
+
+/* Single-token decode attention over the layer's retained slots, both head types in one launch:
+ * out[s,h] = sum_i softmax_i(scale * <q[s,h], K_i>) V_i over the prompt, static and ring slots
+ * that hold a token (the token just appended included).  fp32 accumulation, bf16 output.
+ *   q, out [n_seqs, n_heads, head_dim]
+ * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
+int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
+
+/* One decode step of one layer from HOST buffers (pinned memory recommended): copies q, k_new and
+ * v_new to the device, appends, attends, and copies the output back, all enqueued on `stream`.
+ *   q_host, k_new_host, v_new_host, out_host [n_seqs, n_heads, head_dim] bf16 on the host
+ * The host buffers must stay untouched until the stream has drained.  Asynchronous. */
+int ssd_step_host(ssd_cache *cache, int32_t layer, const void *q_host, const void *k_new_host,
+                  const void *v_new_host, void *out_host, void *stream);
+
+/* Absolute positions held by each slot of a layer, for inspection and index-set parity:
+ * idx_host [n_seqs, n_heads, max_slots] int32 with max_slots = ssd_cache_max_slots(); slots are
+ * ordered prompt, static (ascending position), ring (physical ring order); -1 = empty or unused.
+ * Synchronises the device. */
+int ssd_cache_get_indices(ssd_cache *cache, int32_t layer, int32_t *idx_host);
+int32_t ssd_cache_max_slots(const ssd_cache *cache); /* prompt_len + max(window, M + R) */
+
+/* Number of slots currently holding a token, per head of a layer: len_host [n_heads]. */
+int ssd_cache_get_lengths(ssd_cache *cache, int32_t layer, int32_t *len_host);
+
+/* Current labels ([n_layers * n_heads] uint8) and image tokens held so far by a layer. */
+int ssd_cache_get_labels(ssd_cache *cache, uint8_t *labels_host);
+int32_t ssd_cache_tokens(const ssd_cache *cache, int32_t layer); /* -1 on bad arguments */
+
+/* Set a layer's image-token counter back to an earlier value t (n0 <= t <= current), so a
+ * benchmark can replay the same decode steps; ring contents are not restored. */
+int ssd_cache_rewind(ssd_cache *cache, int32_t layer, int32_t t);
+
+/* K+V bytes the cache holds per sequence over all layers at full occupancy (slots * 512 B). */
+int ssd_cache_kv_bytes(ssd_cache *cache, size_t *bytes_per_seq);
+
+/* Number of kernels this library has launched since the process started (for audit). */
+uint64_t ssd_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSD_B200_H */

@@ -1,0 +1,257 @@
+"""ctypes binding of the C ABI in ``include/ssd_b200.h`` -- argument marshalling only.
+
+Every step of the path runs inside the CUDA library.  If the library is missing or cannot be
+loaded this module raises; there is no CPU fallback.  torch is used for device memory and the
+current stream, nothing else.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+SSD_OK = 0
+SSD_ERR_INVALID_ARG = -1
+SSD_ERR_BAD_STATE = -2
+SSD_ERR_OVERFLOW = -3
+SSD_ERR_NO_MEM = -4
+SSD_ERR_CUDA = -5
+
+EXPORTS = [
+    "ssd_status_string", "ssd_cache_required_bytes", "ssd_cache_create", "ssd_cache_free",
+    "ssd_classify_heads", "ssd_classify_partial", "ssd_set_head_labels", "ssd_compress", "ssd_append",
+    "ssd_decode_attn", "ssd_step_host", "ssd_cache_get_indices", "ssd_cache_max_slots",
+    "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
+    "ssd_cache_kv_bytes", "ssd_kernel_launch_count",
+]
+
+
+class SsdConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_layers", "n_seqs", "n_heads", "head_dim", "prompt_len", "max_image_tokens", "window",
+        "sink_budget", "sink_recent", "cls_window")] + [("tau", C.c_float), ("softmax_scale", C.c_float)]
+
+
+class SsdError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} ({code})")
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load():
+    """Load (building first if the sources are newer) the CUDA library.  Raises if impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    L = C.CDLL(path)
+    vp, i32, u64 = C.c_void_p, C.c_int32, C.c_uint64
+    cfgp = C.POINTER(SsdConfig)
+    L.ssd_status_string.argtypes = [C.c_int]
+    L.ssd_status_string.restype = C.c_char_p
+    L.ssd_cache_required_bytes.argtypes = [cfgp, i32]
+    L.ssd_cache_required_bytes.restype = C.c_size_t
+    L.ssd_cache_create.argtypes = [cfgp, vp, C.c_size_t, C.POINTER(vp)]
+    L.ssd_cache_free.argtypes = [vp]
+    L.ssd_classify_heads.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp]
+    L.ssd_classify_partial.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+    L.ssd_set_head_labels.argtypes = [vp, vp]
+    L.ssd_compress.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
+    L.ssd_append.argtypes = [vp, i32, vp, vp, vp]
+    L.ssd_decode_attn.argtypes = [vp, i32, vp, vp, vp]
+    L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
+    L.ssd_cache_max_slots.argtypes = [vp]
+    L.ssd_cache_max_slots.restype = i32
+    L.ssd_cache_get_lengths.argtypes = [vp, i32, vp]
+    L.ssd_cache_get_labels.argtypes = [vp, vp]
+    L.ssd_cache_tokens.argtypes = [vp, i32]
+    L.ssd_cache_tokens.restype = i32
+    L.ssd_cache_rewind.argtypes = [vp, i32, i32]
+    L.ssd_cache_kv_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.ssd_kernel_launch_count.argtypes = []
+    L.ssd_kernel_launch_count.restype = u64
+    for n in EXPORTS:
+        f = getattr(L, n)
+        if f.restype is C.c_int and n not in ("ssd_cache_max_slots", "ssd_cache_tokens"):
+            f.restype = C.c_int
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return load().ssd_status_string(int(code)).decode()
+
+
+def kernel_launch_count() -> int:
+    return int(load().ssd_kernel_launch_count())
+
+
+def make_config(n_layers, n_seqs, n_heads, prompt_len, max_image_tokens, window, sink_budget,
+                sink_recent, cls_window=32, tau=0.45, softmax_scale=0.0, head_dim=128) -> SsdConfig:
+    return SsdConfig(n_layers, n_seqs, n_heads, head_dim, prompt_len, max_image_tokens, window,
+                     sink_budget, sink_recent, cls_window, tau, softmax_scale)
+
+
+def config_from_workload(w, n_layers: Optional[int] = None, n_seqs: Optional[int] = None) -> SsdConfig:
+    return make_config(n_layers or w.n_layers, n_seqs or w.n_seqs, w.n_heads, w.prompt_len, w.n_img,
+                       w.window, w.sink_budget, w.sink_recent, w.cls_window, w.tau)
+
+
+def required_bytes(cfg: SsdConfig, n_sink_heads_total: int = -1) -> int:
+    return int(load().ssd_cache_required_bytes(C.byref(cfg), int(n_sink_heads_total)))
+
+
+def _stream() -> int:
+    return int(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t: torch.Tensor, shape, what: str) -> int:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and tuple(t.shape) == tuple(shape)):
+        raise ValueError(f"{what}: want contiguous CUDA bf16 {tuple(shape)}, got {t.dtype} {tuple(t.shape)} on {t.device}")
+    return t.data_ptr()
+
+
+class SsdCache:
+    """Python handle of an ``ssd_cache`` (one GPU, one stream at a time)."""
+
+    def __init__(self, cfg: SsdConfig, n_sink_heads_total: int = -1, device="cuda:0"):
+        self._h = None
+        self.lib = load()
+        self.cfg = cfg
+        nbytes = required_bytes(cfg, n_sink_heads_total)
+        if nbytes == 0:
+            raise SsdError(SSD_ERR_INVALID_ARG, "ssd_cache_required_bytes")
+        if not torch.cuda.is_available():
+            raise RuntimeError("ssd_b200 needs a CUDA device; there is no CPU path")
+        self.device = torch.device(device)
+        self.mem = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.mem.data_ptr() + 255) // 256 * 256
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = self.lib.ssd_cache_create(C.byref(cfg), base, nbytes, C.byref(h))
+        if rc != SSD_OK:
+            raise SsdError(rc, "ssd_cache_create")
+        self._h = h
+        self.nbytes = nbytes
+
+    # -- lifetime
+    def close(self):
+        if self._h is not None:
+            self.lib.ssd_cache_free(self._h)
+            self._h = None
+            self.mem = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc, what):
+        if rc != SSD_OK:
+            raise SsdError(rc, what)
+
+    # -- labels
+    def set_head_labels(self, labels):
+        lab = np.ascontiguousarray(labels, np.uint8).reshape(-1)
+        assert lab.size == self.cfg.n_layers * self.cfg.n_heads
+        self._check(self.lib.ssd_set_head_labels(self._h, lab.ctypes.data), "ssd_set_head_labels")
+
+    def classify_heads(self, q_cal: torch.Tensor, k_cal: torch.Tensor):
+        c = self.cfg
+        P, n_img = q_cal.shape[1], q_cal.shape[3]
+        qp = _dev(q_cal, (c.n_layers, P, c.n_heads, n_img, c.head_dim), "q_cal")
+        kp = _dev(k_cal, (c.n_layers, P, c.n_heads, c.prompt_len + n_img, c.head_dim), "k_cal")
+        s = np.empty(c.n_layers * c.n_heads, np.float32)
+        lab = np.empty(c.n_layers * c.n_heads, np.uint8)
+        self._check(self.lib.ssd_classify_heads(self._h, qp, kp, P, n_img, s.ctypes.data, lab.ctypes.data,
+                                                _stream()), "ssd_classify_heads")
+        return s.reshape(c.n_layers, c.n_heads), lab.reshape(c.n_layers, c.n_heads)
+
+    def classify_partial(self, q_cal: torch.Tensor, k_cal: torch.Tensor):
+        c = self.cfg
+        P, n_img = q_cal.shape[1], q_cal.shape[3]
+        qp = _dev(q_cal, (c.n_layers, P, c.n_heads, n_img, c.head_dim), "q_cal")
+        kp = _dev(k_cal, (c.n_layers, P, c.n_heads, c.prompt_len + n_img, c.head_dim), "k_cal")
+        sums = np.empty(c.n_layers * c.n_heads, np.float64)
+        self._check(self.lib.ssd_classify_partial(self._h, qp, kp, P, n_img, sums.ctypes.data, _stream()),
+                    "ssd_classify_partial")
+        return sums.reshape(c.n_layers, c.n_heads)
+
+    # -- hot path
+    def compress(self, layer: int, q_obs: Optional[torch.Tensor], k_full: torch.Tensor, v_full: torch.Tensor,
+                 n0: int, n_obs: Optional[int] = None):
+        c = self.cfg
+        n_obs = (0 if q_obs is None else q_obs.shape[2]) if n_obs is None else n_obs
+        qp = None if q_obs is None else _dev(q_obs, (c.n_seqs, c.n_heads, n_obs, c.head_dim), "q_obs")
+        kp = _dev(k_full, (c.n_seqs, c.n_heads, c.prompt_len + n0, c.head_dim), "k_full")
+        vp = _dev(v_full, (c.n_seqs, c.n_heads, c.prompt_len + n0, c.head_dim), "v_full")
+        self._check(self.lib.ssd_compress(self._h, layer, qp, kp, vp, n0, n_obs, _stream()), "ssd_compress")
+
+    def append(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor):
+        c = self.cfg
+        shp = (c.n_seqs, c.n_heads, c.head_dim)
+        self._check(self.lib.ssd_append(self._h, layer, _dev(k_new, shp, "k_new"), _dev(v_new, shp, "v_new"),
+                                        _stream()), "ssd_append")
+
+    def decode_attn(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        c = self.cfg
+        shp = (c.n_seqs, c.n_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
+        self._check(self.lib.ssd_decode_attn(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"), _stream()),
+                    "ssd_decode_attn")
+        return out
+
+    def step_host(self, layer: int, q_host, k_new_host, v_new_host, out_host):
+        """One append + decode of a layer from (pinned) host bf16 tensors; asynchronous."""
+        for t in (q_host, k_new_host, v_new_host, out_host):
+            assert (not t.is_cuda) and t.dtype == torch.bfloat16 and t.is_contiguous()
+        self._check(self.lib.ssd_step_host(self._h, layer, q_host.data_ptr(), k_new_host.data_ptr(),
+                                           v_new_host.data_ptr(), out_host.data_ptr(), _stream()), "ssd_step_host")
+
+    # -- inspection
+    def max_slots(self) -> int:
+        return int(self.lib.ssd_cache_max_slots(self._h))
+
+    def get_indices(self, layer: int) -> np.ndarray:
+        c = self.cfg
+        idx = np.empty((c.n_seqs, c.n_heads, self.max_slots()), np.int32)
+        self._check(self.lib.ssd_cache_get_indices(self._h, layer, idx.ctypes.data), "ssd_cache_get_indices")
+        return idx
+
+    def get_lengths(self, layer: int) -> np.ndarray:
+        ln = np.empty(self.cfg.n_heads, np.int32)
+        self._check(self.lib.ssd_cache_get_lengths(self._h, layer, ln.ctypes.data), "ssd_cache_get_lengths")
+        return ln
+
+    def get_labels(self) -> np.ndarray:
+        lab = np.empty(self.cfg.n_layers * self.cfg.n_heads, np.uint8)
+        self._check(self.lib.ssd_cache_get_labels(self._h, lab.ctypes.data), "ssd_cache_get_labels")
+        return lab.reshape(self.cfg.n_layers, self.cfg.n_heads)
+
+    def tokens(self, layer: int) -> int:
+        return int(self.lib.ssd_cache_tokens(self._h, layer))
+
+    def rewind(self, layer: int, t: int):
+        self._check(self.lib.ssd_cache_rewind(self._h, layer, t), "ssd_cache_rewind")
+
+    def kv_bytes_per_seq(self) -> int:
+        v = C.c_size_t(0)
+        self._check(self.lib.ssd_cache_kv_bytes(self._h, C.byref(v)), "ssd_cache_kv_bytes")
+        return int(v.value)

@@ -1,0 +1,462 @@
+// Host side of the C ABI: argument checking, the per-head variable-length layout, per-layer
+// state, and the sequencing of kernels.  No device memory is allocated here: everything lives in
+// the buffer the caller passed to ssd_cache_create.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "ssd_internal.cuh"
+
+namespace ssd {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Regions {
+  size_t desc, idx, counters, partial, score, staging, slab;  // byte offsets
+  size_t score_bytes, partial_bytes, front_bytes;
+};
+
+static bool config_ok(const ssd_config* c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->n_seqs < 1 || c->n_heads < 1 || c->n_heads > kMaxHeads) return false;
+  if (c->head_dim != kHeadDim) return false;
+  if (c->prompt_len < 0 || c->max_image_tokens < 1) return false;
+  if (c->window < 1 || c->sink_budget < 0 || c->sink_recent < 1) return false;
+  if (c->cls_window < 0) return false;
+  if (!(c->softmax_scale >= 0.f) || !std::isfinite(c->softmax_scale)) return false;
+  if (!std::isfinite(c->tau)) return false;
+  // keep every index in 32 bits with room to spare
+  const double slots = (double)c->prompt_len + std::fmax((double)c->window, (double)c->sink_budget + c->sink_recent);
+  if (slots * c->n_heads > 1.0e9 || (double)c->n_seqs * c->n_heads > 5.0e8) return false;
+  if ((double)c->prompt_len + c->max_image_tokens > 1.0e8) return false;
+  return true;
+}
+
+static Regions plan_regions(const ssd_config& c) {
+  Regions r;
+  size_t off = 0;
+  const size_t pairs_layer = (size_t)c.n_seqs * c.n_heads;
+  r.desc = off;      off = align_up(off + (size_t)c.n_layers * c.n_heads * sizeof(HeadDesc));
+  r.idx = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * (c.sink_budget > 0 ? c.sink_budget : 1) * 4);
+  r.counters = off;  off = align_up(off + pairs_layer * 4);
+  r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
+  r.partial = off;   off = align_up(off + r.partial_bytes);
+  r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
+  r.score = off;     off = align_up(off + r.score_bytes);
+  r.staging = off;   off = align_up(off + 4 * pairs_layer * kHeadDim * 2);
+  r.front_bytes = off;
+  r.slab = off;
+  return r;
+}
+
+}  // namespace ssd
+
+using namespace ssd;
+
+struct ssd_cache {
+  ssd_config cfg;
+  float scale;
+  char* base;
+  size_t bytes;
+  Regions reg;
+  bool labels_set;
+  std::vector<uint8_t> labels;        // [layers*H]
+  std::vector<HeadDesc> desc;         // [layers*H]
+  std::vector<int32_t> seq_slots;     // [layers]
+  std::vector<int64_t> layer_base;    // [layers] first slot of the layer in the slab
+  std::vector<int32_t> n_sink;        // [layers]
+  std::vector<int32_t> t_img, n0, prompt_valid, static_valid;  // [layers]
+
+  HeadDesc* d_desc(int layer) const { return reinterpret_cast<HeadDesc*>(base + reg.desc) + (size_t)layer * cfg.n_heads; }
+  int32_t* d_idx(int layer) const {
+    size_t per = (size_t)cfg.n_seqs * cfg.n_heads * (cfg.sink_budget > 0 ? cfg.sink_budget : 1);
+    return reinterpret_cast<int32_t*>(base + reg.idx) + (size_t)layer * per;
+  }
+  uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
+  float* d_partial() const { return reinterpret_cast<float*>(base + reg.partial); }
+  float* d_score() const { return reinterpret_cast<float*>(base + reg.score); }
+  char* d_staging() const { return base + reg.staging; }
+  uint4* d_slab(int layer) const { return reinterpret_cast<uint4*>(base + reg.slab) + (size_t)layer_base[layer] * kSlotU4; }
+  int max_slots() const {
+    int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
+    return cfg.prompt_len + (a > b ? a : b);
+  }
+  long valid_per_seq(int layer) const {
+    long v = 0;
+    for (int h = 0; h < cfg.n_heads; ++h) {
+      const HeadDesc& d = desc[(size_t)layer * cfg.n_heads + h];
+      v += prompt_valid[layer] + (d.w ? static_valid[layer] : 0) + (t_img[layer] < d.z ? t_img[layer] : d.z);
+    }
+    return v;
+  }
+};
+
+static size_t slab_slots_for(const ssd_config& c, long n_sink_total) {
+  const long heads_total = (long)c.n_layers * c.n_heads;
+  const size_t spatial = (size_t)c.prompt_len + c.window;
+  const size_t sink = (size_t)c.prompt_len + c.sink_budget + c.sink_recent;
+  if (n_sink_total < 0) return (size_t)heads_total * (spatial > sink ? spatial : sink) * c.n_seqs;
+  return ((size_t)n_sink_total * sink + (size_t)(heads_total - n_sink_total) * spatial) * c.n_seqs;
+}
+
+extern "C" {
+
+const char* ssd_status_string(int s) {
+  switch (s) {
+    case SSD_OK: return "SSD_OK";
+    case SSD_ERR_INVALID_ARG: return "SSD_ERR_INVALID_ARG";
+    case SSD_ERR_BAD_STATE: return "SSD_ERR_BAD_STATE";
+    case SSD_ERR_OVERFLOW: return "SSD_ERR_OVERFLOW";
+    case SSD_ERR_NO_MEM: return "SSD_ERR_NO_MEM";
+    case SSD_ERR_CUDA: return "SSD_ERR_CUDA";
+    default: return "SSD_ERR_UNKNOWN";
+  }
+}
+
+uint64_t ssd_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t ssd_cache_required_bytes(const ssd_config* cfg, int32_t n_sink_heads_total) {
+  if (!config_ok(cfg)) return 0;
+  if (n_sink_heads_total > cfg->n_layers * cfg->n_heads) return 0;
+  Regions r = plan_regions(*cfg);
+  return r.front_bytes + slab_slots_for(*cfg, n_sink_heads_total) * kSlotBytes;
+}
+
+int ssd_cache_create(const ssd_config* cfg, void* dev_mem, size_t dev_bytes, ssd_cache** out) {
+  if (!out) return SSD_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg) || !dev_mem) return SSD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dev_mem) % 256 != 0) return SSD_ERR_INVALID_ARG;
+  Regions r = plan_regions(*cfg);
+  // at least the all-spatial or all-semantic layout, whichever is smaller, must fit
+  size_t a = slab_slots_for(*cfg, 0), b = slab_slots_for(*cfg, (long)cfg->n_layers * cfg->n_heads);
+  if (dev_bytes < r.front_bytes + (a < b ? a : b) * kSlotBytes) return SSD_ERR_NO_MEM;
+  ssd_cache* c = new (std::nothrow) ssd_cache();
+  if (!c) return SSD_ERR_NO_MEM;
+  c->cfg = *cfg;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  c->base = static_cast<char*>(dev_mem);
+  c->bytes = dev_bytes;
+  c->reg = r;
+  c->labels_set = false;
+  const size_t nh = (size_t)cfg->n_layers * cfg->n_heads;
+  c->labels.assign(nh, 0);
+  c->desc.assign(nh, HeadDesc{0, 0, 0, 0});
+  c->seq_slots.assign(cfg->n_layers, 0);
+  c->layer_base.assign(cfg->n_layers, 0);
+  c->n_sink.assign(cfg->n_layers, 0);
+  c->t_img.assign(cfg->n_layers, 0);
+  c->n0.assign(cfg->n_layers, 0);
+  c->prompt_valid.assign(cfg->n_layers, 0);
+  c->static_valid.assign(cfg->n_layers, 0);
+  if (cudaMemset(c->base, 0, r.front_bytes) != cudaSuccess ||
+      cudaMemset(c->base + r.idx, 0xFF, r.counters - r.idx) != cudaSuccess ||
+      cudaDeviceSynchronize() != cudaSuccess) {
+    cudaGetLastError();
+    delete c;
+    return SSD_ERR_CUDA;
+  }
+  *out = c;
+  return SSD_OK;
+}
+
+int ssd_cache_free(ssd_cache* c) {
+  delete c;
+  return SSD_OK;
+}
+
+int ssd_set_head_labels(ssd_cache* c, const uint8_t* labels_host) {
+  if (!c || !labels_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  const size_t nh = (size_t)g.n_layers * g.n_heads;
+  long n_sink_total = 0;
+  for (size_t i = 0; i < nh; ++i) n_sink_total += labels_host[i] ? 1 : 0;
+  if (c->reg.front_bytes + slab_slots_for(g, n_sink_total) * kSlotBytes > c->bytes) return SSD_ERR_NO_MEM;
+  std::vector<HeadDesc> desc(nh);
+  int64_t base = 0;
+  for (int l = 0; l < g.n_layers; ++l) {
+    int off = 0, ns = 0;
+    for (int h = 0; h < g.n_heads; ++h) {
+      const bool sem = labels_host[(size_t)l * g.n_heads + h] != 0;
+      HeadDesc d;
+      d.x = off;
+      d.y = sem ? g.sink_budget : 0;
+      d.z = sem ? g.sink_recent : g.window;
+      d.w = sem ? 1 : 0;
+      desc[(size_t)l * g.n_heads + h] = d;
+      off += g.prompt_len + d.y + d.z;
+      ns += sem;
+    }
+    c->seq_slots[l] = off;
+    c->layer_base[l] = base;
+    c->n_sink[l] = ns;
+    base += (int64_t)off * g.n_seqs;
+  }
+  if (cudaMemcpy(c->base + c->reg.desc, desc.data(), nh * sizeof(HeadDesc), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  c->desc.swap(desc);
+  for (size_t i = 0; i < nh; ++i) c->labels[i] = labels_host[i] ? 1 : 0;
+  for (int l = 0; l < g.n_layers; ++l) c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = 0;
+  c->labels_set = true;
+  return SSD_OK;
+}
+
+int ssd_classify_partial(ssd_cache* c, const void* q_cal, const void* k_cal, int32_t n_cal_seqs, int32_t n_img,
+                         double* ratio_sums_host, void* stream) {
+  if (!c || !q_cal || !k_cal || !ratio_sums_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (n_cal_seqs < 1 || n_img < 1 || n_img > g.max_image_tokens) return SSD_ERR_INVALID_ARG;
+  const int rpb = classify_rows_per_block();
+  const int nrb = (n_img + rpb - 1) / rpb;
+  const size_t units = (size_t)g.n_layers * n_cal_seqs * g.n_heads;
+  if (units * nrb * sizeof(float) > c->reg.score_bytes || units * nrb > 0x7fffffffULL) return SSD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ClassifyParams p;
+  p.q_cal = static_cast<const __nv_bfloat16*>(q_cal);
+  p.k_cal = static_cast<const __nv_bfloat16*>(k_cal);
+  p.ratio_part = c->d_score();
+  p.n_units = (int)units;
+  p.L = g.prompt_len;
+  p.N = n_img;
+  p.w = g.cls_window;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  if (launch_classify(p, nrb, st) != cudaSuccess) return SSD_ERR_CUDA;
+  std::vector<float> part(units * nrb);
+  if (cudaMemcpyAsync(part.data(), c->d_score(), part.size() * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  for (int l = 0; l < g.n_layers; ++l)
+    for (int h = 0; h < g.n_heads; ++h) {
+      double acc = 0.0;
+      for (int pp = 0; pp < n_cal_seqs; ++pp) {
+        const size_t unit = ((size_t)l * n_cal_seqs + pp) * g.n_heads + h;
+        for (int rb = 0; rb < nrb; ++rb) acc += (double)part[unit * nrb + rb];
+      }
+      ratio_sums_host[(size_t)l * g.n_heads + h] = acc;
+    }
+  return SSD_OK;
+}
+
+int ssd_classify_heads(ssd_cache* c, const void* q_cal, const void* k_cal, int32_t n_cal_seqs, int32_t n_img,
+                       float* s_out_host, uint8_t* labels_out_host, void* stream) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  const size_t nh = (size_t)c->cfg.n_layers * c->cfg.n_heads;
+  std::vector<double> sums(nh);
+  int rc = ssd_classify_partial(c, q_cal, k_cal, n_cal_seqs, n_img, sums.data(), stream);
+  if (rc != SSD_OK) return rc;
+  std::vector<uint8_t> lab(nh);
+  for (size_t i = 0; i < nh; ++i) {
+    const float s = (float)(sums[i] / ((double)n_cal_seqs * (double)n_img));
+    if (s_out_host) s_out_host[i] = s;
+    lab[i] = s > c->cfg.tau ? 1 : 0;   // equality is spatial
+  }
+  rc = ssd_set_head_labels(c, lab.data());
+  if (rc != SSD_OK) return rc;
+  if (labels_out_host) std::memcpy(labels_out_host, lab.data(), nh);
+  return SSD_OK;
+}
+
+int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_full, const void* v_full, int32_t n0,
+                 int32_t n_obs, void* stream) {
+  if (!c || !k_full || !v_full) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (n0 < 0 || n0 > g.max_image_tokens || n_obs < 0 || n_obs > n0) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (g.prompt_len + n0 < 1) return SSD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_cand = n0 - g.sink_recent > 0 ? n0 - g.sink_recent : 0;
+  const int sv = g.sink_budget < n_cand ? g.sink_budget : n_cand;
+  const bool select = c->n_sink[layer] > 0 && sv > 0;
+  if (select && n_obs > 0 && !q_obs) return SSD_ERR_INVALID_ARG;
+  const HeadDesc* desc = c->d_desc(layer);
+  if (select) {
+    if (n_obs > 0) {
+      ScoreParams sp;
+      sp.q_obs = static_cast<const __nv_bfloat16*>(q_obs);
+      sp.k_full = static_cast<const __nv_bfloat16*>(k_full);
+      sp.desc = desc;
+      sp.score = c->d_score();
+      sp.n_seqs = g.n_seqs; sp.H = g.n_heads; sp.L = g.prompt_len; sp.n0 = n0; sp.n_obs = n_obs;
+      sp.scale_log2 = c->scale * 1.4426950408889634f;
+      if (launch_score(sp, st) != cudaSuccess) return SSD_ERR_CUDA;
+    } else {
+      if (cudaMemsetAsync(c->d_score(), 0, (size_t)g.n_seqs * g.n_heads * n0 * 4, st) != cudaSuccess) return SSD_ERR_CUDA;
+    }
+    SelectParams sl;
+    sl.score = c->d_score();
+    sl.desc = desc;
+    sl.static_idx = c->d_idx(layer);
+    sl.n_seqs = g.n_seqs; sl.H = g.n_heads; sl.M = g.sink_budget; sl.n0 = n0; sl.n_cand = n_cand;
+    if (launch_select(sl, st) != cudaSuccess) return SSD_ERR_CUDA;
+  }
+  GatherParams gp;
+  gp.slab = c->d_slab(layer);
+  gp.desc = desc;
+  gp.static_idx = c->d_idx(layer);
+  gp.k_full = static_cast<const uint4*>(k_full);
+  gp.v_full = static_cast<const uint4*>(v_full);
+  gp.n_seqs = g.n_seqs; gp.H = g.n_heads; gp.L = g.prompt_len; gp.M = g.sink_budget; gp.n0 = n0;
+  gp.static_valid = select ? sv : 0;
+  gp.seq_slots = c->seq_slots[layer];
+  if (launch_gather(gp, c->max_slots(), st) != cudaSuccess) return SSD_ERR_CUDA;
+  c->t_img[layer] = n0;
+  c->n0[layer] = n0;
+  c->prompt_valid[layer] = g.prompt_len;
+  c->static_valid[layer] = select ? sv : 0;
+  return SSD_OK;
+}
+
+int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new, void* stream) {
+  if (!c || !k_new || !v_new) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  AppendParams p;
+  p.slab = c->d_slab(layer);
+  p.desc = c->d_desc(layer);
+  p.k_new = static_cast<const uint4*>(k_new);
+  p.v_new = static_cast<const uint4*>(v_new);
+  p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
+  p.j = c->t_img[layer];
+  p.seq_slots = c->seq_slots[layer];
+  if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  c->t_img[layer] += 1;
+  return SSD_OK;
+}
+
+int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void* stream) {
+  if (!c || !q || !out) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
+  DecodeParams p;
+  p.slab = c->d_slab(layer);
+  p.desc = c->d_desc(layer);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.partial = c->d_partial();
+  p.counters = c->d_counters();
+  p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
+  p.prompt_valid = c->prompt_valid[layer];
+  p.static_valid = c->static_valid[layer];
+  p.t_img = c->t_img[layer];
+  p.seq_slots = c->seq_slots[layer];
+  p.n_workers = 0;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  const long total = c->valid_per_seq(layer) * g.n_seqs;
+  if (launch_decode(p, total, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  return SSD_OK;
+}
+
+int ssd_step_host(ssd_cache* c, int32_t layer, const void* q_host, const void* k_new_host, const void* v_new_host,
+                  void* out_host, void* stream) {
+  if (!c || !q_host || !k_new_host || !v_new_host || !out_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t nb = (size_t)g.n_seqs * g.n_heads * kHeadDim * 2;
+  char* s = c->d_staging();
+  if (cudaMemcpyAsync(s, q_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(s + nb, k_new_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(s + 2 * nb, v_new_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  int rc = ssd_append(c, layer, s + nb, s + 2 * nb, stream);
+  if (rc != SSD_OK) return rc;
+  rc = ssd_decode_attn(c, layer, s, s + 3 * nb, stream);
+  if (rc != SSD_OK) return rc;
+  if (cudaMemcpyAsync(out_host, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  return SSD_OK;
+}
+
+int32_t ssd_cache_max_slots(const ssd_cache* c) { return c ? c->max_slots() : -1; }
+
+int ssd_cache_get_indices(ssd_cache* c, int32_t layer, int32_t* idx_host) {
+  if (!c || !idx_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  const int ms = c->max_slots(), M = g.sink_budget;
+  std::vector<int32_t> sidx((size_t)g.n_seqs * g.n_heads * (M > 0 ? M : 1));
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(sidx.data(), c->d_idx(layer), sidx.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  const int t = c->t_img[layer], L = g.prompt_len;
+  for (int s = 0; s < g.n_seqs; ++s)
+    for (int h = 0; h < g.n_heads; ++h) {
+      const HeadDesc& d = c->desc[(size_t)layer * g.n_heads + h];
+      int32_t* o = idx_host + ((size_t)s * g.n_heads + h) * ms;
+      for (int i = 0; i < ms; ++i) o[i] = -1;
+      for (int i = 0; i < c->prompt_valid[layer]; ++i) o[i] = i;
+      if (d.w)
+        for (int m = 0; m < c->static_valid[layer]; ++m) {
+          int j = sidx[((size_t)s * g.n_heads + h) * (M > 0 ? M : 1) + m];
+          o[L + m] = j >= 0 ? L + j : -1;
+        }
+      for (int r = 0; r < d.z; ++r)
+        if (t - 1 >= r) o[L + d.y + r] = L + ((t - 1 - r) / d.z) * d.z + r;
+    }
+  return SSD_OK;
+}
+
+int ssd_cache_get_lengths(ssd_cache* c, int32_t layer, int32_t* len_host) {
+  if (!c || !len_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  for (int h = 0; h < g.n_heads; ++h) {
+    const HeadDesc& d = c->desc[(size_t)layer * g.n_heads + h];
+    len_host[h] = c->prompt_valid[layer] + (d.w ? c->static_valid[layer] : 0) +
+                  (c->t_img[layer] < d.z ? c->t_img[layer] : d.z);
+  }
+  return SSD_OK;
+}
+
+int ssd_cache_get_labels(ssd_cache* c, uint8_t* labels_host) {
+  if (!c || !labels_host) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  std::memcpy(labels_host, c->labels.data(), c->labels.size());
+  return SSD_OK;
+}
+
+int32_t ssd_cache_tokens(const ssd_cache* c, int32_t layer) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return -1;
+  return c->t_img[layer];
+}
+
+int ssd_cache_rewind(ssd_cache* c, int32_t layer, int32_t t) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return SSD_ERR_INVALID_ARG;
+  if (t < c->n0[layer] || t > c->t_img[layer]) return SSD_ERR_INVALID_ARG;
+  c->t_img[layer] = t;
+  return SSD_OK;
+}
+
+int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
+  if (!c || !bytes_per_seq) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  size_t slots = 0;
+  for (int l = 0; l < c->cfg.n_layers; ++l) slots += (size_t)c->seq_slots[l];
+  *bytes_per_seq = slots * kSlotBytes;
+  return SSD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of the SSD B200 library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "ssd_b200.h"
+
+namespace ssd {
+
+constexpr int kHeadDim = 128;
+constexpr int kSlotBytes = 512;          // one token of one head: K row (256 B) then V row (256 B)
+constexpr int kSlotU4 = kSlotBytes / 16; // 32 uint4 per slot
+constexpr int kMaxHeads = 128;
+constexpr int kPartialFloats = 132;      // m, l, 2 pad, acc[128]
+
+// Per (layer, head) layout record, resident in device memory.
+//   x = slot offset of the head inside one sequence's block of the layer
+//   y = static capacity (M for semantic heads, 0 for spatial)
+//   z = ring capacity (R for semantic heads, W for spatial)
+//   w = 1 for semantic heads
+typedef int4 HeadDesc;
+
+struct DecodeParams {
+  const uint4* slab;        // first slot of the layer
+  const HeadDesc* desc;     // [H] records of the layer
+  const __nv_bfloat16* q;   // [n_seqs, H, 128]
+  __nv_bfloat16* out;       // [n_seqs, H, 128]
+  float* partial;           // [n_workers * 2, kPartialFloats]
+  uint32_t* counters;       // [n_seqs * H], zero between launches
+  int n_seqs, H, L;
+  int prompt_valid;         // 0 or L
+  int static_valid;         // valid static slots of semantic heads
+  int t_img;                // image tokens held (ring_valid = min(t_img, ring_cap))
+  int seq_slots;            // physical slots per sequence in this layer
+  int n_workers;            // warps that take a share of the work
+  float scale_log2;         // softmax scale * log2(e)
+};
+
+struct AppendParams {
+  uint4* slab;
+  const HeadDesc* desc;
+  const uint4* k_new;       // [n_seqs, H, 16] uint4
+  const uint4* v_new;
+  int n_seqs, H, L;
+  int j;                    // image index of the token being appended
+  int seq_slots;
+};
+
+struct GatherParams {
+  uint4* slab;
+  const HeadDesc* desc;
+  const int32_t* static_idx; // [n_seqs, H, M] image indices, ascending, -1 padded
+  const uint4* k_full;       // [n_seqs, H, L + n0, 16] uint4
+  const uint4* v_full;
+  int n_seqs, H, L, M, n0;
+  int static_valid;
+  int seq_slots;
+};
+
+struct ScoreParams {
+  const __nv_bfloat16* q_obs;  // [n_seqs, H, n_obs, 128]
+  const __nv_bfloat16* k_full; // [n_seqs, H, L + n0, 128]
+  const HeadDesc* desc;
+  float* score;                // [n_seqs, H, n0]
+  int n_seqs, H, L, n0, n_obs;
+  float scale_log2;
+};
+
+struct SelectParams {
+  const float* score;          // [n_seqs, H, n0]
+  const HeadDesc* desc;
+  int32_t* static_idx;         // [n_seqs, H, M]
+  int n_seqs, H, M, n0, n_cand;
+};
+
+struct ClassifyParams {
+  const __nv_bfloat16* q_cal;  // [n_units, N, 128], unit = (layer, p, head)
+  const __nv_bfloat16* k_cal;  // [n_units, L + N, 128]
+  float* ratio_part;           // [n_units, n_row_blocks]
+  int n_units, L, N, w;
+  float scale_log2;
+};
+
+cudaError_t launch_decode(const DecodeParams& p, long total_valid, cudaStream_t st);
+cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
+cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
+cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
+cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st);
+int classify_rows_per_block();
+int decode_max_workers();
+
+void count_launch(int n = 1);
+
+}  // namespace ssd

@@ -1,0 +1,195 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_18716_b200 import binding as B
+from paper_2510_18716_b200 import workloads as wl
+
+from parity_util import check_outputs, run_workload
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_every_step():
+    cfg = wl.CONFIGS["tiny"]
+    r = run_workload(cfg, [0], [0], check_steps=(), full_every_step=True, check_planted=True)
+    assert r.steps_checked == cfg.n_img - cfg.n0 and r.n_pairs == 8
+
+
+def test_tiny_fewer_observation_queries():
+    cfg = wl.CONFIGS["tiny"]
+    for n_obs in (1, 5, 0):
+        run_workload(cfg, [0], [0], check_steps=(cfg.n0 + 1, cfg.n_img), classify=False, n_obs=n_obs)
+
+
+def test_janus1b_sampled_layers_all_sequences():
+    cfg = wl.CONFIGS["janus1b"]
+    steps = (cfg.n0 + 1, cfg.n0 + 2, cfg.n0 + 25, cfg.n_img)
+    r = run_workload(cfg, [0, 23], list(range(cfg.n_seqs)), steps, check_planted=True)
+    assert r.steps_checked == 2 * len(steps)
+
+
+def test_janus7b_sampled_layers_all_sequences():
+    cfg = wl.CONFIGS["janus7b"]
+    steps = (cfg.n0 + 1, cfg.n0 + 24, cfg.n_img)
+    r = run_workload(cfg, [0, 29], list(range(cfg.n_seqs)), steps, check_planted=True)
+    assert r.steps_checked == 2 * len(steps)
+
+
+def test_hires7b_one_layer_two_sequences():
+    cfg = wl.CONFIGS["hires7b"]
+    steps = (cfg.n0 + 1, cfg.n0 + 65, cfg.n_img)
+    run_workload(cfg, [0], [0, 1], steps, classify=False)
+
+
+def test_sweep_points():
+    for cfg, seqs in ((wl.sweep(32, 5, 0.25), [0, 1, 2, 3]), (wl.sweep(32, 10, 0.75), [0, 1]),
+                      (wl.sweep(32, 2, 0.5), [5, 6])):
+        run_workload(cfg, [3], seqs, (cfg.n0 + 1, cfg.n0 + 30, cfg.n_img), classify=False)
+
+
+def _full_cache_case(cfg: wl.Workload, seqs, steps):
+    """Uncompressed baseline: every head spatial with W = N, prompt loaded with n0 = 0."""
+    dev = torch.device("cuda:0")
+    L, N, H, S = cfg.prompt_len, cfg.n_img, cfg.n_heads, len(seqs)
+    c = B.make_config(1, S, H, L, N, N, 0, 1, cfg.cls_window, cfg.tau)
+    cache = B.SsdCache(c)
+    cache.set_head_labels(np.zeros(H, np.uint8))
+    q, k, v, _ = wl.gen_layer(cfg, 0, seqs, device=dev)
+    qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
+    cache.compress(0, None, k[:, :, :L].contiguous(), v[:, :, :L].contiguous(), 0, 0)
+    sem = np.zeros((S, H), np.uint8)
+    for t in range(1, N + 1):
+        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
+        if t in steps:
+            out = cache.decode_attn(0, q[:, :, t - 1].contiguous())
+            want = oracle.decode_batch(qu[:, :, t - 1], ku, vu, sem, None, None, L, t, N, 0, 1, full=True)
+            check_outputs(out, want, f"full cache step {t}")
+            assert (cache.get_lengths(0) == L + t).all()
+    cache.close()
+
+
+def test_full_cache_baseline_matches_full_attention():
+    _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65))
+    _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576))
+
+
+def _small_cfg(seed):
+    rng = np.random.default_rng(seed)
+    h = int(rng.integers(2, 7))
+    w = int(rng.integers(2, 7))
+    N = h * w
+    H = int(rng.integers(1, 6))
+    n0 = int(rng.integers(0, N))
+    return wl.Workload(f"rand{seed}", 1, int(rng.integers(1, 4)), H, int(rng.integers(0, 6)), (h, w),
+                       int(rng.integers(1, N + 2)), int(rng.integers(0, N + 2)), int(rng.integers(1, 6)),
+                       int(rng.integers(0, 8)), int(rng.integers(0, H + 1)), n0, 1, 1.0, seed=seed)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_small_shapes(seed):
+    cfg = _small_cfg(seed)
+    if cfg.prompt_len + cfg.n0 == 0:
+        pytest.skip("nothing to load")
+    run_workload(cfg, [0], list(range(cfg.n_seqs)), (), classify=False, full_every_step=True,
+                 n_obs=min(cfg.n0, seed % 5 + (cfg.n0 if seed % 2 else 0)))
+
+
+def test_decode_before_any_compress_fills_ring_from_zero():
+    cfg = wl.CONFIGS["tiny"]
+    dev = torch.device("cuda:0")
+    L, N, H = cfg.prompt_len, cfg.n_img, cfg.n_heads
+    cache = B.SsdCache(B.config_from_workload(cfg))
+    labels = wl.sink_mask(cfg, 0)
+    cache.set_head_labels(labels)
+    q, k, v, _ = wl.gen_layer(cfg, 0, [0], device=dev)
+    qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
+    with pytest.raises(B.SsdError) as e:
+        cache.decode_attn(0, q[:, :, 0].contiguous())
+    assert e.value.code == B.SSD_ERR_BAD_STATE
+    sem = labels[None, :]
+    for t in range(1, N + 1):
+        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
+        out = cache.decode_attn(0, q[:, :, t - 1].contiguous())
+        # no prompt, no static set: windows over image tokens only
+        want = np.empty((1, H, 128))
+        for h in range(H):
+            capn = cfg.sink_recent if labels[h] else cfg.window
+            pos = np.arange(max(0, t - capn), t, dtype=np.int32) + L
+            want[0, h] = oracle.attend(qu[0, h, t - 1], ku[0, h], vu[0, h], pos)
+        check_outputs(out, want, f"ring-only step {t}")
+    with pytest.raises(B.SsdError) as e:
+        cache.append(0, k[:, :, L].contiguous(), v[:, :, L].contiguous())
+    assert e.value.code == B.SSD_ERR_OVERFLOW
+    cache.close()
+
+
+def test_classifier_scores_match_oracle_on_mixed_heads():
+    # sparsity values themselves (not only labels), on data with no planted structure
+    cfg = wl.Workload("cls", 2, 2, 5, 7, (6, 9), 8, 8, 4, 11, 0, 20, 3, 1.2, seed=7)
+    dev = torch.device("cuda:0")
+    qc, kc = wl.gen_calibration(cfg, [0, 1], device=dev)
+    cache = B.SsdCache(B.config_from_workload(cfg))
+    s_gpu, lab = cache.classify_heads(qc, kc)
+    s_ora = oracle.sparsity(wl.to_u16(qc), wl.to_u16(kc), cfg.prompt_len, cfg.cls_window)
+    assert np.allclose(s_gpu, s_ora, rtol=2e-4, atol=2e-5)
+    sums = cache.classify_partial(qc[:, :2].contiguous(), kc[:, :2].contiguous())
+    s2 = oracle.sparsity(wl.to_u16(qc[:, :2]), wl.to_u16(kc[:, :2]), cfg.prompt_len, cfg.cls_window)
+    assert np.allclose(sums / (2 * cfg.n_img), s2, rtol=2e-4, atol=2e-5)
+    cache.close()
+
+
+def test_step_host_matches_device_path():
+    cfg = wl.CONFIGS["tiny"]
+    dev = torch.device("cuda:0")
+    L, n0 = cfg.prompt_len, cfg.n0
+    q, k, v, _ = wl.gen_layer(cfg, 0, [0], device=dev)
+    outs = []
+    for mode in ("device", "host"):
+        cache = B.SsdCache(B.config_from_workload(cfg))
+        cache.set_head_labels(wl.sink_mask(cfg, 0))
+        cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        res = []
+        for t in range(n0 + 1, n0 + 6):
+            qt, kt, vt = (x.contiguous() for x in (q[:, :, t - 1], k[:, :, L + t - 1], v[:, :, L + t - 1]))
+            if mode == "device":
+                cache.append(0, kt, vt)
+                res.append(cache.decode_attn(0, qt).cpu())
+            else:
+                hq, hk, hv = (x.cpu().pin_memory() for x in (qt, kt, vt))
+                ho = torch.empty_like(hq).pin_memory()
+                cache.step_host(0, hq, hk, hv, ho)
+                torch.cuda.synchronize()
+                res.append(ho.clone())
+        outs.append(res)
+        cache.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_argument_errors_launch_nothing():
+    cfg = B.make_config(2, 2, 4, 8, 16, 4, 4, 2)
+    cache = B.SsdCache(cfg)
+    dev = torch.device("cuda:0")
+    x = torch.zeros((2, 4, 128), dtype=torch.bfloat16, device=dev)
+    before = B.kernel_launch_count()
+    for fn in (lambda: cache.append(0, x, x), lambda: cache.decode_attn(0, x)):
+        with pytest.raises(B.SsdError) as e:
+            fn()
+        assert e.value.code == B.SSD_ERR_BAD_STATE          # no labels yet
+    cache.set_head_labels(np.array([0, 1, 0, 1, 1, 1, 0, 0], np.uint8))
+    for layer in (-1, 2):
+        with pytest.raises(B.SsdError) as e:
+            cache.append(layer, x, x)
+        assert e.value.code == B.SSD_ERR_INVALID_ARG
+    kf = torch.zeros((2, 4, 8 + 17, 128), dtype=torch.bfloat16, device=dev)
+    with pytest.raises(B.SsdError) as e:
+        cache.compress(0, None, kf, kf, 17, 0)               # n0 beyond max_image_tokens
+    assert e.value.code == B.SSD_ERR_INVALID_ARG
+    assert B.kernel_launch_count() == before
+    assert cache.kv_bytes_per_seq() == ((8 + 4) * 4 + (8 + 6) * 4) * 512
+    cache.close()
+    bad = B.make_config(1, 1, 1, 0, 4, 1, 1, 1, head_dim=64)
+    assert B.required_bytes(bad) == 0
