@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the SSD decode hot path (append + decode attention over every layer, per step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload janus7b] [--impl reference]
+
+Prints ONE JSON line.  A "step" is one decoded image token for every sequence: for each layer,
+ssd_append of the new K/V then ssd_decode_attn.  `value` is decoded image tokens per second
+(one per CFG pair per step) over the whole job with inputs resident in HBM; `e2e` is the same
+through ssd_step_host with pinned HOST buffers (copies inside the timed region).  Under torchrun
+each rank owns its own block of sequences (weak scaling, no data-path collective); time is the max
+over ranks.  `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_18716_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decoded image tokens/sec (attention+cache ops)"
+UNIT = "image tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                d = json.load(f)
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_sample(cfg: wl.Workload, layers, n_steps, device):
+    """Inputs (host, bf16 bits) and the oracle's own selection for a bounded sample of the workload."""
+    import oracle
+    L, n0 = cfg.prompt_len, cfg.n0
+    seqs = list(range(cfg.n_seqs))
+    data = []
+    for layer in layers:
+        q, k, v, _ = wl.gen_layer(cfg, layer, seqs, device=device)
+        sem = wl.sink_mask(cfg, layer)[None, :].repeat(len(seqs), 0)
+        qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
+        _, idx, cnt = oracle.select_batch(qu[:, :, :n0], ku[:, :, : L + n0], sem, L, n0, cfg.sink_budget,
+                                          cfg.sink_recent)
+        data.append((qu, ku, vu, sem, idx, cnt))
+    return data
+
+
+def oracle_time_steps(cfg: wl.Workload, data, t_first, n_steps):
+    """Seconds the oracle needs for n_steps decode steps over the sampled layers."""
+    import oracle
+    L = cfg.prompt_len
+    t0 = time.perf_counter()
+    for i in range(n_steps):
+        t = t_first + i
+        for (qu, ku, vu, sem, idx, cnt) in data:
+            oracle.decode_batch(np.ascontiguousarray(qu[:, :, t - 1]), ku, vu, sem, idx, cnt, L, t, cfg.window,
+                                cfg.sink_budget, cfg.sink_recent)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, cfg):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    layers = sorted({0, cfg.n_layers - 1})
+    data = oracle_sample(cfg, layers, 0, "cuda" if torch.cuda.is_available() else "cpu")
+    scale = cfg.n_layers / len(layers)
+    for _ in range(args.warmup):
+        oracle_time_steps(cfg, data, cfg.n0 + 1, 1)
+    secs = oracle_time_steps(cfg, data, cfg.n0 + 1, args.steps)
+    ms_per_step = secs / args.steps * scale * 1e3
+    value = cfg.images_per_step / (ms_per_step * 1e-3)
+    sample = (f"decode attention of layers {layers} (of {cfg.n_layers}) x all {cfg.n_seqs} sequences x "
+              f"{cfg.n_heads} heads per step, time scaled by {scale:g} (extrapolated)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "n_layers": cfg.n_layers, "n_seqs": cfg.n_seqs, "n_heads": cfg.n_heads,
+                   "prompt_len": cfg.prompt_len, "image_tokens": cfg.n_img, "window": cfg.window,
+                   "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0):
+    """Create, classify, load and compress every layer; returns the cache and per-layer step inputs."""
+    from paper_2510_18716_b200 import binding as B
+    from paper_2510_18716_b200 import dist as D
+    L, N, n0, H, S = cfg.prompt_len, cfg.n_img, cfg.n0, cfg.n_heads, cfg.n_seqs
+    if full_cache:
+        ccfg = B.make_config(cfg.n_layers, S, H, L, N, N, 0, 1, cfg.cls_window, cfg.tau)
+        cache = B.SsdCache(ccfg, n_sink_heads_total=0, device=device)
+        cache.set_head_labels(np.zeros(cfg.n_layers * H, np.uint8))
+    else:
+        ccfg = B.config_from_workload(cfg)
+        cache = B.SsdCache(ccfg, n_sink_heads_total=cfg.n_layers * cfg.n_sink_heads, device=device)
+        mine = D.shard_calibration(cfg.n_cal, rank, world)
+        qs, ks = [], []
+        for layer in range(cfg.n_layers):
+            if mine:
+                q, k, _, _ = wl.gen_layer(cfg, layer, [wl.CAL_SEQ_BASE + p for p in mine], device=device)
+                qs.append(q)
+                ks.append(k)
+        qc = torch.stack(qs) if mine else None
+        kc = torch.stack(ks) if mine else None
+        labels = D.classify_sharded(cache, qc, kc, cfg.n_cal, N, cfg.tau)
+        want = np.stack([wl.sink_mask(cfg, l) for l in range(cfg.n_layers)])
+        if not np.array_equal(labels, want):
+            raise RuntimeError("classifier did not recover the generator's head split")
+        del qc, kc, qs, ks
+    steps_in = []
+    seqs = list(range(seq_lo, seq_lo + S))
+    for layer in range(cfg.n_layers):
+        q, k, v, _ = wl.gen_layer(cfg, layer, seqs, device=device)
+        if full_cache:
+            cache.compress(layer, None, k[:, :, :L].contiguous(), v[:, :, :L].contiguous(), 0, 0)
+            # bulk-append the first n0 tokens so both caches sit at the same image step
+            for j in range(n0):
+                cache.append(layer, k[:, :, L + j].contiguous(), v[:, :, L + j].contiguous())
+        else:
+            cache.compress(layer, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(),
+                           v[:, :, : L + n0].contiguous(), n0)
+        T = min(t_steps, N - n0)
+        steps_in.append((q[:, :, n0:n0 + T].permute(2, 0, 1, 3).contiguous(),
+                         k[:, :, L + n0:L + n0 + T].permute(2, 0, 1, 3).contiguous(),
+                         v[:, :, L + n0:L + n0 + T].permute(2, 0, 1, 3).contiguous()))
+        del q, k, v
+    torch.cuda.synchronize()
+    return cache, steps_in
+
+
+class Stepper:
+    """Replays decode steps n0+1.. over all layers, wrapping back to n0 when the grid is full."""
+
+    def __init__(self, cfg, cache, steps_in, out):
+        self.cfg, self.cache, self.steps_in, self.out = cfg, cache, steps_in, out
+        self.i = 0
+        self.T = steps_in[0][0].shape[0]
+
+    def step(self, append=True, decode=True):
+        if self.i == self.T:
+            for layer in range(self.cfg.n_layers):
+                self.cache.rewind(layer, self.cfg.n0)
+            self.i = 0
+        i = self.i
+        for layer in range(self.cfg.n_layers):
+            q, k, v = self.steps_in[layer]
+            if append:
+                self.cache.append(layer, k[i], v[i])
+            if decode:
+                self.cache.decode_attn(layer, q[i], self.out)
+        self.i += 1
+
+
+def timed(fn, n, barrier):
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args, cfg):
+    from paper_2510_18716_b200 import binding as B
+    import torch.distributed as dist
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    B.load()
+    K, W = args.steps, args.warmup
+    S, H, N, n0 = cfg.n_seqs, cfg.n_heads, cfg.n_img, cfg.n0
+    cache, steps_in = build_cache(cfg, device, rank * S, rank, world, t_steps=K + W)
+    out = torch.empty((S, H, 128), dtype=torch.bfloat16, device=device)
+    stepper = Stepper(cfg, cache, steps_in, out)
+
+    # ---- device-resident timing (the headline `value`)
+    for _ in range(W):
+        stepper.step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    cache.profile_enable(K * cfg.n_layers)
+    l0 = B.kernel_launch_count()
+    ms = timed(stepper.step, K, barrier)
+    launches = B.kernel_launch_count() - l0
+    dec_ms = cache.profile_collect()
+    cache.profile_enable(0)
+    clocks = sampler.stop()
+    ms = max_over_ranks(ms)
+    ms_per_step = ms / K
+    value = cfg.images_per_step * world / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel (decode): algorithmic bytes per launch / mean launch time
+    slots_layer = int(sum(int(cache.get_lengths(l).sum()) for l in range(cfg.n_layers))) / cfg.n_layers
+    bytes_launch = S * (slots_layer * 512 + H * 2 * 256)       # K+V rows, plus q in and out
+    peak, peak_kind = measured_peaks()
+    dec_mean_ms = float(np.mean(dec_ms)) if len(dec_ms) else float("nan")
+    achieved = bytes_launch / (dec_mean_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "bytes_per_launch": bytes_launch, "launch_ms_mean": dec_mean_ms,
+                "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
+                "launches_timed": int(len(dec_ms)), "frac_of_8TBs_nominal": achieved / 8000.0,
+                "step_gbs": bytes_launch * cfg.n_layers / (ms_per_step * 1e-3) / 1e9}
+
+    # ---- end to end: the same step through ssd_step_host with pinned host buffers
+    pool = 4
+    hq = [[steps_in[l][0][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
+    hk = [[steps_in[l][1][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
+    hv = [[steps_in[l][2][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
+    ho = [torch.empty((S, H, 128), dtype=torch.bfloat16).pin_memory() for _ in range(cfg.n_layers)]
+    state = {"i": 0}
+
+    def host_step():
+        if cache.tokens(0) >= N:
+            for layer in range(cfg.n_layers):
+                cache.rewind(layer, n0)
+        i = state["i"] % pool
+        for layer in range(cfg.n_layers):
+            cache.step_host(layer, hq[layer][i], hk[layer][i], hv[layer][i], ho[layer])
+        state["i"] += 1
+
+    Ke = max(4, min(K, 16))
+    for _ in range(3):
+        host_step()
+    ms_e = max_over_ranks(timed(host_step, Ke, barrier))
+    e2e_val = cfg.images_per_step * world / (ms_e / Ke * 1e-3)
+    tensor_bytes = S * H * 128 * 2
+    e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 3 * tensor_bytes * cfg.n_layers,
+           "d2h_bytes_per_step": tensor_bytes * cfg.n_layers, "steps": Ke, "ms_per_step": ms_e / Ke}
+
+    kv_bytes_per_seq = cache.kv_bytes_per_seq()
+    cache.close()
+    del cache, steps_in, stepper
+    torch.cuda.empty_cache()
+
+    # ---- same library, uncompressed full cache (every head keeps everything)
+    full = None
+    if not args.no_full_cache:
+        Kf = max(2, min(K, 8))
+        fcache, fsteps = build_cache(cfg, device, rank * S, rank, world, full_cache=True, t_steps=Kf + 3)
+        fst = Stepper(cfg, fcache, fsteps, out)
+        for _ in range(3):
+            fst.step()
+        ms_f = max_over_ranks(timed(fst.step, Kf, barrier))
+        t_mid = n0 + 3 + (Kf + 1) / 2
+        fbytes = cfg.n_layers * S * H * ((cfg.prompt_len + t_mid) * 512 + 512)
+        full = {"value": cfg.images_per_step * world / (ms_f / Kf * 1e-3), "unit": UNIT, "ms_per_step": ms_f / Kf,
+                "steps": Kf, "image_step": t_mid, "gbs": fbytes / (ms_f / Kf * 1e-3) / 1e9,
+                "kv_bytes_per_seq": fcache.kv_bytes_per_seq()}
+        fcache.close()
+        del fcache, fsteps, fst
+        torch.cuda.empty_cache()
+
+    # ---- CPU oracle on the host cores (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        layers = sorted({0, cfg.n_layers - 1})
+        data = oracle_sample(cfg, layers, 0, device)
+        oracle_time_steps(cfg, data, n0 + 1, 1)
+        n_cpu = 4
+        secs = oracle_time_steps(cfg, data, n0 + 1, n_cpu)
+        scale = cfg.n_layers / len(layers)
+        cpu_ms = secs / n_cpu * scale * 1e3
+        cpu = {"value": cfg.images_per_step / (cpu_ms * 1e-3), "unit": UNIT, "cores": oracle.threads(),
+               "kind": "oracle", "ms_per_step": cpu_ms,
+               "sample": (f"{n_cpu} decode steps over layers {layers} of {cfg.n_layers}, all {S} sequences x {H} "
+                          f"heads; time scaled by {scale:g} (extrapolated)")}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "n_layers": cfg.n_layers, "n_seqs_per_gpu": S, "n_heads": H,
+                       "prompt_len": cfg.prompt_len, "image_tokens": N, "compressed_at": n0, "window": cfg.window,
+                       "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent,
+                       "sink_heads_per_layer": cfg.n_sink_heads, "kv_dtype": "bf16", "parallelism": f"sequence-sharded x{world}",
+                       "l2": "inputs larger than L2 (each layer's slab is >126 MB and is touched once per step)",
+                       "kv_bytes_per_seq": kv_bytes_per_seq},
+            "sequence_tokens_per_s": value * 2 if S > 1 else value,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "cpu_baseline": cpu, "full_cache": full,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="janus7b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (small profiling case)")
+    ap.add_argument("--no-full-cache", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = wl.CONFIGS[args.workload]
+    if args.layers > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n_layers=min(args.layers, cfg.n_layers), name=f"{cfg.name}[:{args.layers} layers]")
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

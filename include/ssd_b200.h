@@ -152,6 +152,14 @@ int ssd_cache_rewind(ssd_cache *cache, int32_t layer, int32_t t);
 /* K+V bytes the cache holds per sequence over all layers at full occupancy (slots * 512 B). */
 int ssd_cache_kv_bytes(ssd_cache *cache, size_t *bytes_per_seq);
 
+/* Device-side timing of decode launches, for measurement.  ssd_profile_enable creates CUDA events
+ * for up to max_launches launches (0 switches timing off); while enabled, every ssd_decode_attn
+ * records an event before and after its kernel on the caller's stream.  ssd_profile_collect waits
+ * for the recorded launches, writes their durations in milliseconds to ms_host (room for
+ * max_launches floats), their number to *n_out, and starts over.  No paper counterpart. */
+int ssd_profile_enable(ssd_cache *cache, int32_t max_launches);
+int ssd_profile_collect(ssd_cache *cache, float *ms_host, int32_t *n_out);
+
 /* Number of kernels this library has launched since the process started (for audit). */
 uint64_t ssd_kernel_launch_count(void);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "ssd_classify_heads", "ssd_classify_partial", "ssd_set_head_labels", "ssd_compress", "ssd_append",
     "ssd_decode_attn", "ssd_step_host", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
-    "ssd_cache_kv_bytes", "ssd_kernel_launch_count",
+    "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
 ]
 
 
@@ -83,6 +83,8 @@ def load():
     L.ssd_cache_tokens.restype = i32
     L.ssd_cache_rewind.argtypes = [vp, i32, i32]
     L.ssd_cache_kv_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.ssd_profile_enable.argtypes = [vp, i32]
+    L.ssd_profile_collect.argtypes = [vp, vp, C.POINTER(i32)]
     L.ssd_kernel_launch_count.argtypes = []
     L.ssd_kernel_launch_count.restype = u64
     for n in EXPORTS:
@@ -250,6 +252,16 @@ class SsdCache:
 
     def rewind(self, layer: int, t: int):
         self._check(self.lib.ssd_cache_rewind(self._h, layer, t), "ssd_cache_rewind")
+
+    def profile_enable(self, max_launches: int):
+        self._prof_cap = int(max_launches)
+        self._check(self.lib.ssd_profile_enable(self._h, int(max_launches)), "ssd_profile_enable")
+
+    def profile_collect(self) -> np.ndarray:
+        ms = np.empty(max(getattr(self, "_prof_cap", 0), 1), np.float32)
+        n = C.c_int32(0)
+        self._check(self.lib.ssd_profile_collect(self._h, ms.ctypes.data, C.byref(n)), "ssd_profile_collect")
+        return ms[: n.value].copy()
 
     def kv_bytes_per_seq(self) -> int:
         v = C.c_size_t(0)

@@ -70,6 +70,8 @@ struct ssd_cache {
   std::vector<int64_t> layer_base;    // [layers] first slot of the layer in the slab
   std::vector<int32_t> n_sink;        // [layers]
   std::vector<int32_t> t_img, n0, prompt_valid, static_valid;  // [layers]
+  std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
+  int prof_n = 0;                     // launches recorded since the last collect
 
   HeadDesc* d_desc(int layer) const { return reinterpret_cast<HeadDesc*>(base + reg.desc) + (size_t)layer * cfg.n_heads; }
   int32_t* d_idx(int layer) const {
@@ -164,8 +166,44 @@ int ssd_cache_create(const ssd_config* cfg, void* dev_mem, size_t dev_bytes, ssd
   return SSD_OK;
 }
 
+static void destroy_events(ssd_cache* c) {
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  c->prof_ev.clear();
+  c->prof_n = 0;
+}
+
 int ssd_cache_free(ssd_cache* c) {
+  if (c) destroy_events(c);
   delete c;
+  return SSD_OK;
+}
+
+int ssd_profile_enable(ssd_cache* c, int32_t max_launches) {
+  if (!c || max_launches < 0) return SSD_ERR_INVALID_ARG;
+  destroy_events(c);
+  for (int i = 0; i < 2 * max_launches; ++i) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) {
+      cudaGetLastError();
+      destroy_events(c);
+      return SSD_ERR_CUDA;
+    }
+    c->prof_ev.push_back(e);
+  }
+  return SSD_OK;
+}
+
+int ssd_profile_collect(ssd_cache* c, float* ms_host, int32_t* n_out) {
+  if (!c || !ms_host || !n_out) return SSD_ERR_INVALID_ARG;
+  for (int i = 0; i < c->prof_n; ++i) {
+    if (cudaEventSynchronize(c->prof_ev[2 * i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(ms_host + i, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      return SSD_ERR_CUDA;
+    }
+  }
+  *n_out = c->prof_n;
+  c->prof_n = 0;
   return SSD_OK;
 }
 
@@ -355,7 +393,14 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.n_workers = 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   const long total = c->valid_per_seq(layer) * g.n_seqs;
-  if (launch_decode(p, total, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
+  if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
+  if (launch_decode(p, total, st) != cudaSuccess) return SSD_ERR_CUDA;
+  if (timed) {
+    cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
+    c->prof_n += 1;
+  }
   return SSD_OK;
 }
 
