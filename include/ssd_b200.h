@@ -120,7 +120,7 @@ int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v
 /* Single-token decode attention over the layer's retained slots, both head types in one launch:
  * out[s,h] = sum_i softmax_i(scale * <q[s,h], K_i>) V_i over the prompt, static and ring slots
  * that hold a token (the token just appended included).  fp32 accumulation, bf16 output.
- *   q, out [n_seqs, n_heads, head_dim]
+ *   q, out [n_seqs, n_heads, head_dim], 16-byte aligned
  * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
 int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
@@ -159,6 +159,30 @@ int ssd_cache_kv_bytes(ssd_cache *cache, size_t *bytes_per_seq);
  * max_launches floats), their number to *n_out, and starts over.  No paper counterpart. */
 int ssd_profile_enable(ssd_cache *cache, int32_t max_launches);
 int ssd_profile_collect(ssd_cache *cache, float *ms_host, int32_t *n_out);
+
+/* Device status word of the cache (0 = healthy).  Bit 0: a decode warp gave up a bounded wait
+ * for one of its asynchronous copies or for a partial result (each wait is limited to about a
+ * second); the outputs of that launch are then incomplete.  The kernels never trap and never spin
+ * without a limit, so the CUDA context stays usable.  Synchronises the device.  No paper
+ * counterpart. */
+int ssd_cache_device_status(ssd_cache *cache, uint32_t *status_host);
+
+/* Inspection of the decode kernel's work decomposition, computed on the host by the same code the
+ * kernel runs (no GPU needed): lists every bulk copy one ssd_decode_attn launch would issue for a
+ * layer with the given per-head layout and occupancy.
+ *   head_recs [n_heads][4] = {first slot of the head inside a sequence's block, static capacity,
+ *             ring capacity, 1 if semantic}; heads are packed back to back (prompt_len + static
+ *             + ring slots each)
+ *   prompt_valid 0 or prompt_len; static_valid valid top-M slots of semantic heads; t_img image
+ *   tokens held; max_workers warps available; chunk slots per copy stage (0 = the kernel's own)
+ *   copies_out [cap][6] = {worker, chunk number within the worker, source slot (from the layer's
+ *             first slot), destination slot within the stage, slots copied, sequence*n_heads+head}
+ * Returns the number of copies (which may exceed cap; only the first cap are written) or a negative
+ * ssd_status.  No paper counterpart. */
+int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t *head_recs, int32_t prompt_len,
+                              int32_t n_seqs, int32_t prompt_valid, int32_t static_valid,
+                              int32_t t_img, int32_t max_workers, int32_t chunk,
+                              int64_t *copies_out, int64_t cap);
 
 /* Number of kernels this library has launched since the process started (for audit). */
 uint64_t ssd_kernel_launch_count(void);

@@ -28,6 +28,7 @@ EXPORTS = [
     "ssd_decode_attn", "ssd_step_host", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
+    "ssd_cache_device_status", "ssd_debug_decode_plan",
 ]
 
 
@@ -85,6 +86,9 @@ def load():
     L.ssd_cache_kv_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.ssd_profile_enable.argtypes = [vp, i32]
     L.ssd_profile_collect.argtypes = [vp, vp, C.POINTER(i32)]
+    L.ssd_cache_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    L.ssd_debug_decode_plan.argtypes = [i32, vp, i32, i32, i32, i32, i32, i32, i32, vp, C.c_int64]
+    L.ssd_debug_decode_plan.restype = C.c_int64
     L.ssd_kernel_launch_count.argtypes = []
     L.ssd_kernel_launch_count.restype = u64
     for n in EXPORTS:
@@ -263,7 +267,26 @@ class SsdCache:
         self._check(self.lib.ssd_profile_collect(self._h, ms.ctypes.data, C.byref(n)), "ssd_profile_collect")
         return ms[: n.value].copy()
 
+    def device_status(self) -> int:
+        v = C.c_uint32(0)
+        self._check(self.lib.ssd_cache_device_status(self._h, C.byref(v)), "ssd_cache_device_status")
+        return int(v.value)
+
     def kv_bytes_per_seq(self) -> int:
         v = C.c_size_t(0)
         self._check(self.lib.ssd_cache_kv_bytes(self._h, C.byref(v)), "ssd_cache_kv_bytes")
         return int(v.value)
+
+
+def decode_plan(head_recs, prompt_len, n_seqs, prompt_valid, static_valid, t_img, max_workers, chunk=0):
+    """Copies one decode launch would issue (host-side enumeration): int64 [n, 6] rows of
+    (worker, chunk, source slot, destination slot, slots, sequence * n_heads + head)."""
+    recs = np.ascontiguousarray(head_recs, np.int32).reshape(-1, 4)
+    args = (recs.shape[0], recs.ctypes.data, prompt_len, n_seqs, prompt_valid, static_valid, t_img, max_workers, chunk)
+    n = int(load().ssd_debug_decode_plan(*args, None, 0))
+    if n < 0:
+        raise SsdError(n, "ssd_debug_decode_plan")
+    out = np.empty((max(n, 1), 6), np.int64)
+    n2 = int(load().ssd_debug_decode_plan(*args, out.ctypes.data, n))
+    assert n2 == n
+    return out[:n]

@@ -16,7 +16,7 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Regions {
-  size_t desc, idx, counters, partial, score, staging, slab;  // byte offsets
+  size_t desc, idx, counters, status, partial, score, staging, slab;  // byte offsets
   size_t score_bytes, partial_bytes, front_bytes;
 };
 
@@ -32,6 +32,7 @@ static bool config_ok(const ssd_config* c) {
   // keep every index in 32 bits with room to spare
   const double slots = (double)c->prompt_len + std::fmax((double)c->window, (double)c->sink_budget + c->sink_recent);
   if (slots * c->n_heads > 1.0e9 || (double)c->n_seqs * c->n_heads > 5.0e8) return false;
+  if (slots * c->n_heads * c->n_seqs > 2.0e9) return false;   // slots of one layer are counted in 32 bits
   if ((double)c->prompt_len + c->max_image_tokens > 1.0e8) return false;
   return true;
 }
@@ -43,6 +44,7 @@ static Regions plan_regions(const ssd_config& c) {
   r.desc = off;      off = align_up(off + (size_t)c.n_layers * c.n_heads * sizeof(HeadDesc));
   r.idx = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * (c.sink_budget > 0 ? c.sink_budget : 1) * 4);
   r.counters = off;  off = align_up(off + pairs_layer * 4);
+  r.status = off;    off = align_up(off + 4);
   r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
   r.partial = off;   off = align_up(off + r.partial_bytes);
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
@@ -79,6 +81,7 @@ struct ssd_cache {
     return reinterpret_cast<int32_t*>(base + reg.idx) + (size_t)layer * per;
   }
   uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
+  uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(base + reg.status); }
   float* d_partial() const { return reinterpret_cast<float*>(base + reg.partial); }
   float* d_score() const { return reinterpret_cast<float*>(base + reg.score); }
   char* d_staging() const { return base + reg.staging; }
@@ -87,13 +90,21 @@ struct ssd_cache {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
     return cfg.prompt_len + (a > b ? a : b);
   }
-  long valid_per_seq(int layer) const {
-    long v = 0;
+  // layout and occupancy of a layer, as the decode kernel sees it
+  void fill_view(int layer, LayerView& v) const {
+    v.H = cfg.n_heads; v.L = cfg.prompt_len; v.n_seqs = cfg.n_seqs; v.seq_slots = seq_slots[layer];
+    v.prompt_valid = prompt_valid[layer];
+    v.static_valid = static_valid[layer];
+    v.t_img = t_img[layer];
+    int run = 0;
     for (int h = 0; h < cfg.n_heads; ++h) {
       const HeadDesc& d = desc[(size_t)layer * cfg.n_heads + h];
-      v += prompt_valid[layer] + (d.w ? static_valid[layer] : 0) + (t_img[layer] < d.z ? t_img[layer] : d.z);
+      v.head[h] = HeadRec{d.x, d.y, d.z, d.w};
+      v.cum[h] = run;
+      run += head_valid(v, h);
     }
-    return v;
+    v.cum[cfg.n_heads] = run;
+    v.contig = view_contiguous(v) ? 1 : 0;
   }
 };
 
@@ -378,25 +389,21 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   DecodeParams p;
   p.slab = c->d_slab(layer);
-  p.desc = c->d_desc(layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.partial = c->d_partial();
   p.counters = c->d_counters();
-  p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
-  p.prompt_valid = c->prompt_valid[layer];
-  p.static_valid = c->static_valid[layer];
-  p.t_img = c->t_img[layer];
-  p.seq_slots = c->seq_slots[layer];
-  p.n_workers = 0;
+  p.status = c->d_status();
   p.scale_log2 = c->scale * 1.4426950408889634f;
-  const long total = c->valid_per_seq(layer) * g.n_seqs;
+  p.split = Split{0, 0, 0, 0, 0.f};
+  c->fill_view(layer, p.view);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
-  if (launch_decode(p, total, st) != cudaSuccess) return SSD_ERR_CUDA;
+  if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -502,6 +509,74 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
   for (int l = 0; l < c->cfg.n_layers; ++l) slots += (size_t)c->seq_slots[l];
   *bytes_per_seq = slots * kSlotBytes;
   return SSD_OK;
+}
+
+int ssd_cache_device_status(ssd_cache* c, uint32_t* status_host) {
+  if (!c || !status_host) return SSD_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(status_host, c->d_status(), 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  return SSD_OK;
+}
+
+int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t prompt_len, int32_t n_seqs,
+                              int32_t prompt_valid, int32_t static_valid, int32_t t_img, int32_t max_workers,
+                              int32_t chunk, int64_t* copies_out, int64_t cap) {
+  if (n_heads < 1 || n_heads > kMaxHeads || !head_recs || n_seqs < 1 || prompt_len < 0 || max_workers < 1)
+    return SSD_ERR_INVALID_ARG;
+  if ((prompt_valid != 0 && prompt_valid != prompt_len) || static_valid < 0 || t_img < 0 || cap < 0 ||
+      (cap > 0 && !copies_out))
+    return SSD_ERR_INVALID_ARG;
+  if (chunk <= 0) chunk = decode_chunk_slots();
+  LayerView v;
+  v.H = n_heads; v.L = prompt_len; v.n_seqs = n_seqs;
+  v.prompt_valid = prompt_valid; v.static_valid = static_valid; v.t_img = t_img;
+  int off = 0, run = 0;
+  for (int h = 0; h < n_heads; ++h) {
+    const int32_t* r = head_recs + 4 * h;
+    if (r[1] < 0 || r[2] < 1 || r[0] != off || (r[3] == 0 && r[1] != 0) || (r[3] != 0 && static_valid > r[1]))
+      return SSD_ERR_INVALID_ARG;
+    v.head[h] = HeadRec{r[0], r[1], r[2], r[3]};
+    off += prompt_len + r[1] + r[2];
+    v.cum[h] = run;
+    run += head_valid(v, h);
+  }
+  v.cum[n_heads] = run;
+  v.seq_slots = off;
+  v.contig = view_contiguous(v) ? 1 : 0;
+  const long T = (long)run * n_seqs;
+  if (T < 1) return SSD_ERR_BAD_STATE;
+  if (T > 0x7fffffffL) return SSD_ERR_INVALID_ARG;
+  const long W = plan_workers(T, max_workers);
+  const Split sp = make_split(T, W);
+  int64_t n = 0;
+  for (int32_t wk = 0; wk < (int32_t)W; ++wk) {
+    const Share sh = share_plan(v, sp, wk);
+    if (sh.g_begin >= sh.g_end) continue;
+    if (share_of(sp, sh.g_begin) != wk || share_of(sp, sh.g_end - 1) != wk) return SSD_ERR_BAD_STATE;
+    Walk w;
+    share_walk_init(w, v, sh);
+    int64_t k = 0;
+    while (share_walk_more(w)) {
+      const int nn = walk_chunk(w, chunk);
+      if (nn < 1) return SSD_ERR_BAD_STATE;
+      const int64_t hbase = (int64_t)w.seq * v.seq_slots + v.head[w.head].x;
+      auto emit = [&](int src, int dst, int len) {
+        if (n < cap) {
+          int64_t* o = copies_out + 6 * n;
+          o[0] = wk; o[1] = k; o[2] = hbase + src; o[3] = dst; o[4] = len; o[5] = (int64_t)w.seq * n_heads + w.head;
+        }
+        ++n;
+      };
+      if (v.contig) emit(w.i, 0, nn);   // the kernel's fast path: one copy per chunk
+      else chunk_runs(v, w.head, w.i, nn, emit);
+      share_walk_advance(w, v, sh, nn);
+      ++k;
+    }
+  }
+  return n;
 }
 
 }  // extern "C"

@@ -3,306 +3,520 @@
 //
 // Decode (consumer of Algorithm 1's output): for every (sequence, head) of one layer,
 //   out = sum_i softmax_i(scale * <q, K_i>) V_i   over the slots that hold a token.
-// It is a GEMV per head (1 flop per byte), so the kernel is built around HBM streaming, not
-// tensor cores:
-//   * the valid slots of the whole layer form one logical stream of 512-byte slots
-//     ([K row | V row]); the stream is cut into equal, 8-slot-aligned shares, one per warp
-//     ("worker"), regardless of head type or length, so every SM gets the same bytes;
-//   * a worker walks its share pair by pair; half-warp 0/1 take even/odd slots, 16 lanes x
-//     128-bit loads cover one row; dot products are reduced with shuffles inside the
-//     half-warp; online softmax in fp32 (base-2 exponent, scale folded into q);
-//   * a pair that lies inside one share is finished in registers; a pair cut by a share
-//     boundary leaves (m, l, acc[128]) partials in scratch and the last contributor to
-//     arrive (atomic counter, never waits) merges them in worker order, which keeps the
-//     result independent of arrival order.
+// It is a GEMV per head (1 flop per byte), so the kernel is built around keeping HBM busy and
+// the instruction count per byte low, not around tensor cores:
+//   * one CTA per SM, every streaming warp an independent worker.  The valid slots of the whole
+//     layer form one logical stream of 512-byte slots ([K row | V row]) that is cut into equal
+//     shares, one per worker, regardless of head type or length, so every SM moves the same bytes;
+//   * a worker owns a ring of shared-memory stages.  Lane 0 fills them with bulk asynchronous
+//     copies (cp.async.bulk, completion counted on an mbarrier per stage), one chunk of up to
+//     kChunk slots per stage, and runs kStages chunks ahead of the arithmetic across head
+//     boundaries; the query row of a head travels with the head's first chunk.  A stage is
+//     pulled into registers and handed back to the copy engine before the arithmetic starts;
+//   * arithmetic per chunk: the warp works as four groups of 8 lanes, group g taking slots g,
+//     g + 4, ...; a lane covers 16 of the 128 dimensions with two 128-bit reads per row, packed
+//     two-wide fp32 FMAs, three shuffles per dot product, and an online softmax in fp32 (base-2
+//     exponent, scale folded into q);
+//   * a head that lies inside one share is finished in registers.  A head cut by a share boundary
+//     leaves a partial (m, l, acc[128]) in the worker's shared-memory mailbox, and an extra
+//     finisher warp per CTA merges the partials: straight from shared memory when all pieces of
+//     the head belong to this CTA (workers of a CTA hold consecutive shares, so that is the usual
+//     case), through global scratch and an arrival counter for the at most two heads that cross
+//     the CTA's own range (last CTA to arrive merges; nobody waits for another CTA).  Merges run
+//     in worker order, then CTA order, so results do not depend on arrival order.  A worker takes
+//     the cut piece at the end of its share first, so all of this happens while the bulk of the
+//     streaming is still under way, and no streaming warp ever executes a fence or an atomic.
+// Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
+// waits (bounded again) for its other copies in flight and leaves.
 #include "ssd_internal.cuh"
+
+#ifndef SSD_DECODE_WARPS
+#define SSD_DECODE_WARPS 8
+#endif
+#ifndef SSD_DECODE_STAGES
+#define SSD_DECODE_STAGES 2
+#endif
+#ifndef SSD_DECODE_CHUNK
+#define SSD_DECODE_CHUNK 16
+#endif
 
 namespace ssd {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-constexpr int kCtasPerSm = 3;
-constexpr int kU = 4;               // slots per half-warp per iteration
-constexpr int kAlign = 8;           // share boundaries are multiples of this many slots
-constexpr int kMinShare = 16;       // never cut shares smaller than this
+constexpr int kWarps = SSD_DECODE_WARPS;             // streaming workers per CTA
+constexpr int kThreads = (kWarps + 1) * 32;          // plus one finisher warp
+constexpr int kStages = SSD_DECODE_STAGES;
+constexpr int kChunk = SSD_DECODE_CHUNK;             // slots per stage
+constexpr int kGroups = 4;                           // 8-lane groups of a warp
+constexpr int kPer = kChunk / kGroups;               // slots of a stage each group takes
+constexpr int kU = kPer < 4 ? kPer : 4;              // slots a group folds in at a time
+constexpr int kQBytes = kHeadDim * 2;
+constexpr int kStageBytes = kChunk * kSlotBytes + kQBytes;
+constexpr int kRingBytes = kWarps * kStages * kStageBytes;
+constexpr int kBarBytes = (kWarps * kStages + kWarps * 2) * 8;   // stage barriers, then mailbox barriers
+constexpr int kMailBytes = kWarps * 2 * kPartialFloats * 4;      // two partials per worker
+constexpr int kSmemBytes = kRingBytes + kBarBytes + kMailBytes;
 constexpr float kNegBig = -1.0e30f;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait, then give up
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-      : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-      : "l"(p));
-  return v;
+static_assert(kChunk % kGroups == 0 && kPer % kU == 0, "a stage is folded in groups of kGroups * kU slots");
+static_assert(kSmemBytes <= 227 * 1024, "stage rings exceed the shared memory of an SM");
+static_assert(kBarBytes % 16 == 0, "mailboxes are read as float4");
+
+// ------------------------------------------------------------------ asynchronous-copy plumbing
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Wait for a phase of the barrier, for at most kWaitLimitNs.  Uniform over the warp.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  bool ok = mbar_try_wait(bar, parity);
+  if (!ok) {
+    const unsigned long long t0 = global_ns();
+    do {
+#pragma unroll 1
+      for (int i = 0; i < 64 && !ok; ++i) ok = mbar_try_wait(bar, parity);
+    } while (!ok && global_ns() - t0 < kWaitLimitNs);
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+// Global -> shared bulk copy; bytes is a multiple of 16 and both addresses are 16-byte aligned.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
 }
 
+// ------------------------------------------------------------------ arithmetic
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 
-__device__ __forceinline__ float lo_f(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-__device__ __forceinline__ float dot8(const uint4& k, const float (&q)[8]) {
-  float a = lo_f(k.x) * q[0];
-  a = fmaf(hi_f(k.x), q[1], a);
-  a = fmaf(lo_f(k.y), q[2], a);
-  a = fmaf(hi_f(k.y), q[3], a);
-  a = fmaf(lo_f(k.z), q[4], a);
-  a = fmaf(hi_f(k.z), q[5], a);
-  a = fmaf(lo_f(k.w), q[6], a);
-  a = fmaf(hi_f(k.w), q[7], a);
-  return a;
+// the two bf16 values of a 32-bit word, widened exactly
+__device__ __forceinline__ float2 widen2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
 
-__device__ __forceinline__ void axpy8(float p, const uint4& v, float (&acc)[8]) {
-  acc[0] = fmaf(p, lo_f(v.x), acc[0]);
-  acc[1] = fmaf(p, hi_f(v.x), acc[1]);
-  acc[2] = fmaf(p, lo_f(v.y), acc[2]);
-  acc[3] = fmaf(p, hi_f(v.y), acc[3]);
-  acc[4] = fmaf(p, lo_f(v.z), acc[4]);
-  acc[5] = fmaf(p, hi_f(v.z), acc[5]);
-  acc[6] = fmaf(p, lo_f(v.w), acc[6]);
-  acc[7] = fmaf(p, hi_f(v.w), acc[7]);
-}
-
+// A lane's share of a row: 16 of the 128 dimensions, as 8 pairs.  Lane l8 of a group holds
+// dimensions [8*l8, 8*l8 + 8) in pairs 0..3 and [64 + 8*l8, 64 + 8*l8 + 8) in pairs 4..7.
 struct State {
   float m, l;
-  float acc[8];
+  float2 acc[8];
 };
 
 __device__ __forceinline__ void state_init(State& s) {
   s.m = kNegBig;
   s.l = 0.f;
 #pragma unroll
-  for (int d = 0; d < 8; ++d) s.acc[d] = 0.f;
+  for (int d = 0; d < 8; ++d) s.acc[d] = make_float2(0.f, 0.f);
 }
 
-// s <- s (+) (m2, l2, acc2)
-__device__ __forceinline__ void state_merge(State& s, float m2, float l2, const float (&a2)[8]) {
-  float mn = fmaxf(s.m, m2);
-  float c1 = ex2(s.m - mn), c2 = ex2(m2 - mn);
+// s <- s (+) the state held by lane (lane ^ mask)
+__device__ __forceinline__ void state_merge_lane(State& s, int mask) {
+  const float m2 = __shfl_xor_sync(0xffffffffu, s.m, mask);
+  const float l2 = __shfl_xor_sync(0xffffffffu, s.l, mask);
+  const float mn = fmaxf(s.m, m2);
+  const float c1 = ex2(s.m - mn), c2 = ex2(m2 - mn);
   s.l = s.l * c1 + l2 * c2;
 #pragma unroll
-  for (int d = 0; d < 8; ++d) s.acc[d] = s.acc[d] * c1 + a2[d] * c2;
+  for (int d = 0; d < 8; ++d) {
+    const float ax = __shfl_xor_sync(0xffffffffu, s.acc[d].x, mask);
+    const float ay = __shfl_xor_sync(0xffffffffu, s.acc[d].y, mask);
+    s.acc[d].x = s.acc[d].x * c1 + ax * c2;
+    s.acc[d].y = s.acc[d].y * c1 + ay * c2;
+  }
   s.m = mn;
 }
 
-// Stream `n` physically contiguous slots starting at `base` into the running state of this
-// half-warp (hw = 0/1 takes even/odd slots).
-__device__ __forceinline__ void process_piece(const uint4* __restrict__ base, int n, int hw, int l16,
-                                              const float (&q)[8], State& st) {
-  for (int s = 0; s < n; s += 2 * kU) {
-    uint4 k[kU], v[kU];
-    bool ok[kU];
+// (m, l, acc4) <- (m, l, acc4) (+) (mj, lj, aj): four output dimensions of a partial
+__device__ __forceinline__ void merge4(float& m, float& l, float4& acc, float mj, float lj, const float4& aj) {
+  const float mn = fmaxf(m, mj);
+  const float c1 = ex2(m - mn), c2 = ex2(mj - mn);
+  l = l * c1 + lj * c2;
+  acc.x = acc.x * c1 + aj.x * c2;
+  acc.y = acc.y * c1 + aj.y * c2;
+  acc.z = acc.z * c1 + aj.z * c2;
+  acc.w = acc.w * c1 + aj.w * c2;
+  m = mn;
+}
+
+__device__ __forceinline__ float dot16(const uint4& k0, const uint4& k1, const float2 (&q)[8]) {
+  float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
+  a = __ffma2_rn(widen2(k0.x), q[0], a);
+  b = __ffma2_rn(widen2(k1.x), q[4], b);
+  a = __ffma2_rn(widen2(k0.y), q[1], a);
+  b = __ffma2_rn(widen2(k1.y), q[5], b);
+  a = __ffma2_rn(widen2(k0.z), q[2], a);
+  b = __ffma2_rn(widen2(k1.z), q[6], b);
+  a = __ffma2_rn(widen2(k0.w), q[3], a);
+  b = __ffma2_rn(widen2(k1.w), q[7], b);
+  return (a.x + a.y) + (b.x + b.y);
+}
+
+__device__ __forceinline__ void axpy16(float p, const uint4& v0, const uint4& v1, float2 (&acc)[8]) {
+  const float2 pp = make_float2(p, p);
+  acc[0] = __ffma2_rn(pp, widen2(v0.x), acc[0]);
+  acc[1] = __ffma2_rn(pp, widen2(v0.y), acc[1]);
+  acc[2] = __ffma2_rn(pp, widen2(v0.z), acc[2]);
+  acc[3] = __ffma2_rn(pp, widen2(v0.w), acc[3]);
+  acc[4] = __ffma2_rn(pp, widen2(v1.x), acc[4]);
+  acc[5] = __ffma2_rn(pp, widen2(v1.y), acc[5]);
+  acc[6] = __ffma2_rn(pp, widen2(v1.z), acc[6]);
+  acc[7] = __ffma2_rn(pp, widen2(v1.w), acc[7]);
+}
+
+// The rows of a stage as one lane holds them: slot 4*u + grp, two 16-byte pieces of K and of V.
+struct Rows {
+  uint4 k0[kPer], k1[kPer], v0[kPer], v1[kPer];
+};
+
+// Pull the `n` slots of a stage out of shared memory so that the stage can be refilled before
+// the arithmetic starts.
+__device__ __forceinline__ void load_stage(const uint4* __restrict__ sb, int n, int grp, int l8, Rows& r) {
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      int slot = s + 2 * u + hw;
-      ok[u] = slot < n;
-      const uint4* p = base + (size_t)slot * kSlotU4 + l16;
-      if (ok[u]) {
-        k[u] = ld_stream(p);
-        v[u] = ld_stream(p + 16);
-      } else {
-        k[u] = make_uint4(0, 0, 0, 0);
-        v[u] = make_uint4(0, 0, 0, 0);
-      }
+  for (int u = 0; u < kPer; ++u) {
+    const int slot = kGroups * u + grp;
+    const uint4* p = sb + slot * kSlotU4 + l8;
+    if (slot < n) {
+      r.k0[u] = p[0];
+      r.k1[u] = p[8];
+      r.v0[u] = p[16];
+      r.v1[u] = p[24];
+    } else {               // slots past n hold whatever an earlier chunk left there
+      r.k0[u] = r.k1[u] = r.v0[u] = r.v1[u] = make_uint4(0, 0, 0, 0);
     }
+  }
+}
+
+// Fold those slots into the running state of this lane's group.
+__device__ __forceinline__ void fold_stage(const Rows& r, int n, int grp, const float2 (&q)[8], State& st) {
+#pragma unroll
+  for (int s = 0; s < kPer; s += kU) {
+    if (kGroups * s >= n) break;
     float x[kU];
 #pragma unroll
-    for (int u = 0; u < kU; ++u) x[u] = dot8(k[u], q);
+    for (int u = 0; u < kU; ++u) x[u] = dot16(r.k0[s + u], r.k1[s + u], q);
 #pragma unroll
-    for (int off = 8; off >= 1; off >>= 1) {
+    for (int off = 4; off >= 1; off >>= 1) {
 #pragma unroll
       for (int u = 0; u < kU; ++u) x[u] += __shfl_xor_sync(0xffffffffu, x[u], off);
     }
     float mn = st.m;
 #pragma unroll
-    for (int u = 0; u < kU; ++u) mn = fmaxf(mn, ok[u] ? x[u] : kNegBig);
-    float corr = ex2(st.m - mn);
+    for (int u = 0; u < kU; ++u) {
+      if (kGroups * (s + u) + grp >= n) x[u] = kNegBig;
+      mn = fmaxf(mn, x[u]);
+    }
+    const float corr = ex2(st.m - mn);
     float p[kU], psum = 0.f;
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-      p[u] = ok[u] ? ex2(x[u] - mn) : 0.f;
+      p[u] = kGroups * (s + u) + grp < n ? ex2(x[u] - mn) : 0.f;
       psum += p[u];
     }
     st.l = st.l * corr + psum;
     st.m = mn;
+    const float2 cc = make_float2(corr, corr);
 #pragma unroll
-    for (int d = 0; d < 8; ++d) st.acc[d] *= corr;
+    for (int d = 0; d < 8; ++d) st.acc[d] = __fmul2_rn(st.acc[d], cc);
 #pragma unroll
-    for (int u = 0; u < kU; ++u) axpy8(p[u], v[u], st.acc);
+    for (int u = 0; u < kU; ++u) axpy16(p[u], r.v0[s + u], r.v1[s + u], st.acc);
   }
 }
 
-__device__ __forceinline__ long share_start(long i, long T, long W) {
-  if (i >= W) return T;
-  return ((i * T) / W) & ~(long)(kAlign - 1);
+__device__ __forceinline__ uint32_t pack_bf16(float2 a, float inv) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(a.x * inv, a.y * inv);
+  return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// Largest worker index whose share starts at or before logical slot g.
-__device__ __forceinline__ long share_of(long g, long T, long W) {
-  long gp = (g & ~(long)(kAlign - 1)) + kAlign;
-  long w = (gp * W - 1) / T;
-  return w < W - 1 ? w : W - 1;
+// lanes 0..7 write the row: 16 bytes at dimension 8*l8 and 16 bytes at dimension 64 + 8*l8
+__device__ __forceinline__ void write_out(__nv_bfloat16* out, const State& st, int l8) {
+  const float inv = 1.f / st.l;
+  uint4* o = reinterpret_cast<uint4*>(out);
+  o[l8] = make_uint4(pack_bf16(st.acc[0], inv), pack_bf16(st.acc[1], inv), pack_bf16(st.acc[2], inv),
+                     pack_bf16(st.acc[3], inv));
+  o[8 + l8] = make_uint4(pack_bf16(st.acc[4], inv), pack_bf16(st.acc[5], inv), pack_bf16(st.acc[6], inv),
+                         pack_bf16(st.acc[7], inv));
 }
 
-__device__ __forceinline__ void write_out(__nv_bfloat16* out, const State& st, int l16) {
-  float inv = 1.f / st.l;
-  uint4 o;
-  __nv_bfloat162 t;
-  t = __floats2bfloat162_rn(st.acc[0] * inv, st.acc[1] * inv);
-  o.x = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(st.acc[2] * inv, st.acc[3] * inv);
-  o.y = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(st.acc[4] * inv, st.acc[5] * inv);
-  o.z = *reinterpret_cast<uint32_t*>(&t);
-  t = __floats2bfloat162_rn(st.acc[6] * inv, st.acc[7] * inv);
-  o.w = *reinterpret_cast<uint32_t*>(&t);
-  reinterpret_cast<uint4*>(out)[l16] = o;
+// all 32 lanes write the row, lane i the dimensions [4i, 4i + 4)
+__device__ __forceinline__ void write_out4(__nv_bfloat16* out, float l, const float4& acc, int lane) {
+  const float inv = 1.f / l;
+  uint2 o;
+  o.x = pack_bf16(make_float2(acc.x, acc.y), inv);
+  o.y = pack_bf16(make_float2(acc.z, acc.w), inv);
+  reinterpret_cast<uint2*>(out)[lane] = o;
 }
 
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const DecodeParams p) {
-  __shared__ int s_cum[kMaxHeads + 1];  // exclusive prefix of valid slots per head
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int hw = lane >> 4, l16 = lane & 15;
+// The finisher warp of a CTA.  The CTA's workers hold consecutive shares, so most heads that are
+// cut by a share boundary are cut between two workers of the same CTA: the finisher merges their
+// partials straight from the shared-memory mailboxes, in worker order, and writes the output.
+// Only the (at most two) heads that cross the CTA's own range go through global scratch: the
+// finisher stores the CTA's merged partial, counts arrivals per head with an atomic (it never
+// waits for another CTA) and, where this CTA was the last to arrive, merges the CTAs' partials
+// in CTA order.  All fences and atomics of the launch are issued here, off the streaming warps'
+// path.  Lane i holds output dimensions [4i, 4i + 4).
+__device__ void finisher(const DecodeParams& p, const unsigned char* smem, int lane) {
+  const LayerView& v = p.view;
+  const Split& sp = p.split;
+  const uint32_t mail_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
+  const float* mail = reinterpret_cast<const float*>(smem + kRingBytes + kBarBytes);
+  const int lo_c = (int)blockIdx.x * kWarps;
+  const int hi_c = (lo_c + kWarps < sp.W ? lo_c + kWarps : sp.W) - 1;
+  int n_glob = 0;                         // heads of this CTA that go through global scratch (<= 2)
+  int my_pair = 0, my_g0 = 0, my_vh = 0;  // lane k keeps the record of the k-th of them
+  bool ok = true;
 
-  // valid slots per head, then an exclusive scan by warp 0 (4 heads per lane)
-  if (tid < 32) {
-    int v[4], sum = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      int h = tid * 4 + i;
-      v[i] = 0;
-      if (h < p.H) {
-        HeadDesc d = p.desc[h];
-        v[i] = p.prompt_valid + (d.w ? p.static_valid : 0) + min(p.t_img, d.z);
+  // worker `w` posts a partial of the head that covers logical slot g_piece (walk t points there)
+  auto handle = [&](int w, const Walk& t, int g_piece) {
+    if (!ok) return;
+    const int g0 = g_piece - t.i, g1 = g0 + t.vh;
+    const int w_lo = share_of(sp, g0), w_hi = share_of(sp, g1 - 1);
+    const int f = w_lo > lo_c ? w_lo : lo_c;       // first contributor inside this CTA
+    if (w != f) return;                            // the head is dealt with at that worker
+    const int e = w_hi < hi_c ? w_hi : hi_c;       // last contributor inside this CTA
+    float m = kNegBig, l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = f; j <= e; ++j) {
+      // the head is worker j's leading piece unless j's share starts before the head does
+      const int which = (j == w_lo && share_start(sp, j) < g0) ? 1 : 0;
+      const int box = (j - lo_c) * 2 + which;
+      if (!mbar_wait(mail_bar0 + 8 * box, 0)) {
+        ok = false;
+        if (lane == 0) atomicOr(p.status, 1u);
+        return;
       }
-      sum += v[i];
+      const float* P = mail + (size_t)box * kPartialFloats;
+      merge4(m, l, acc, P[0], P[1], reinterpret_cast<const float4*>(P + 4)[lane]);
     }
-    int incl = sum;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      int o = __shfl_up_sync(0xffffffffu, incl, off);
-      if (tid >= off) incl += o;
-    }
-    int run = incl - sum;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      int h = tid * 4 + i;
-      if (h <= p.H) s_cum[h] = run;
-      run += v[i];
-    }
-    if (tid == 31 && p.H == kMaxHeads) s_cum[kMaxHeads] = run;
-  }
-  __syncthreads();
-
-  const long Vseq = s_cum[p.H];
-  const long T = Vseq * p.n_seqs;
-  const long W = p.n_workers;
-  const long wk = (long)blockIdx.x * kWarps + warp;
-  if (wk >= W) return;
-
-  long g = share_start(wk, T, W);
-  const long g_end = share_start(wk + 1, T, W);
-  bool first = true;
-
-  while (g < g_end) {
-    const int seq = (int)(g / Vseq);
-    const int r = (int)(g - (long)seq * Vseq);
-    int lo = 0, hi = p.H;  // find head with s_cum[head] <= r < s_cum[head+1]
-    while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if (s_cum[mid] <= r) lo = mid; else hi = mid;
-    }
-    const int head = lo;
-    const int vh = s_cum[head + 1] - s_cum[head];
-    const int i0 = r - s_cum[head];
-    const long left = g_end - g;
-    const int i1 = (long)(vh - i0) <= left ? vh : i0 + (int)left;
-
-    const HeadDesc d = p.desc[head];
-    const int pair = seq * p.H + head;
-    const uint4* pbase = p.slab + ((size_t)seq * p.seq_slots + d.x) * kSlotU4;
-
-    float q[8];
-    {
-      uint4 qq = reinterpret_cast<const uint4*>(p.q + (size_t)pair * kHeadDim)[l16];
-      q[0] = lo_f(qq.x) * p.scale_log2; q[1] = hi_f(qq.x) * p.scale_log2;
-      q[2] = lo_f(qq.y) * p.scale_log2; q[3] = hi_f(qq.y) * p.scale_log2;
-      q[4] = lo_f(qq.z) * p.scale_log2; q[5] = hi_f(qq.z) * p.scale_log2;
-      q[6] = lo_f(qq.w) * p.scale_log2; q[7] = hi_f(qq.w) * p.scale_log2;
-    }
-    State st;
-    state_init(st);
-
-    // three physically contiguous runs: prompt, static, ring
-    const int sv = d.w ? p.static_valid : 0;
-    const int rv = min(p.t_img, d.z);
-    const int run_l0[3] = {0, p.prompt_valid, p.prompt_valid + sv};
-    const int run_n[3] = {p.prompt_valid, sv, rv};
-    const int run_p0[3] = {0, p.L, p.L + d.y};
-#pragma unroll
-    for (int rr = 0; rr < 3; ++rr) {
-      int a = max(i0, run_l0[rr]);
-      int b = min(i1, run_l0[rr] + run_n[rr]);
-      if (b > a)
-        process_piece(pbase + (size_t)(run_p0[rr] + (a - run_l0[rr])) * kSlotU4, b - a, hw, l16, q, st);
-    }
-
-    // merge the two half-warps (lanes i and i+16 hold the same 8 output dims)
-    {
-      float m2 = __shfl_xor_sync(0xffffffffu, st.m, 16);
-      float l2 = __shfl_xor_sync(0xffffffffu, st.l, 16);
-      float a2[8];
-#pragma unroll
-      for (int dd = 0; dd < 8; ++dd) a2[dd] = __shfl_xor_sync(0xffffffffu, st.acc[dd], 16);
-      state_merge(st, m2, l2, a2);
-    }
-
-    __nv_bfloat16* outp = p.out + (size_t)pair * kHeadDim;
-    if (i0 == 0 && i1 == vh) {
-      if (hw == 0) write_out(outp, st, l16);
+    const int pair = t.seq * v.H + t.head;
+    if (w_lo >= lo_c && w_hi <= hi_c) {            // the whole head lies inside this CTA
+      write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
     } else {
-      float* P = p.partial + ((size_t)wk * 2 + (first ? 0 : 1)) * kPartialFloats;
+      // slot 0: the head began in an earlier CTA; slot 1: it begins here and runs on
+      float* G = p.partial + ((size_t)blockIdx.x * 2 + (w_lo < lo_c ? 0 : 1)) * kPartialFloats;
       if (lane == 0) {
-        P[0] = st.m;
-        P[1] = st.l;
+        G[0] = m;
+        G[1] = l;
       }
-      if (hw == 0) {
-        reinterpret_cast<float4*>(P + 4)[l16 * 2] = make_float4(st.acc[0], st.acc[1], st.acc[2], st.acc[3]);
-        reinterpret_cast<float4*>(P + 4)[l16 * 2 + 1] = make_float4(st.acc[4], st.acc[5], st.acc[6], st.acc[7]);
+      reinterpret_cast<float4*>(G + 4)[lane] = acc;
+      if (lane == n_glob) {
+        my_pair = pair;
+        my_g0 = g0;
+        my_vh = t.vh;
       }
-      __threadfence();
-      __syncwarp();
-      const long g0 = g - i0, g1 = g0 + vh;
-      const long w_lo = share_of(g0, T, W), w_hi = share_of(g1 - 1, T, W);
-      const uint32_t n_contrib = (uint32_t)(w_hi - w_lo + 1);
-      uint32_t old = 0;
-      if (lane == 0) old = atomicAdd(p.counters + pair, 1u);
-      old = __shfl_sync(0xffffffffu, old, 0);
-      if (old == n_contrib - 1) {
-        __threadfence();
-        State tot;
-        state_init(tot);
-        for (long j = w_lo; j <= w_hi; ++j) {
-          int which = (j == w_lo && share_start(j, T, W) < g0) ? 1 : 0;
-          const float* Pj = p.partial + ((size_t)j * 2 + which) * kPartialFloats;
-          float mj = __ldcg(Pj), lj = __ldcg(Pj + 1);
-          float4 x0 = __ldcg(reinterpret_cast<const float4*>(Pj + 4) + l16 * 2);
-          float4 x1 = __ldcg(reinterpret_cast<const float4*>(Pj + 4) + l16 * 2 + 1);
-          float aj[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-          state_merge(tot, mj, lj, aj);
-        }
-        if (hw == 0) write_out(outp, tot, l16);
-        if (lane == 0) p.counters[pair] = 0u;
-      }
+      ++n_glob;
     }
-    g += i1 - i0;
-    first = false;
+  };
+
+  for (int w = lo_c; w <= hi_c; ++w) {
+    const Share sh = share_plan(v, sp, w);
+    if (sh.g_begin >= sh.g_end) continue;
+    Walk t;
+    if (sh.g_tail < sh.g_end) {          // the cut piece at the end of the share
+      walk_init(t, v, sh.g_tail, sh.g_end);
+      handle(w, t, sh.g_tail);
+    }
+    if (sh.g_begin < sh.g_tail) {        // the piece at the start, if its head began earlier
+      walk_init(t, v, sh.g_begin, sh.g_tail);
+      if (t.i != 0) handle(w, t, sh.g_begin);
+    }
+  }
+  if (!ok || n_glob == 0) return;
+
+  __threadfence();                       // the partials above, before the arrivals below
+  bool last = false;
+  if (lane < n_glob) {
+    const int g0 = my_g0, g1 = g0 + my_vh;
+    const uint32_t n_contrib = (uint32_t)(share_of(sp, g1 - 1) / kWarps - share_of(sp, g0) / kWarps + 1);
+    last = atomicAdd(p.counters + my_pair, 1u) == n_contrib - 1;
+  }
+  unsigned todo = __ballot_sync(0xffffffffu, last);
+  if (todo) __threadfence();
+  while (todo) {
+    const int src_lane = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int pair = __shfl_sync(0xffffffffu, my_pair, src_lane);
+    const int g0 = __shfl_sync(0xffffffffu, my_g0, src_lane);
+    const int g1 = g0 + __shfl_sync(0xffffffffu, my_vh, src_lane);
+    const int c_lo = share_of(sp, g0) / kWarps, c_hi = share_of(sp, g1 - 1) / kWarps;
+    float m = kNegBig, l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = c_lo; c <= c_hi; ++c) {
+      const float* G = p.partial + ((size_t)c * 2 + (c > c_lo ? 0 : 1)) * kPartialFloats;
+      merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
+    }
+    write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
+    if (lane == 0) p.counters[pair] = 0u;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const LayerView& v = p.view;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = lane >> 3, l8 = lane & 7;
+
+  const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
+  const uint32_t mail_bar = smem_u32(smem + kRingBytes) + kWarps * kStages * 8 + (uint32_t)warp * 16;
+  if (warp < kWarps && lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    mbar_init(mail_bar, 1);
+    mbar_init(mail_bar + 8, 1);
+    mbar_init_fence();
+  }
+  __syncthreads();   // the only CTA-wide barrier: mailboxes exist before anyone posts or waits
+
+  if (warp == kWarps) {
+    finisher(p, smem, lane);
+    return;
+  }
+  const int wk = (int)blockIdx.x * kWarps + warp;
+  if (wk >= p.split.W) return;
+  const Share sh = share_plan(v, p.split, wk);
+  if (sh.g_begin >= sh.g_end) return;
+
+  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
+  const uint32_t ring_s = smem_u32(ring);
+  float* mailbox = reinterpret_cast<float*>(smem + kRingBytes + kBarBytes) + (size_t)warp * 2 * kPartialFloats;
+
+  Walk prod;
+  share_walk_init(prod, v, sh);
+  Walk cons = prod;
+  int ahead = 0;   // chunks issued and not yet consumed
+
+  // lane 0 starts the copies of the producer's current chunk into `stage`; every lane advances
+  auto issue = [&](int stage) {
+    const int n = walk_chunk(prod, kChunk);
+    if (lane == 0) {
+      const bool begin = prod.i == 0 || prod.g == sh.g_begin;
+      const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
+      const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
+                                   ((size_t)prod.seq * v.seq_slots + v.head[prod.head].x) * kSlotBytes;
+      // order the warp's reads of this stage (made visible to this lane by __syncwarp) before
+      // the asynchronous writes that follow
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + (begin ? kQBytes : 0)));
+      if (v.contig) {
+        bulk_g2s(dst, hbase + (size_t)prod.i * kSlotBytes, (uint32_t)n * kSlotBytes, bar);
+      } else {
+        chunk_runs(v, prod.head, prod.i, n, [&](int src, int d, int len) {
+          bulk_g2s(dst + (uint32_t)d * kSlotBytes, hbase + (size_t)src * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
+        });
+      }
+      if (begin)
+        bulk_g2s(dst + kChunk * kSlotBytes, p.q + ((size_t)prod.seq * v.H + prod.head) * kHeadDim, kQBytes, bar);
+    }
+    share_walk_advance(prod, v, sh, n);
+    ++ahead;
+  };
+
+#pragma unroll 1
+  for (int s = 0; s < kStages && share_walk_more(prod); ++s) issue(s);
+
+  int stage = 0;
+  uint32_t parity = 0;
+  bool begin = true, leading = true;
+  int piece_i0 = 0;
+  float2 q[8];
+  State st;
+
+#pragma unroll 1
+  while (share_walk_more(cons)) {
+    const int n = walk_chunk(cons, kChunk);
+    if (!mbar_wait(bar0 + 8 * stage, parity)) {
+      // give up: flag it, let the copies still in flight land (bounded), and leave
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int k = 0; k < ahead; ++k) {
+        mbar_wait(bar0 + 8 * stage, parity);
+        if (++stage == kStages) { stage = 0; parity ^= 1u; }
+      }
+      return;
+    }
+    const uint4* sb = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageBytes);
+    if (begin) {
+      const uint4 qa = sb[kChunk * kSlotU4 + l8], qb = sb[kChunk * kSlotU4 + 8 + l8];
+      const float2 sc = make_float2(p.scale_log2, p.scale_log2);
+      q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
+      q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
+      q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
+      q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
+      state_init(st);
+      piece_i0 = cons.i;
+      leading = cons.g == sh.g_begin;   // the piece that holds the share's first slot
+      begin = false;
+    }
+    Rows rows;
+    load_stage(sb, n, grp, l8, rows);
+    __syncwarp();          // every lane has its rows in registers: the stage may be refilled
+    --ahead;
+    if (share_walk_more(prod)) issue(stage);
+    fold_stage(rows, n, grp, q, st);
+
+    const int i1 = cons.i + n;
+    if (i1 == cons.vh || cons.g + n == cons.g_end) {
+      // end of this worker's piece of the head: merge the four groups (lanes l, l^8, l^16, l^24
+      // hold the same 16 output dims), then write the output, or post a partial to the finisher
+      State tot = st;
+      state_merge_lane(tot, 8);
+      state_merge_lane(tot, 16);
+      if (piece_i0 == 0 && i1 == cons.vh) {
+        if (grp == 0) write_out(p.out + ((size_t)cons.seq * v.H + cons.head) * kHeadDim, tot, l8);
+      } else {
+        float* P = mailbox + (leading ? 0 : 1) * kPartialFloats;
+        if (lane == 0) {
+          P[0] = tot.m;
+          P[1] = tot.l;
+        }
+        if (grp == 0) {
+          float4* lo = reinterpret_cast<float4*>(P + 4 + 8 * l8);
+          float4* hi = reinterpret_cast<float4*>(P + 4 + 64 + 8 * l8);
+          lo[0] = make_float4(tot.acc[0].x, tot.acc[0].y, tot.acc[1].x, tot.acc[1].y);
+          lo[1] = make_float4(tot.acc[2].x, tot.acc[2].y, tot.acc[3].x, tot.acc[3].y);
+          hi[0] = make_float4(tot.acc[4].x, tot.acc[4].y, tot.acc[5].x, tot.acc[5].y);
+          hi[1] = make_float4(tot.acc[6].x, tot.acc[6].y, tot.acc[7].x, tot.acc[7].y);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(mail_bar + (leading ? 0 : 8));   // releases the writes above
+      }
+      begin = true;
+    }
+    share_walk_advance(cons, v, sh, n);
+    if (++stage == kStages) { stage = 0; parity ^= 1u; }
   }
 }
 
@@ -319,25 +533,42 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
 
 }  // namespace
 
+int decode_chunk_slots() { return kChunk; }
+
 int decode_max_workers() {
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+  } else {
+    cudaGetLastError();
   }
   if (sms < 148) sms = 148;  // size scratch for at least a full B200
-  return sms * kCtasPerSm * kWarps;
+  return sms * kWarps;
 }
 
-cudaError_t launch_decode(const DecodeParams& p_in, long total_valid, cudaStream_t st) {
+cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
+  static bool smem_set[64] = {};
+  static int max_workers[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < 64;
+  if (!cached || !smem_set[dev]) {
+    e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (cached) {
+      smem_set[dev] = true;
+      max_workers[dev] = decode_max_workers();
+    }
+  }
   DecodeParams p = p_in;
-  long w = decode_max_workers();
-  long cap = total_valid / kMinShare;
-  if (cap < 1) cap = 1;
-  if (w > cap) w = cap;
-  p.n_workers = (int)w;
-  int grid = (int)((w + kWarps - 1) / kWarps);
-  decode_kernel<<<grid, kThreads, 0, st>>>(p);
+  const long total = (long)p.view.cum[p.view.H] * p.view.n_seqs;
+  if (total < 1 || total > 0x7fffffffL) return cudaErrorInvalidValue;
+  const long w = plan_workers(total, cached ? max_workers[dev] : decode_max_workers());
+  p.split = make_split(total, w);
+  const int grid = (int)((w + kWarps - 1) / kWarps);
+  decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "ssd_b200.h"
+#include "ssd_plan.h"
 
 namespace ssd {
 
@@ -26,18 +27,14 @@ typedef int4 HeadDesc;
 
 struct DecodeParams {
   const uint4* slab;        // first slot of the layer
-  const HeadDesc* desc;     // [H] records of the layer
   const __nv_bfloat16* q;   // [n_seqs, H, 128]
   __nv_bfloat16* out;       // [n_seqs, H, 128]
-  float* partial;           // [n_workers * 2, kPartialFloats]
+  float* partial;           // [max workers * 2, kPartialFloats]
   uint32_t* counters;       // [n_seqs * H], zero between launches
-  int n_seqs, H, L;
-  int prompt_valid;         // 0 or L
-  int static_valid;         // valid static slots of semantic heads
-  int t_img;                // image tokens held (ring_valid = min(t_img, ring_cap))
-  int seq_slots;            // physical slots per sequence in this layer
-  int n_workers;            // warps that take a share of the work
+  uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
   float scale_log2;         // softmax scale * log2(e)
+  Split split;              // how the layer's slots are shared out (set by launch_decode)
+  LayerView view;           // layout and occupancy of the layer
 };
 
 struct AppendParams {
@@ -85,7 +82,7 @@ struct ClassifyParams {
   float scale_log2;
 };
 
-cudaError_t launch_decode(const DecodeParams& p, long total_valid, cudaStream_t st);
+cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
@@ -93,6 +90,7 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st);
 int classify_rows_per_block();
 int decode_max_workers();
+int decode_chunk_slots();
 
 void count_launch(int n = 1);
 

@@ -157,5 +157,6 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
     if errs:
         res.max_err = max(e[0] for e in errs)
         res.mean_err = float(np.mean([e[1] for e in errs]))
+    assert cache.device_status() == 0, "a decode warp gave up a bounded wait"
     cache.close()
     return res
