@@ -557,9 +557,9 @@ int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t
     if (sh.g_begin >= sh.g_end) continue;
     if (share_of(sp, sh.g_begin) != wk || share_of(sp, sh.g_end - 1) != wk) return SSD_ERR_BAD_STATE;
     Walk w;
-    share_walk_init(w, v, sh);
+    walk_init(w, v, sh.g_begin, sh.g_end);
     int64_t k = 0;
-    while (share_walk_more(w)) {
+    while (w.g < w.g_end) {
       const int nn = walk_chunk(w, chunk);
       if (nn < 1) return SSD_ERR_BAD_STATE;
       const int64_t hbase = (int64_t)w.seq * v.seq_slots + v.head[w.head].x;
@@ -572,7 +572,7 @@ int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t
       };
       if (v.contig) emit(w.i, 0, nn);   // the kernel's fast path: one copy per chunk
       else chunk_runs(v, w.head, w.i, nn, emit);
-      share_walk_advance(w, v, sh, nn);
+      walk_advance(w, v, nn);
       ++k;
     }
   }

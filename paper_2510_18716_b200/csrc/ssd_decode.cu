@@ -23,9 +23,8 @@
 //     the head belong to this CTA (workers of a CTA hold consecutive shares, so that is the usual
 //     case), through global scratch and an arrival counter for the at most two heads that cross
 //     the CTA's own range (last CTA to arrive merges; nobody waits for another CTA).  Merges run
-//     in worker order, then CTA order, so results do not depend on arrival order.  A worker takes
-//     the cut piece at the end of its share first, so all of this happens while the bulk of the
-//     streaming is still under way, and no streaming warp ever executes a fence or an atomic.
+//     in worker order, then CTA order, so results do not depend on arrival order, and no
+//     streaming warp ever executes a fence or an atomic.
 // Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
 // waits (bounded again) for its other copies in flight and leaves.
 #include "ssd_internal.cuh"
@@ -63,6 +62,7 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per w
 static_assert(kChunk % kGroups == 0 && kPer % kU == 0, "a stage is folded in groups of kGroups * kU slots");
 static_assert(kSmemBytes <= 227 * 1024, "stage rings exceed the shared memory of an SM");
 static_assert(kBarBytes % 16 == 0, "mailboxes are read as float4");
+static_assert(2 * kWarps <= 32, "the finisher plans one possible post per lane");
 
 // ------------------------------------------------------------------ asynchronous-copy plumbing
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -288,7 +288,7 @@ __device__ __forceinline__ void write_out4(__nv_bfloat16* out, float l, const fl
 // finisher stores the CTA's merged partial, counts arrivals per head with an atomic (it never
 // waits for another CTA) and, where this CTA was the last to arrive, merges the CTAs' partials
 // in CTA order.  All fences and atomics of the launch are issued here, off the streaming warps'
-// path.  Lane i holds output dimensions [4i, 4i + 4).
+// path.  While merging, lane i holds output dimensions [4i, 4i + 4).
 __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int lane) {
   const LayerView& v = p.view;
   const Split& sp = p.split;
@@ -296,33 +296,68 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   const float* mail = reinterpret_cast<const float*>(smem + kRingBytes + kBarBytes);
   const int lo_c = (int)blockIdx.x * kWarps;
   const int hi_c = (lo_c + kWarps < sp.W ? lo_c + kWarps : sp.W) - 1;
+
+  // Planning, one lane per possible post, before any post can have arrived: lane 2k looks at the
+  // cut piece at the end of worker k's share, lane 2k + 1 at the piece at its start.  A lane keeps
+  // the head only if its worker is the head's first contributor inside this CTA.
+  int r_pair = -1, r_g0 = 0, r_vh = 0, r_first = 0, r_last = 0, r_wlo = 0, r_whi = 0, r_locut = 0;
+  {
+    const int w = lo_c + (lane >> 1);
+    if ((lane >> 1) < kWarps && w <= hi_c) {
+      const Share sh = share_plan(v, sp, w);
+      Walk t;
+      int g_piece = -1;
+      if (sh.g_begin < sh.g_end) {
+        if ((lane & 1) == 0) {
+          if (sh.g_tail < sh.g_end) {
+            walk_init(t, v, sh.g_tail, sh.g_end);
+            g_piece = sh.g_tail;
+          }
+        } else if (sh.g_begin < sh.g_tail) {
+          walk_init(t, v, sh.g_begin, sh.g_tail);
+          if (t.i != 0) g_piece = sh.g_begin;    // its head began in an earlier share
+        }
+      }
+      if (g_piece >= 0) {
+        const int g0 = g_piece - t.i, g1 = g0 + t.vh;
+        const int w_lo = share_of(sp, g0), w_hi = share_of(sp, g1 - 1);
+        const int f = w_lo > lo_c ? w_lo : lo_c;
+        if (w == f) {
+          r_pair = t.seq * v.H + t.head;
+          r_g0 = g0;
+          r_vh = t.vh;
+          r_first = f;
+          r_last = w_hi < hi_c ? w_hi : hi_c;
+          r_wlo = w_lo;
+          r_whi = w_hi;
+          r_locut = share_start(sp, w_lo) < g0 ? 1 : 0;   // the head is worker w_lo's tail piece
+        }
+      }
+    }
+  }
+
   int n_glob = 0;                         // heads of this CTA that go through global scratch (<= 2)
   int my_pair = 0, my_g0 = 0, my_vh = 0;  // lane k keeps the record of the k-th of them
-  bool ok = true;
-
-  // worker `w` posts a partial of the head that covers logical slot g_piece (walk t points there)
-  auto handle = [&](int w, const Walk& t, int g_piece) {
-    if (!ok) return;
-    const int g0 = g_piece - t.i, g1 = g0 + t.vh;
-    const int w_lo = share_of(sp, g0), w_hi = share_of(sp, g1 - 1);
-    const int f = w_lo > lo_c ? w_lo : lo_c;       // first contributor inside this CTA
-    if (w != f) return;                            // the head is dealt with at that worker
-    const int e = w_hi < hi_c ? w_hi : hi_c;       // last contributor inside this CTA
+  unsigned heads = __ballot_sync(0xffffffffu, r_pair >= 0);
+  while (heads) {
+    const int src = __ffs(heads) - 1;
+    heads &= heads - 1;
+    const int pair = __shfl_sync(0xffffffffu, r_pair, src);
+    const int first = __shfl_sync(0xffffffffu, r_first, src), last = __shfl_sync(0xffffffffu, r_last, src);
+    const int w_lo = __shfl_sync(0xffffffffu, r_wlo, src), w_hi = __shfl_sync(0xffffffffu, r_whi, src);
+    const int locut = __shfl_sync(0xffffffffu, r_locut, src);
     float m = kNegBig, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j = f; j <= e; ++j) {
-      // the head is worker j's leading piece unless j's share starts before the head does
-      const int which = (j == w_lo && share_start(sp, j) < g0) ? 1 : 0;
-      const int box = (j - lo_c) * 2 + which;
+    for (int j = first; j <= last; ++j) {
+      // worker j holds the head as its leading piece, unless the head starts inside j's share
+      const int box = (j - lo_c) * 2 + ((j == w_lo && locut) ? 1 : 0);
       if (!mbar_wait(mail_bar0 + 8 * box, 0)) {
-        ok = false;
         if (lane == 0) atomicOr(p.status, 1u);
         return;
       }
       const float* P = mail + (size_t)box * kPartialFloats;
       merge4(m, l, acc, P[0], P[1], reinterpret_cast<const float4*>(P + 4)[lane]);
     }
-    const int pair = t.seq * v.H + t.head;
     if (w_lo >= lo_c && w_hi <= hi_c) {            // the whole head lies inside this CTA
       write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
     } else {
@@ -333,38 +368,25 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
         G[1] = l;
       }
       reinterpret_cast<float4*>(G + 4)[lane] = acc;
+      const int g0 = __shfl_sync(0xffffffffu, r_g0, src), vh = __shfl_sync(0xffffffffu, r_vh, src);
       if (lane == n_glob) {
         my_pair = pair;
         my_g0 = g0;
-        my_vh = t.vh;
+        my_vh = vh;
       }
       ++n_glob;
     }
-  };
-
-  for (int w = lo_c; w <= hi_c; ++w) {
-    const Share sh = share_plan(v, sp, w);
-    if (sh.g_begin >= sh.g_end) continue;
-    Walk t;
-    if (sh.g_tail < sh.g_end) {          // the cut piece at the end of the share
-      walk_init(t, v, sh.g_tail, sh.g_end);
-      handle(w, t, sh.g_tail);
-    }
-    if (sh.g_begin < sh.g_tail) {        // the piece at the start, if its head began earlier
-      walk_init(t, v, sh.g_begin, sh.g_tail);
-      if (t.i != 0) handle(w, t, sh.g_begin);
-    }
   }
-  if (!ok || n_glob == 0) return;
+  if (n_glob == 0) return;
 
   __threadfence();                       // the partials above, before the arrivals below
-  bool last = false;
+  bool last_in = false;
   if (lane < n_glob) {
     const int g0 = my_g0, g1 = g0 + my_vh;
     const uint32_t n_contrib = (uint32_t)(share_of(sp, g1 - 1) / kWarps - share_of(sp, g0) / kWarps + 1);
-    last = atomicAdd(p.counters + my_pair, 1u) == n_contrib - 1;
+    last_in = atomicAdd(p.counters + my_pair, 1u) == n_contrib - 1;
   }
-  unsigned todo = __ballot_sync(0xffffffffu, last);
+  unsigned todo = __ballot_sync(0xffffffffu, last_in);
   if (todo) __threadfence();
   while (todo) {
     const int src_lane = __ffs(todo) - 1;
@@ -407,15 +429,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   }
   const int wk = (int)blockIdx.x * kWarps + warp;
   if (wk >= p.split.W) return;
-  const Share sh = share_plan(v, p.split, wk);
-  if (sh.g_begin >= sh.g_end) return;
+  const int g_begin = share_start(p.split, wk), g_end = share_start(p.split, wk + 1);
+  if (g_begin >= g_end) return;
 
   unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
   const uint32_t ring_s = smem_u32(ring);
   float* mailbox = reinterpret_cast<float*>(smem + kRingBytes + kBarBytes) + (size_t)warp * 2 * kPartialFloats;
 
   Walk prod;
-  share_walk_init(prod, v, sh);
+  walk_init(prod, v, g_begin, g_end);
   Walk cons = prod;
   int ahead = 0;   // chunks issued and not yet consumed
 
@@ -423,7 +445,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   auto issue = [&](int stage) {
     const int n = walk_chunk(prod, kChunk);
     if (lane == 0) {
-      const bool begin = prod.i == 0 || prod.g == sh.g_begin;
+      const bool begin = prod.i == 0 || prod.g == g_begin;
       const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
       const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
                                    ((size_t)prod.seq * v.seq_slots + v.head[prod.head].x) * kSlotBytes;
@@ -441,12 +463,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       if (begin)
         bulk_g2s(dst + kChunk * kSlotBytes, p.q + ((size_t)prod.seq * v.H + prod.head) * kHeadDim, kQBytes, bar);
     }
-    share_walk_advance(prod, v, sh, n);
+    walk_advance(prod, v, n);
     ++ahead;
   };
 
 #pragma unroll 1
-  for (int s = 0; s < kStages && share_walk_more(prod); ++s) issue(s);
+  for (int s = 0; s < kStages && prod.g < g_end; ++s) issue(s);
 
   int stage = 0;
   uint32_t parity = 0;
@@ -456,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   State st;
 
 #pragma unroll 1
-  while (share_walk_more(cons)) {
+  while (cons.g < g_end) {
     const int n = walk_chunk(cons, kChunk);
     if (!mbar_wait(bar0 + 8 * stage, parity)) {
       // give up: flag it, let the copies still in flight land (bounded), and leave
@@ -477,18 +499,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
       state_init(st);
       piece_i0 = cons.i;
-      leading = cons.g == sh.g_begin;   // the piece that holds the share's first slot
+      leading = cons.g == g_begin;      // the piece that holds the share's first slot
       begin = false;
     }
     Rows rows;
     load_stage(sb, n, grp, l8, rows);
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
-    if (share_walk_more(prod)) issue(stage);
+    if (prod.g < g_end) issue(stage);
     fold_stage(rows, n, grp, q, st);
 
     const int i1 = cons.i + n;
-    if (i1 == cons.vh || cons.g + n == cons.g_end) {
+    if (i1 == cons.vh || cons.g + n == g_end) {
       // end of this worker's piece of the head: merge the four groups (lanes l, l^8, l^16, l^24
       // hold the same 16 output dims), then write the output, or post a partial to the finisher
       State tot = st;
@@ -515,7 +537,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       }
       begin = true;
     }
-    share_walk_advance(cons, v, sh, n);
+    walk_advance(cons, v, n);
     if (++stage == kStages) { stage = 0; parity ^= 1u; }
   }
 }

@@ -142,11 +142,10 @@ SSD_HD void walk_advance(Walk& w, const LayerView& v, int n) {
   }
 }
 
-// Order in which a worker takes its share [g_begin, g_end).  If the head at the end of the share is
-// cut by the share boundary (the next worker holds the rest of it), that tail piece [g_tail, g_end)
-// is taken first and the rest [g_begin, g_tail) afterwards: every piece that needs a cross-worker
-// merge is then finished early in the launch, and the merges overlap with the remaining streaming
-// instead of trailing it.  g_tail == g_end when the last head is not cut.
+// A worker's share [g_begin, g_end), walked in stream order.  If the head at the end of the share is
+// cut by the share boundary (the next worker holds the rest of it), g_tail is where the worker's
+// piece of that head starts (g_begin if the head began in an earlier share); g_tail == g_end when
+// the last head is not cut.
 struct Share {
   int32_t g_begin, g_end, g_tail;
 };
@@ -163,22 +162,6 @@ SSD_HD Share share_plan(const LayerView& v, const Split& sp, int32_t wk) {
     if (head_start + w.vh > s.g_end) s.g_tail = head_start > s.g_begin ? head_start : s.g_begin;
   }
   return s;
-}
-
-// Start the walk over a share, in the order described above (w.g_end is the end of the current part).
-SSD_HD void share_walk_init(Walk& w, const LayerView& v, const Share& s) {
-  if (s.g_tail < s.g_end) walk_init(w, v, s.g_tail, s.g_end);
-  else walk_init(w, v, s.g_begin, s.g_end);
-}
-
-// True while the walk has slots left.
-SSD_HD bool share_walk_more(const Walk& w) { return w.g < w.g_end; }
-
-SSD_HD void share_walk_advance(Walk& w, const LayerView& v, const Share& s, int n) {
-  walk_advance(w, v, n);
-  // the tail piece is done: go back for the part before it (it ends on a head boundary)
-  if (w.g == s.g_end && w.g_end == s.g_end && s.g_tail < s.g_end && s.g_begin < s.g_tail)
-    walk_init(w, v, s.g_begin, s.g_tail);
 }
 
 // Physical runs that make up valid slots [i, i + n) of head h.  emit(src, dst, len) is called once
