@@ -177,6 +177,8 @@ int ssd_cache_device_status(ssd_cache *cache, uint32_t *status_host);
  *   tokens held; max_workers warps available; chunk slots per copy stage (0 = the kernel's own)
  *   copies_out [cap][6] = {worker, chunk number within the worker, source slot (from the layer's
  *             first slot), destination slot within the stage, slots copied, sequence*n_heads+head}
+ * Copies are listed in stream order per worker; the kernel issues the same copies, except that a
+ * worker whose last head runs past its thread block's range starts with that head's piece.
  * Returns the number of copies (which may exceed cap; only the first cap are written) or a negative
  * ssd_status.  No paper counterpart. */
 int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t *head_recs, int32_t prompt_len,

@@ -96,15 +96,11 @@ struct ssd_cache {
     v.prompt_valid = prompt_valid[layer];
     v.static_valid = static_valid[layer];
     v.t_img = t_img[layer];
-    int run = 0;
     for (int h = 0; h < cfg.n_heads; ++h) {
       const HeadDesc& d = desc[(size_t)layer * cfg.n_heads + h];
       v.head[h] = HeadRec{d.x, d.y, d.z, d.w};
-      v.cum[h] = run;
-      run += head_valid(v, h);
     }
-    v.cum[cfg.n_heads] = run;
-    v.contig = view_contiguous(v) ? 1 : 0;
+    view_finish(v);
   }
 };
 
@@ -533,19 +529,17 @@ int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t
   LayerView v;
   v.H = n_heads; v.L = prompt_len; v.n_seqs = n_seqs;
   v.prompt_valid = prompt_valid; v.static_valid = static_valid; v.t_img = t_img;
-  int off = 0, run = 0;
+  int off = 0;
   for (int h = 0; h < n_heads; ++h) {
     const int32_t* r = head_recs + 4 * h;
     if (r[1] < 0 || r[2] < 1 || r[0] != off || (r[3] == 0 && r[1] != 0) || (r[3] != 0 && static_valid > r[1]))
       return SSD_ERR_INVALID_ARG;
     v.head[h] = HeadRec{r[0], r[1], r[2], r[3]};
     off += prompt_len + r[1] + r[2];
-    v.cum[h] = run;
-    run += head_valid(v, h);
   }
-  v.cum[n_heads] = run;
   v.seq_slots = off;
-  v.contig = view_contiguous(v) ? 1 : 0;
+  view_finish(v);
+  const int run = v.cum[n_heads];
   const long T = (long)run * n_seqs;
   if (T < 1) return SSD_ERR_BAD_STATE;
   if (T > 0x7fffffffL) return SSD_ERR_INVALID_ARG;

@@ -300,7 +300,7 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   // Planning, one lane per possible post, before any post can have arrived: lane 2k looks at the
   // cut piece at the end of worker k's share, lane 2k + 1 at the piece at its start.  A lane keeps
   // the head only if its worker is the head's first contributor inside this CTA.
-  int r_pair = -1, r_g0 = 0, r_vh = 0, r_first = 0, r_last = 0, r_wlo = 0, r_whi = 0, r_locut = 0;
+  int r_pair = -1, r_first = 0, r_last = 0, r_wlo = 0, r_whi = 0, r_locut = 0;
   {
     const int w = lo_c + (lane >> 1);
     if ((lane >> 1) < kWarps && w <= hi_c) {
@@ -324,8 +324,6 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
         const int f = w_lo > lo_c ? w_lo : lo_c;
         if (w == f) {
           r_pair = t.seq * v.H + t.head;
-          r_g0 = g0;
-          r_vh = t.vh;
           r_first = f;
           r_last = w_hi < hi_c ? w_hi : hi_c;
           r_wlo = w_lo;
@@ -336,73 +334,81 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
     }
   }
 
-  int n_glob = 0;                         // heads of this CTA that go through global scratch (<= 2)
-  int my_pair = 0, my_g0 = 0, my_vh = 0;  // lane k keeps the record of the k-th of them
-  unsigned heads = __ballot_sync(0xffffffffu, r_pair >= 0);
-  while (heads) {
-    const int src = __ffs(heads) - 1;
-    heads &= heads - 1;
-    const int pair = __shfl_sync(0xffffffffu, r_pair, src);
-    const int first = __shfl_sync(0xffffffffu, r_first, src), last = __shfl_sync(0xffffffffu, r_last, src);
-    const int w_lo = __shfl_sync(0xffffffffu, r_wlo, src), w_hi = __shfl_sync(0xffffffffu, r_whi, src);
-    const int locut = __shfl_sync(0xffffffffu, r_locut, src);
-    float m = kNegBig, l = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const uint32_t FULL = 0xffffffffu;
+  const bool r_global = r_pair >= 0 && (r_wlo < lo_c || r_whi > hi_c);
+
+  // merge, in worker order, the partials this CTA's workers hold of the head planned by lane `src`
+  auto merge_local = [&](int src, float& m, float& l, float4& acc) -> bool {
+    const int first = __shfl_sync(FULL, r_first, src), last = __shfl_sync(FULL, r_last, src);
+    const int w_lo = __shfl_sync(FULL, r_wlo, src), locut = __shfl_sync(FULL, r_locut, src);
+    m = kNegBig;
+    l = 0.f;
+    acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j = first; j <= last; ++j) {
       // worker j holds the head as its leading piece, unless the head starts inside j's share
       const int box = (j - lo_c) * 2 + ((j == w_lo && locut) ? 1 : 0);
       if (!mbar_wait(mail_bar0 + 8 * box, 0)) {
         if (lane == 0) atomicOr(p.status, 1u);
-        return;
+        return false;
       }
       const float* P = mail + (size_t)box * kPartialFloats;
       merge4(m, l, acc, P[0], P[1], reinterpret_cast<const float4*>(P + 4)[lane]);
     }
-    if (w_lo >= lo_c && w_hi <= hi_c) {            // the whole head lies inside this CTA
-      write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
-    } else {
+    return true;
+  };
+
+  // 1. heads that cross this CTA's range (at most two; their pieces are taken early by the workers)
+  unsigned heads = __ballot_sync(FULL, r_global);
+  const int n_glob = __popc(heads);
+  if (n_glob) {
+    while (heads) {
+      const int src = __ffs(heads) - 1;
+      heads &= heads - 1;
+      float m, l;
+      float4 acc;
+      if (!merge_local(src, m, l, acc)) return;
       // slot 0: the head began in an earlier CTA; slot 1: it begins here and runs on
+      const int w_lo = __shfl_sync(FULL, r_wlo, src);
       float* G = p.partial + ((size_t)blockIdx.x * 2 + (w_lo < lo_c ? 0 : 1)) * kPartialFloats;
       if (lane == 0) {
         G[0] = m;
         G[1] = l;
       }
       reinterpret_cast<float4*>(G + 4)[lane] = acc;
-      const int g0 = __shfl_sync(0xffffffffu, r_g0, src), vh = __shfl_sync(0xffffffffu, r_vh, src);
-      if (lane == n_glob) {
-        my_pair = pair;
-        my_g0 = g0;
-        my_vh = vh;
+    }
+    __threadfence();                     // the partials above, before the arrivals below
+    bool last_in = false;
+    if (r_global) {
+      const uint32_t n_contrib = (uint32_t)(r_whi / kWarps - r_wlo / kWarps + 1);
+      last_in = atomicAdd(p.counters + r_pair, 1u) == n_contrib - 1;
+    }
+    unsigned todo = __ballot_sync(FULL, last_in);
+    if (todo) __threadfence();
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int pair = __shfl_sync(FULL, r_pair, src);
+      const int c_lo = __shfl_sync(FULL, r_wlo, src) / kWarps, c_hi = __shfl_sync(FULL, r_whi, src) / kWarps;
+      float m = kNegBig, l = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int c = c_lo; c <= c_hi; ++c) {
+        const float* G = p.partial + ((size_t)c * 2 + (c > c_lo ? 0 : 1)) * kPartialFloats;
+        merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
       }
-      ++n_glob;
+      write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
+      if (lane == 0) p.counters[pair] = 0u;
     }
   }
-  if (n_glob == 0) return;
 
-  __threadfence();                       // the partials above, before the arrivals below
-  bool last_in = false;
-  if (lane < n_glob) {
-    const int g0 = my_g0, g1 = g0 + my_vh;
-    const uint32_t n_contrib = (uint32_t)(share_of(sp, g1 - 1) / kWarps - share_of(sp, g0) / kWarps + 1);
-    last_in = atomicAdd(p.counters + my_pair, 1u) == n_contrib - 1;
-  }
-  unsigned todo = __ballot_sync(0xffffffffu, last_in);
-  if (todo) __threadfence();
-  while (todo) {
-    const int src_lane = __ffs(todo) - 1;
-    todo &= todo - 1;
-    const int pair = __shfl_sync(0xffffffffu, my_pair, src_lane);
-    const int g0 = __shfl_sync(0xffffffffu, my_g0, src_lane);
-    const int g1 = g0 + __shfl_sync(0xffffffffu, my_vh, src_lane);
-    const int c_lo = share_of(sp, g0) / kWarps, c_hi = share_of(sp, g1 - 1) / kWarps;
-    float m = kNegBig, l = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = c_lo; c <= c_hi; ++c) {
-      const float* G = p.partial + ((size_t)c * 2 + (c > c_lo ? 0 : 1)) * kPartialFloats;
-      merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
-    }
-    write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
-    if (lane == 0) p.counters[pair] = 0u;
+  // 2. heads cut only between workers of this CTA
+  heads = __ballot_sync(FULL, r_pair >= 0 && !r_global);
+  while (heads) {
+    const int src = __ffs(heads) - 1;
+    heads &= heads - 1;
+    float m, l;
+    float4 acc;
+    if (!merge_local(src, m, l, acc)) return;
+    write_out4(p.out + (size_t)__shfl_sync(FULL, r_pair, src) * kHeadDim, l, acc, lane);
   }
 }
 
@@ -431,13 +437,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   if (wk >= p.split.W) return;
   const int g_begin = share_start(p.split, wk), g_end = share_start(p.split, wk + 1);
   if (g_begin >= g_end) return;
+  // If the head at the end of the share runs past this CTA's range, its merge goes through global
+  // memory: take that piece first ([g_tail, g_end), then [g_begin, g_tail)) so that the merge's
+  // latency is hidden behind the rest of the streaming.  Otherwise stream order (g_tail == g_end).
+  int g_tail = g_end;
+  {
+    const int w_next = ((int)blockIdx.x + 1) * kWarps < p.split.W ? ((int)blockIdx.x + 1) * kWarps : p.split.W;
+    const int cta_end = share_start(p.split, w_next);
+    if (cta_end - g_end < v.max_vh) {
+      Walk t;
+      walk_init(t, v, g_end - 1, g_end);
+      const int head_start = g_end - 1 - t.i;
+      if (head_start + t.vh > cta_end) g_tail = head_start > g_begin ? head_start : g_begin;
+    }
+  }
+  const bool two_parts = g_begin < g_tail && g_tail < g_end;
+  auto advance = [&](Walk& w, int n) {
+    walk_advance(w, v, n);
+    if (two_parts && w.g == g_end && w.g_end == g_end) walk_init(w, v, g_begin, g_tail);
+  };
 
   unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
   const uint32_t ring_s = smem_u32(ring);
   float* mailbox = reinterpret_cast<float*>(smem + kRingBytes + kBarBytes) + (size_t)warp * 2 * kPartialFloats;
 
   Walk prod;
-  walk_init(prod, v, g_begin, g_end);
+  walk_init(prod, v, two_parts ? g_tail : g_begin, g_end);
   Walk cons = prod;
   int ahead = 0;   // chunks issued and not yet consumed
 
@@ -463,12 +488,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       if (begin)
         bulk_g2s(dst + kChunk * kSlotBytes, p.q + ((size_t)prod.seq * v.H + prod.head) * kHeadDim, kQBytes, bar);
     }
-    walk_advance(prod, v, n);
+    advance(prod, n);
     ++ahead;
   };
 
 #pragma unroll 1
-  for (int s = 0; s < kStages && prod.g < g_end; ++s) issue(s);
+  for (int s = 0; s < kStages && prod.g < prod.g_end; ++s) issue(s);
 
   int stage = 0;
   uint32_t parity = 0;
@@ -478,7 +503,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   State st;
 
 #pragma unroll 1
-  while (cons.g < g_end) {
+  while (cons.g < cons.g_end) {
     const int n = walk_chunk(cons, kChunk);
     if (!mbar_wait(bar0 + 8 * stage, parity)) {
       // give up: flag it, let the copies still in flight land (bounded), and leave
@@ -506,11 +531,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     load_stage(sb, n, grp, l8, rows);
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
-    if (prod.g < g_end) issue(stage);
+    if (prod.g < prod.g_end) issue(stage);
     fold_stage(rows, n, grp, q, st);
 
     const int i1 = cons.i + n;
-    if (i1 == cons.vh || cons.g + n == g_end) {
+    if (i1 == cons.vh || cons.g + n == cons.g_end) {
       // end of this worker's piece of the head: merge the four groups (lanes l, l^8, l^16, l^24
       // hold the same 16 output dims), then write the output, or post a partial to the finisher
       State tot = st;
@@ -537,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       }
       begin = true;
     }
-    walk_advance(cons, v, n);
+    advance(cons, n);
     if (++stage == kStages) { stage = 0; parity ^= 1u; }
   }
 }

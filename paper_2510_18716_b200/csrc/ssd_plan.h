@@ -37,6 +37,7 @@ struct LayerView {
   int32_t static_valid;             // valid static slots of semantic heads
   int32_t t_img;                    // image tokens held; a ring holds min(t_img, z) of them
   int32_t contig;                   // 1 if every head's valid slots are one run from its first slot
+  int32_t max_vh;                   // most valid slots any head holds
   int32_t cum[kPlanMaxHeads + 1];   // exclusive prefix of valid slots per head
   HeadRec head[kPlanMaxHeads];
 };
@@ -47,6 +48,9 @@ SSD_HD int head_valid(const LayerView& v, int h) {
   return v.prompt_valid + (d.w ? v.static_valid : 0) + rv;
 }
 
+// Fill the fields derived from the others: cum[], max_vh, contig.
+inline void view_finish(LayerView& v);
+
 // True if, for every head, the valid slots are physically contiguous from the head's first slot:
 // the prompt is loaded (or there is none) and the static set of semantic heads is full.
 inline bool view_contiguous(const LayerView& v) {
@@ -54,6 +58,19 @@ inline bool view_contiguous(const LayerView& v) {
   for (int h = 0; h < v.H; ++h)
     if (v.head[h].w && v.static_valid != v.head[h].y) return false;
   return true;
+}
+
+inline void view_finish(LayerView& v) {
+  int run = 0, mx = 0;
+  for (int h = 0; h < v.H; ++h) {
+    v.cum[h] = run;
+    const int n = head_valid(v, h);
+    run += n;
+    if (n > mx) mx = n;
+  }
+  v.cum[v.H] = run;
+  v.max_vh = mx;
+  v.contig = view_contiguous(v) ? 1 : 0;
 }
 
 // How the stream of T valid slots is cut into W shares.  Share i starts at floor(i * T / W) rounded
