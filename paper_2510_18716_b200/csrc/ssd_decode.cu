@@ -18,13 +18,16 @@
 //     two-wide fp32 FMAs, three shuffles per dot product, and an online softmax in fp32 (base-2
 //     exponent, scale folded into q);
 //   * a head that lies inside one share is finished in registers.  A head cut by a share boundary
-//     leaves a partial (m, l, acc[128]) in the worker's shared-memory mailbox, and an extra
-//     finisher warp per CTA merges the partials: straight from shared memory when all pieces of
-//     the head belong to this CTA (workers of a CTA hold consecutive shares, so that is the usual
-//     case), through global scratch and an arrival counter for the at most two heads that cross
-//     the CTA's own range (last CTA to arrive merges; nobody waits for another CTA).  Merges run
-//     in worker order, then CTA order, so results do not depend on arrival order, and no
-//     streaming warp ever executes a fence or an atomic.
+//     leaves a partial (m, l, acc[128]) in the worker's shared-memory mailbox.  Workers of a CTA
+//     hold consecutive shares, so the pieces of such a head usually all belong to one CTA: the
+//     worker that posts the last of them (shared-memory arrival counter, nobody waits) merges
+//     them in worker order and writes the output.  For the at most two heads that cross the CTA's
+//     own range, that worker hands the CTA's merged partial to an extra finisher warp, which
+//     carries it through global scratch and a global arrival counter (last CTA to arrive merges,
+//     in CTA order; no CTA waits for another).  Results therefore do not depend on arrival
+//     order, and no streaming warp executes a global fence or atomic.  A worker whose last head
+//     runs past the CTA's range takes that piece first, which hides the global merge's latency
+//     behind the rest of the streaming.
 // Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
 // waits (bounded again) for its other copies in flight and leaves.
 #include "ssd_internal.cuh"
@@ -53,9 +56,11 @@ constexpr int kU = kPer < 4 ? kPer : 4;              // slots a group folds in a
 constexpr int kQBytes = kHeadDim * 2;
 constexpr int kStageBytes = kChunk * kSlotBytes + kQBytes;
 constexpr int kRingBytes = kWarps * kStages * kStageBytes;
-constexpr int kBarBytes = (kWarps * kStages + kWarps * 2) * 8;   // stage barriers, then mailbox barriers
-constexpr int kMailBytes = kWarps * 2 * kPartialFloats * 4;      // two partials per worker
-constexpr int kSmemBytes = kRingBytes + kBarBytes + kMailBytes;
+constexpr int kBarBytes = (kWarps * kStages + 2) * 8;            // stage barriers, then the finisher's two
+constexpr int kMailBoxes = kWarps * 2 + 2;                       // two partials per worker, two for the CTA
+constexpr int kMailBytes = kMailBoxes * kPartialFloats * 4;
+constexpr int kCountBytes = kWarps * 2 * 4;                      // arrival counter per (first worker, slot)
+constexpr int kSmemBytes = kRingBytes + kBarBytes + kMailBytes + kCountBytes;
 constexpr float kNegBig = -1.0e30f;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait, then give up
 
@@ -63,6 +68,7 @@ static_assert(kChunk % kGroups == 0 && kPer % kU == 0, "a stage is folded in gro
 static_assert(kSmemBytes <= 227 * 1024, "stage rings exceed the shared memory of an SM");
 static_assert(kBarBytes % 16 == 0, "mailboxes are read as float4");
 static_assert(2 * kWarps <= 32, "the finisher plans one possible post per lane");
+static_assert((kWarps * kStages) % 2 == 0, "keeps the mailboxes 16-byte aligned");
 
 // ------------------------------------------------------------------ asynchronous-copy plumbing
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -281,134 +287,80 @@ __device__ __forceinline__ void write_out4(__nv_bfloat16* out, float l, const fl
   reinterpret_cast<uint2*>(out)[lane] = o;
 }
 
-// The finisher warp of a CTA.  The CTA's workers hold consecutive shares, so most heads that are
-// cut by a share boundary are cut between two workers of the same CTA: the finisher merges their
-// partials straight from the shared-memory mailboxes, in worker order, and writes the output.
-// Only the (at most two) heads that cross the CTA's own range go through global scratch: the
-// finisher stores the CTA's merged partial, counts arrivals per head with an atomic (it never
-// waits for another CTA) and, where this CTA was the last to arrive, merges the CTAs' partials
-// in CTA order.  All fences and atomics of the launch are issued here, off the streaming warps'
-// path.  While merging, lane i holds output dimensions [4i, 4i + 4).
+// Which workers hold pieces of the head that spans logical slots [g0, g1), found by stepping from
+// a worker `wk` known to hold one of them.
+__device__ __forceinline__ void head_workers(const Split& sp, int wk, int g0, int g1, int& w_lo, int& w_hi) {
+  w_lo = wk;
+  while (w_lo > 0 && share_start(sp, w_lo) > g0) --w_lo;
+  w_hi = wk;
+  while (w_hi + 1 < sp.W && share_start(sp, w_hi + 1) < g1) ++w_hi;
+}
+
+// The finisher warp of a CTA carries the (at most two) heads that cross the CTA's own range
+// through global memory: it waits for the CTA's merged partial of such a head (left in a shared-
+// memory mailbox by the worker that completed it), stores it in global scratch, counts arrivals
+// per head with an atomic (it never waits for another CTA) and, where this CTA was the last to
+// arrive, merges the CTAs' partials in CTA order.  All global fences and atomics of the launch
+// are issued here, off the streaming warps' path.  Lane i holds output dimensions [4i, 4i + 4).
 __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int lane) {
   const LayerView& v = p.view;
   const Split& sp = p.split;
-  const uint32_t mail_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
-  const float* mail = reinterpret_cast<const float*>(smem + kRingBytes + kBarBytes);
+  const uint32_t FULL = 0xffffffffu;
+  const uint32_t cta_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
+  const float* cta_mail = reinterpret_cast<const float*>(smem + kRingBytes + kBarBytes) +
+                          (size_t)kWarps * 2 * kPartialFloats;
   const int lo_c = (int)blockIdx.x * kWarps;
   const int hi_c = (lo_c + kWarps < sp.W ? lo_c + kWarps : sp.W) - 1;
+  const int r_begin = share_start(sp, lo_c), r_end = share_start(sp, hi_c + 1);   // the CTA's range
 
-  // Planning, one lane per possible post, before any post can have arrived: lane 2k looks at the
-  // cut piece at the end of worker k's share, lane 2k + 1 at the piece at its start.  A lane keeps
-  // the head only if its worker is the head's first contributor inside this CTA.
-  int r_pair = -1, r_first = 0, r_last = 0, r_wlo = 0, r_whi = 0, r_locut = 0;
-  {
-    const int w = lo_c + (lane >> 1);
-    if ((lane >> 1) < kWarps && w <= hi_c) {
-      const Share sh = share_plan(v, sp, w);
-      Walk t;
-      int g_piece = -1;
-      if (sh.g_begin < sh.g_end) {
-        if ((lane & 1) == 0) {
-          if (sh.g_tail < sh.g_end) {
-            walk_init(t, v, sh.g_tail, sh.g_end);
-            g_piece = sh.g_tail;
-          }
-        } else if (sh.g_begin < sh.g_tail) {
-          walk_init(t, v, sh.g_begin, sh.g_tail);
-          if (t.i != 0) g_piece = sh.g_begin;    // its head began in an earlier share
-        }
-      }
-      if (g_piece >= 0) {
-        const int g0 = g_piece - t.i, g1 = g0 + t.vh;
-        const int w_lo = share_of(sp, g0), w_hi = share_of(sp, g1 - 1);
-        const int f = w_lo > lo_c ? w_lo : lo_c;
-        if (w == f) {
-          r_pair = t.seq * v.H + t.head;
-          r_first = f;
-          r_last = w_hi < hi_c ? w_hi : hi_c;
-          r_wlo = w_lo;
-          r_whi = w_hi;
-          r_locut = share_start(sp, w_lo) < g0 ? 1 : 0;   // the head is worker w_lo's tail piece
-        }
-      }
+  // lane 0: the head that covers the range's first slot, if it began earlier; lane 1: the head
+  // that covers its last slot, if it runs on (and is not the same head)
+  int r_pair = -1, r_clo = 0, r_chi = 0;
+  if (lane < 2 && r_begin < r_end) {
+    Walk t;
+    const int g = lane == 0 ? r_begin : r_end - 1;
+    walk_init(t, v, g, r_end);
+    const int g0 = g - t.i, g1 = g0 + t.vh;
+    const bool crosses = lane == 0 ? g0 < r_begin : (g1 > r_end && g0 >= r_begin);
+    if (crosses) {
+      int w_lo, w_hi;
+      head_workers(sp, lane == 0 ? lo_c : hi_c, g0, g1, w_lo, w_hi);
+      r_pair = t.seq * v.H + t.head;
+      r_clo = w_lo / kWarps;
+      r_chi = w_hi / kWarps;
     }
   }
-
-  const uint32_t FULL = 0xffffffffu;
-  const bool r_global = r_pair >= 0 && (r_wlo < lo_c || r_whi > hi_c);
-
-  // merge, in worker order, the partials this CTA's workers hold of the head planned by lane `src`
-  auto merge_local = [&](int src, float& m, float& l, float4& acc) -> bool {
-    const int first = __shfl_sync(FULL, r_first, src), last = __shfl_sync(FULL, r_last, src);
-    const int w_lo = __shfl_sync(FULL, r_wlo, src), locut = __shfl_sync(FULL, r_locut, src);
-    m = kNegBig;
-    l = 0.f;
-    acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int j = first; j <= last; ++j) {
-      // worker j holds the head as its leading piece, unless the head starts inside j's share
-      const int box = (j - lo_c) * 2 + ((j == w_lo && locut) ? 1 : 0);
-      if (!mbar_wait(mail_bar0 + 8 * box, 0)) {
-        if (lane == 0) atomicOr(p.status, 1u);
-        return false;
-      }
-      const float* P = mail + (size_t)box * kPartialFloats;
-      merge4(m, l, acc, P[0], P[1], reinterpret_cast<const float4*>(P + 4)[lane]);
+  unsigned heads = __ballot_sync(FULL, r_pair >= 0);
+  if (!heads) return;
+  for (unsigned h = heads; h; h &= h - 1) {
+    const int slot = __ffs(h) - 1;       // 0: began in an earlier CTA, 1: begins here and runs on
+    if (!mbar_wait(cta_bar0 + 8 * slot, 0)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      return;
     }
-    return true;
-  };
-
-  // 1. heads that cross this CTA's range (at most two; their pieces are taken early by the workers)
-  unsigned heads = __ballot_sync(FULL, r_global);
-  const int n_glob = __popc(heads);
-  if (n_glob) {
-    while (heads) {
-      const int src = __ffs(heads) - 1;
-      heads &= heads - 1;
-      float m, l;
-      float4 acc;
-      if (!merge_local(src, m, l, acc)) return;
-      // slot 0: the head began in an earlier CTA; slot 1: it begins here and runs on
-      const int w_lo = __shfl_sync(FULL, r_wlo, src);
-      float* G = p.partial + ((size_t)blockIdx.x * 2 + (w_lo < lo_c ? 0 : 1)) * kPartialFloats;
-      if (lane == 0) {
-        G[0] = m;
-        G[1] = l;
-      }
-      reinterpret_cast<float4*>(G + 4)[lane] = acc;
-    }
-    __threadfence();                     // the partials above, before the arrivals below
-    bool last_in = false;
-    if (r_global) {
-      const uint32_t n_contrib = (uint32_t)(r_whi / kWarps - r_wlo / kWarps + 1);
-      last_in = atomicAdd(p.counters + r_pair, 1u) == n_contrib - 1;
-    }
-    unsigned todo = __ballot_sync(FULL, last_in);
-    if (todo) __threadfence();
-    while (todo) {
-      const int src = __ffs(todo) - 1;
-      todo &= todo - 1;
-      const int pair = __shfl_sync(FULL, r_pair, src);
-      const int c_lo = __shfl_sync(FULL, r_wlo, src) / kWarps, c_hi = __shfl_sync(FULL, r_whi, src) / kWarps;
-      float m = kNegBig, l = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int c = c_lo; c <= c_hi; ++c) {
-        const float* G = p.partial + ((size_t)c * 2 + (c > c_lo ? 0 : 1)) * kPartialFloats;
-        merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
-      }
-      write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
-      if (lane == 0) p.counters[pair] = 0u;
-    }
+    const float4* src = reinterpret_cast<const float4*>(cta_mail + (size_t)slot * kPartialFloats);
+    float4* dst = reinterpret_cast<float4*>(p.partial + ((size_t)blockIdx.x * 2 + slot) * kPartialFloats);
+    dst[1 + lane] = src[1 + lane];
+    if (lane == 0) dst[0] = src[0];
   }
-
-  // 2. heads cut only between workers of this CTA
-  heads = __ballot_sync(FULL, r_pair >= 0 && !r_global);
-  while (heads) {
-    const int src = __ffs(heads) - 1;
-    heads &= heads - 1;
-    float m, l;
-    float4 acc;
-    if (!merge_local(src, m, l, acc)) return;
-    write_out4(p.out + (size_t)__shfl_sync(FULL, r_pair, src) * kHeadDim, l, acc, lane);
+  __threadfence();                       // the partials above, before the arrivals below
+  bool last_in = false;
+  if (r_pair >= 0) last_in = atomicAdd(p.counters + r_pair, 1u) == (uint32_t)(r_chi - r_clo);
+  unsigned todo = __ballot_sync(FULL, last_in);
+  if (todo) __threadfence();
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int pair = __shfl_sync(FULL, r_pair, src);
+    const int c_lo = __shfl_sync(FULL, r_clo, src), c_hi = __shfl_sync(FULL, r_chi, src);
+    float m = kNegBig, l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = c_lo; c <= c_hi; ++c) {
+      const float* G = p.partial + ((size_t)c * 2 + (c > c_lo ? 0 : 1)) * kPartialFloats;
+      merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
+    }
+    write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
+    if (lane == 0) p.counters[pair] = 0u;
   }
 }
 
@@ -419,15 +371,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const int grp = lane >> 3, l8 = lane & 7;
 
   const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
-  const uint32_t mail_bar = smem_u32(smem + kRingBytes) + kWarps * kStages * 8 + (uint32_t)warp * 16;
-  if (warp < kWarps && lane == 0) {
+  const uint32_t cta_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
+  float* mail = reinterpret_cast<float*>(smem + kRingBytes + kBarBytes);
+  int* arrivals = reinterpret_cast<int*>(smem + kRingBytes + kBarBytes + kMailBytes);
+  if (lane == 0) {
+    if (warp < kWarps) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
-    mbar_init(mail_bar, 1);
-    mbar_init(mail_bar + 8, 1);
+      for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+      arrivals[2 * warp] = 0;
+      arrivals[2 * warp + 1] = 0;
+    } else {
+      mbar_init(cta_bar0, 1);
+      mbar_init(cta_bar0 + 8, 1);
+    }
     mbar_init_fence();
   }
-  __syncthreads();   // the only CTA-wide barrier: mailboxes exist before anyone posts or waits
+  __syncthreads();   // the only CTA-wide barrier: counters and barriers exist before anyone uses them
 
   if (warp == kWarps) {
     finisher(p, smem, lane);
@@ -459,7 +418,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
   unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
   const uint32_t ring_s = smem_u32(ring);
-  float* mailbox = reinterpret_cast<float*>(smem + kRingBytes + kBarBytes) + (size_t)warp * 2 * kPartialFloats;
+  const int lo_c = (int)blockIdx.x * kWarps;
+  const int hi_c = (lo_c + kWarps < p.split.W ? lo_c + kWarps : p.split.W) - 1;
 
   Walk prod;
   walk_init(prod, v, two_parts ? g_tail : g_begin, g_end);
@@ -544,7 +504,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       if (piece_i0 == 0 && i1 == cons.vh) {
         if (grp == 0) write_out(p.out + ((size_t)cons.seq * v.H + cons.head) * kHeadDim, tot, l8);
       } else {
-        float* P = mailbox + (leading ? 0 : 1) * kPartialFloats;
+        // post the partial; the worker that posts a head's last piece in this CTA merges them
+        float* P = mail + (size_t)(2 * warp + (leading ? 0 : 1)) * kPartialFloats;
         if (lane == 0) {
           P[0] = tot.m;
           P[1] = tot.l;
@@ -557,8 +518,42 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
           hi[0] = make_float4(tot.acc[4].x, tot.acc[4].y, tot.acc[5].x, tot.acc[5].y);
           hi[1] = make_float4(tot.acc[6].x, tot.acc[6].y, tot.acc[7].x, tot.acc[7].y);
         }
+        const int g0 = cons.g - cons.i, g1 = g0 + cons.vh;    // the whole head in the stream
+        int w_lo, w_hi;
+        head_workers(p.split, wk, g0, g1, w_lo, w_hi);
+        const int f = w_lo > lo_c ? w_lo : lo_c, e = w_hi < hi_c ? w_hi : hi_c;   // holders in this CTA
+        // worker j holds the head in its slot 0 (leading piece), unless the head starts inside j's share
+        const int locut = share_start(p.split, w_lo) < g0 ? 1 : 0;
+        const int f_box = (f - lo_c) * 2 + ((f == w_lo && locut) ? 1 : 0);
         __syncwarp();
-        if (lane == 0) mbar_arrive(mail_bar + (leading ? 0 : 8));   // releases the writes above
+        int old = 0;
+        if (lane == 0) {
+          __threadfence_block();
+          old = atomicAdd(arrivals + f_box, 1);
+        }
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if (old == e - f) {
+          __threadfence_block();
+          float m = kNegBig, l = 0.f;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int j = f; j <= e; ++j) {
+            const float* Pj = mail + (size_t)((j - lo_c) * 2 + ((j == w_lo && locut) ? 1 : 0)) * kPartialFloats;
+            merge4(m, l, acc, Pj[0], Pj[1], reinterpret_cast<const float4*>(Pj + 4)[lane]);
+          }
+          if (w_lo >= lo_c && w_hi <= hi_c) {              // the whole head lies inside this CTA
+            write_out4(p.out + ((size_t)cons.seq * v.H + cons.head) * kHeadDim, l, acc, lane);
+          } else {                                         // hand the CTA's partial to the finisher
+            const int slot = w_lo < lo_c ? 0 : 1;
+            float* C = mail + (size_t)(2 * kWarps + slot) * kPartialFloats;
+            if (lane == 0) {
+              C[0] = m;
+              C[1] = l;
+            }
+            reinterpret_cast<float4*>(C + 4)[lane] = acc;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(cta_bar0 + 8 * slot);   // releases the writes above
+          }
+        }
       }
       begin = true;
     }
