@@ -55,7 +55,8 @@ enum ssd_status {
   SSD_ERR_BAD_STATE = -2,   /* call order violated (e.g. compress before labels exist) */
   SSD_ERR_OVERFLOW = -3,    /* append beyond max_image_tokens (cf. Algorithm 2, buffer overflow) */
   SSD_ERR_NO_MEM = -4,      /* caller's device buffer too small for the layout */
-  SSD_ERR_CUDA = -5         /* a CUDA runtime call or launch failed */
+  SSD_ERR_CUDA = -5,        /* a CUDA runtime call or launch failed */
+  SSD_ERR_LIMIT = -6        /* a size exceeds a fixed limit of the entry point called */
 };
 
 /* Human-readable name of a status code (static storage; never NULL). */
@@ -123,6 +124,26 @@ int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v
  *   q, out [n_seqs, n_heads, head_dim], 16-byte aligned
  * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
 int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
+
+/* ssd_decode_attn for callers that cannot allocate.  The paper has no counterpart; this is a
+ * packaging variant of the same kernel.  ssd_decode_attn keeps the kernel's scratch (partial sums of
+ * heads that two thread blocks share, and per-head arrival counters) inside the buffer given to
+ * ssd_cache_create.  Some callers have no memory to give beyond their tensors and cannot call
+ * cudaMalloc where they stand: code running between the capture calls of a stream, plugins inside a
+ * host program that owns all device memory through its own pool, or real-time loops in which an
+ * allocation's implicit synchronisation is not acceptable.  For them the same scratch is a fixed
+ * array inside the library image (about 0.4 MB, held by every GPU that loads the library until the
+ * process ends), and this call allocates nothing, on the device or through any library.
+ *   Same arguments, results and errors as ssd_decode_attn (outputs are bit-identical), plus
+ *   SSD_ERR_LIMIT if n_seqs * n_heads > 32768 or the GPU has more than 256 SMs: the array is sized
+ *   for those maxima.
+ * The first call on each device looks up the array's device address (a synchronous runtime query);
+ * make that first call before any stream capture begins.  All calls on a device share the one
+ * array, whatever cache they pass: two calls whose kernels overlap on the GPU (different streams)
+ * race on it; calls on one stream are safe.  The counters are cleared on `stream` at every call,
+ * the partials are always written before they are read.  Bounded-wait failures are reported in the
+ * cache's status word like those of ssd_decode_attn. */
+int ssd_decode_attn_static(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
 /* One decode step of one layer from HOST buffers (pinned memory recommended): copies q, k_new and
  * v_new to the device, appends, attends, and copies the output back, all enqueued on `stream`.

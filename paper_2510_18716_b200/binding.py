@@ -21,6 +21,7 @@ SSD_ERR_BAD_STATE = -2
 SSD_ERR_OVERFLOW = -3
 SSD_ERR_NO_MEM = -4
 SSD_ERR_CUDA = -5
+SSD_ERR_LIMIT = -6
 
 EXPORTS = [
     "ssd_status_string", "ssd_cache_required_bytes", "ssd_cache_create", "ssd_cache_free",
@@ -28,7 +29,7 @@ EXPORTS = [
     "ssd_decode_attn", "ssd_step_host", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
-    "ssd_cache_device_status", "ssd_debug_decode_plan",
+    "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
 ]
 
 
@@ -74,6 +75,7 @@ def load():
     L.ssd_compress.argtypes = [vp, i32, vp, vp, vp, i32, i32, vp]
     L.ssd_append.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_decode_attn.argtypes = [vp, i32, vp, vp, vp]
+    L.ssd_decode_attn_static.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
     L.ssd_cache_max_slots.argtypes = [vp]
@@ -222,6 +224,17 @@ class SsdCache:
             out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
         self._check(self.lib.ssd_decode_attn(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"), _stream()),
                     "ssd_decode_attn")
+        return out
+
+    def decode_attn_static(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """decode_attn with the kernel's scratch in the library's built-in array (allocates nothing
+        inside the library; `out` should be passed by callers that must not allocate at all)."""
+        c = self.cfg
+        shp = (c.n_seqs, c.n_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
+        self._check(self.lib.ssd_decode_attn_static(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"),
+                                                    _stream()), "ssd_decode_attn_static")
         return out
 
     def step_host(self, layer: int, q_host, k_new_host, v_new_host, out_host):

@@ -122,6 +122,7 @@ const char* ssd_status_string(int s) {
     case SSD_ERR_OVERFLOW: return "SSD_ERR_OVERFLOW";
     case SSD_ERR_NO_MEM: return "SSD_ERR_NO_MEM";
     case SSD_ERR_CUDA: return "SSD_ERR_CUDA";
+    case SSD_ERR_LIMIT: return "SSD_ERR_LIMIT";
     default: return "SSD_ERR_UNKNOWN";
   }
 }
@@ -574,3 +575,72 @@ int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot hand the library any scratch memory of their own.
+// The cross-block partials and the per-head arrival counters of the decode kernel live in this
+// array, which is part of the library image: every GPU that loads the library carries it until
+// the process exits.  Layout: [kStaticCtas * 2 partials of kPartialFloats floats | kStaticPairs
+// counters].
+namespace {
+constexpr int kStaticCtas = 256;       // thread blocks (one per SM) the partial area has room for
+constexpr int kStaticPairs = 32768;    // (sequence, head) pairs the counter area has room for
+constexpr size_t kStaticPartialBytes = (size_t)kStaticCtas * 2 * ssd::kPartialFloats * 4;
+constexpr size_t kStaticBytes = kStaticPartialBytes + (size_t)kStaticPairs * 4;
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q, void* out, void* stream) {
+  if (!c || !q || !out) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
+  const long pairs = (long)g.n_seqs * g.n_heads;
+  if (pairs > kStaticPairs) return SSD_ERR_LIMIT;
+
+  // Once per device, with that device current: the array's name is only a host-side handle here,
+  // so ask the runtime where the array lives on this device.
+  static unsigned char* dev_ptr[64] = {};
+  static int dev_sms[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  if (!dev_ptr[dev]) {
+    void* ptr = nullptr;
+    int sms = 0;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError();
+      return SSD_ERR_CUDA;
+    }
+    dev_sms[dev] = sms;
+    dev_ptr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  if (dev_sms[dev] > kStaticCtas) return SSD_ERR_LIMIT;   // the kernel runs one thread block per SM
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* base = dev_ptr[dev];
+  // The array keeps what the previous call left.  Partials are written before they are read, but
+  // the arrival counters must start at zero, which a call that was cut short would not guarantee.
+  if (cudaMemsetAsync(base + kStaticPartialBytes, 0, (size_t)pairs * 4, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  DecodeParams p;
+  p.slab = c->d_slab(layer);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.partial = reinterpret_cast<float*>(base);
+  p.counters = reinterpret_cast<uint32_t*>(base + kStaticPartialBytes);
+  p.status = c->d_status();
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.split = Split{0, 0, 0, 0, 0.f};
+  c->fill_view(layer, p.view);
+  if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  return SSD_OK;
+}

@@ -45,7 +45,7 @@ def test_status_strings():
     assert B.status_string(0) == "SSD_OK"
     codes = {B.SSD_ERR_INVALID_ARG: "SSD_ERR_INVALID_ARG", B.SSD_ERR_BAD_STATE: "SSD_ERR_BAD_STATE",
              B.SSD_ERR_OVERFLOW: "SSD_ERR_OVERFLOW", B.SSD_ERR_NO_MEM: "SSD_ERR_NO_MEM",
-             B.SSD_ERR_CUDA: "SSD_ERR_CUDA"}
+             B.SSD_ERR_CUDA: "SSD_ERR_CUDA", B.SSD_ERR_LIMIT: "SSD_ERR_LIMIT"}
     for c, s in codes.items():
         assert B.status_string(c) == s
     assert B.status_string(-99) == "SSD_ERR_UNKNOWN"
