@@ -295,7 +295,7 @@ def run_ours(args, cfg):
     peak, peak_kind = measured_peaks()
     dec_mean_ms = float(np.mean(dec_ms)) if len(dec_ms) else float("nan")
     achieved = bytes_launch / (dec_mean_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "ssd_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                 "bytes_per_launch": bytes_launch, "launch_ms_mean": dec_mean_ms,
                 "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,

@@ -90,7 +90,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // ----------------------------------------------------------------------------- score
 // One CTA per (sequence, semantic head); loops over blocks of 32 observed queries, two passes
 // over the key tiles per block (row max / row sum, then normalised column sums).
-__global__ void __launch_bounds__(kThreads) score_kernel(const ScoreParams p) {
+__global__ void __launch_bounds__(kThreads) ssd_score_kernel(const ScoreParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
   float* s_part = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));  // [8][kBK]
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const ScoreParams p) {
 // One CTA per (sequence, semantic head): radix-select the k-th largest score (scores are
 // non-negative floats, so their bit patterns order like unsigned integers), then emit, in
 // ascending index order, every candidate above it and the lowest-index candidates equal to it.
-__global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p) {
+__global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams p) {
   __shared__ uint32_t s_hist[256];
   __shared__ uint32_t s_prefix, s_need;
   __shared__ uint32_t s_gt[kThreads + 1], s_eq[kThreads + 1];
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const SelectParams p) 
 
 // ----------------------------------------------------------------------------- gather
 // One warp per destination slot: lanes 0-15 copy the K row, lanes 16-31 the V row.
-__global__ void __launch_bounds__(kThreads) gather_kernel(const GatherParams p, int max_slots) {
+__global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams p, int max_slots) {
   const int pair = blockIdx.x;
   const int seq = pair / p.H, head = pair - seq * p.H;
   const HeadDesc d = p.desc[head];
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kThreads) gather_kernel(const GatherParams p, 
 // ----------------------------------------------------------------------------- classify
 // One CTA per (unit, block of 32 image steps), unit = (layer, calibration sequence, head).
 // Only visual columns are touched: the prompt's share of the softmax cancels in the ratio.
-__global__ void __launch_bounds__(kThreads) classify_kernel(const ClassifyParams p, int n_row_blocks) {
+__global__ void __launch_bounds__(kThreads) ssd_classify_kernel(const ClassifyParams p, int n_row_blocks) {
   __shared__ TileSmem sm;
   __shared__ float s_ratio[kBR];
   const int unit = blockIdx.x / n_row_blocks, rb = blockIdx.x - unit * n_row_blocks;
@@ -358,28 +358,28 @@ int classify_rows_per_block() { return kBR; }
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
   size_t smem = sizeof(TileSmem) + (8 * kBK + (size_t)p.n0) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  score_kernel<<<p.n_seqs * p.H, kThreads, smem, st>>>(p);
+  ssd_score_kernel<<<p.n_seqs * p.H, kThreads, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
-  select_kernel<<<p.n_seqs * p.H, kThreads, 0, st>>>(p);
+  ssd_select_kernel<<<p.n_seqs * p.H, kThreads, 0, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st) {
   dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
-  gather_kernel<<<grid, kThreads, 0, st>>>(p, max_slots);
+  ssd_gather_kernel<<<grid, kThreads, 0, st>>>(p, max_slots);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st) {
-  classify_kernel<<<p.n_units * n_row_blocks, kThreads, 0, st>>>(p, n_row_blocks);
+  ssd_classify_kernel<<<p.n_units * n_row_blocks, kThreads, 0, st>>>(p, n_row_blocks);
   count_launch();
   return cudaGetLastError();
 }

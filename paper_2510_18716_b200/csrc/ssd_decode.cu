@@ -364,7 +364,7 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeParams p) {
+__global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_constant__ DecodeParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const LayerView& v = p.view;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -562,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   }
 }
 
-__global__ void __launch_bounds__(256) append_kernel(const AppendParams p) {
+__global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= p.n_seqs * p.H) return;
   const int seq = warp / p.H, head = warp - seq * p.H;
@@ -597,7 +597,7 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   const bool cached = dev >= 0 && dev < 64;
   if (!cached || !smem_set[dev]) {
-    e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(ssd_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (cached) {
       smem_set[dev] = true;
@@ -610,7 +610,7 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
   const long w = plan_workers(total, cached ? max_workers[dev] : decode_max_workers());
   p.split = make_split(total, w);
   const int grid = (int)((w + kWarps - 1) / kWarps);
-  decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
+  ssd_decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
@@ -618,7 +618,7 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st) {
   int warps = p.n_seqs * p.H;
   int grid = (warps * 32 + 255) / 256;
-  append_kernel<<<grid, 256, 0, st>>>(p);
+  ssd_append_kernel<<<grid, 256, 0, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
