@@ -28,6 +28,24 @@ sys.path.insert(0, ROOT)
 
 from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 
+# DRAM bytes (read + written) of one ssd_decode_kernel launch on a janus7b layer, from the ncu capture
+# summarised in profiles/ssd_decode_kernel_janus7b_layer.md.  Reported only while the kernel's sources
+# still hash to what was captured; otherwise `traffic` is null until the counters are taken again.
+DECODE_TRAFFIC = {"workload": "janus7b", "bytes_per_launch": 163.49e6,
+                  "sha256": "8e018c0810d913ebbb3f2c4d09481ae8ca11e13c0a0d838391682991d0fbd7c0"}
+
+
+def decode_traffic(cfg):
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("ssd_decode.cu", "ssd_plan.h", "ssd_internal.cuh"):
+        with open(os.path.join(ROOT, "paper_2510_18716_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    if h.hexdigest() != DECODE_TRAFFIC["sha256"] or not cfg.name.startswith(DECODE_TRAFFIC["workload"]):
+        return None
+    return DECODE_TRAFFIC["bytes_per_launch"]
+
+
 METRIC = "decoded image tokens/sec (attention+cache ops)"
 UNIT = "image tokens/s"
 
@@ -296,7 +314,7 @@ def run_ours(args, cfg):
     dec_mean_ms = float(np.mean(dec_ms)) if len(dec_ms) else float("nan")
     achieved = bytes_launch / (dec_mean_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "ssd_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": decode_traffic(cfg),
                 "bytes_per_launch": bytes_launch, "launch_ms_mean": dec_mean_ms,
                 "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
                 "launches_timed": int(len(dec_ms)), "frac_of_8TBs_nominal": achieved / 8000.0,
