@@ -124,6 +124,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                : "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start while its predecessor in the stream is still running, once the predecessor has allowed
+// it; it must then wait for the predecessor to complete before touching memory.  Both kernels of
+// the decode step allow their successor at once and wait just before their first global access,
+// so launch latency and the index planning overlap with the predecessor's tail.  Every kernel of
+// the chain waits for its predecessor's completion, so stream order is preserved transitively.
+__device__ __forceinline__ void pdl_allow_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ------------------------------------------------------------------ arithmetic
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -332,6 +341,7 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   }
   unsigned heads = __ballot_sync(FULL, r_pair >= 0);
   if (!heads) return;
+  pdl_wait_predecessor();                // the scratch below may still be in use by the previous launch
   for (unsigned h = heads; h; h &= h - 1) {
     const int slot = __ffs(h) - 1;       // 0: began in an earlier CTA, 1: begins here and runs on
     if (!mbar_wait(cta_bar0 + 8 * slot, 0)) {
@@ -369,6 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   const LayerView& v = p.view;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = lane >> 3, l8 = lane & 7;
+  pdl_allow_successor();
 
   const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
   const uint32_t cta_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
@@ -452,6 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     ++ahead;
   };
 
+  pdl_wait_predecessor();                // everything above read only the launch parameters
 #pragma unroll 1
   for (int s = 0; s < kStages && prod.g < prod.g_end; ++s) issue(s);
 
@@ -564,6 +576,8 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
 
 __global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  pdl_allow_successor();
+  pdl_wait_predecessor();
   if (warp >= p.n_seqs * p.H) return;
   const int seq = warp / p.H, head = warp - seq * p.H;
   const HeadDesc d = p.desc[head];
@@ -610,17 +624,37 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
   const long w = plan_workers(total, cached ? max_workers[dev] : decode_max_workers());
   p.split = make_split(total, w);
   const int grid = (int)((w + kWarps - 1) / kWarps);
-  ssd_decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, ssd_decode_kernel, p);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st) {
   int warps = p.n_seqs * p.H;
   int grid = (warps * 32 + 255) / 256;
-  ssd_append_kernel<<<grid, 256, 0, st>>>(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, ssd_append_kernel, p);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace ssd
