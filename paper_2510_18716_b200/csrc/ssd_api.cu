@@ -267,6 +267,7 @@ int ssd_classify_partial(ssd_cache* c, const void* q_cal, const void* k_cal, int
   p.q_cal = static_cast<const __nv_bfloat16*>(q_cal);
   p.k_cal = static_cast<const __nv_bfloat16*>(k_cal);
   p.ratio_part = c->d_score();
+  p.status = c->d_status();
   p.n_units = (int)units;
   p.L = g.prompt_len;
   p.N = n_img;

@@ -2,7 +2,6 @@
 //   score  : score[j] = sum over observed image steps t of softmax(q_t K^T)[L + j]   (causal)
 //   select : top-M of score over candidates [0, n0 - R), ties to the lowest index, ascending
 //   gather : copy prompt rows, selected rows and the newest ring rows into the slab
-// and the head classification pass (Sec. 3.3 sparsity metric), which shares the logit tile code.
 //
 // This file holds the CUDA-core (fp32 FMA) form of the QK^T tiles: every product of two bf16
 // values is exact in fp32 and sums are taken in a fixed order, so scores are reproducible bit
@@ -293,68 +292,7 @@ __global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams
   }
 }
 
-// ----------------------------------------------------------------------------- classify
-// One CTA per (unit, block of 32 image steps), unit = (layer, calibration sequence, head).
-// Only visual columns are touched: the prompt's share of the softmax cancels in the ratio.
-__global__ void __launch_bounds__(kThreads) ssd_classify_kernel(const ClassifyParams p, int n_row_blocks) {
-  __shared__ TileSmem sm;
-  __shared__ float s_ratio[kBR];
-  const int unit = blockIdx.x / n_row_blocks, rb = blockIdx.x - unit * n_row_blocks;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const __nv_bfloat16* Q = p.q_cal + (size_t)unit * p.N * kHeadDim;
-  const __nv_bfloat16* K = p.k_cal + ((size_t)unit * (p.L + p.N) + p.L) * kHeadDim;  // visual keys
-  const int r0 = rb * kBR;
-  load_q_tile(sm, Q, r0, p.N, p.scale_log2);
-  const int rows_here = min(kBR, p.N - r0);
-  const int vis_max = r0 + rows_here;   // the block's last row (step t = r0+rows_here) sees t visual keys
-  int t_r[4];
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    int row = r0 + warp * 4 + r;
-    t_r[r] = row < p.N ? row + 1 : 0;   // image step of the row; visual keys [0, t) visible
-  }
-  float m[4], far[4], all[4];
-#pragma unroll
-  for (int r = 0; r < 4; ++r) { m[r] = kNegBig; far[r] = 0.f; all[r] = 0.f; }
-  for (int k0 = 0; k0 < vis_max; k0 += kBK) {
-    __syncthreads();
-    load_k_tile(sm, K, k0, p.N);
-    __syncthreads();
-    float x[4][2];
-    tile_logits(sm, warp, lane, x);
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        int i = k0 + lane + 32 * c;     // visual token index
-        if (i < t_r[r]) {
-          float mn = fmaxf(m[r], x[r][c]);
-          float cr = ex2(m[r] - mn), e = ex2(x[r][c] - mn);
-          all[r] = all[r] * cr + e;
-          far[r] = far[r] * cr + (i <= t_r[r] - 1 - p.w ? e : 0.f);
-          m[r] = mn;
-        }
-      }
-    }
-  }
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    float mw = warp_max(m[r]);
-    float c = ex2(m[r] - mw);
-    float a = warp_sum(all[r] * c), f = warp_sum(far[r] * c);
-    if (lane == 0) s_ratio[warp * 4 + r] = (t_r[r] > 0 && a > 0.f) ? f / a : 0.f;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    float tot = 0.f;
-    for (int r = 0; r < kBR; ++r) tot += s_ratio[r];
-    p.ratio_part[(size_t)unit * n_row_blocks + rb] = tot;
-  }
-}
-
 }  // namespace
-
-int classify_rows_per_block() { return kBR; }
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
   size_t smem = sizeof(TileSmem) + (8 * kBK + (size_t)p.n0) * sizeof(float);
@@ -374,12 +312,6 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st) {
   dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
   ssd_gather_kernel<<<grid, kThreads, 0, st>>>(p, max_slots);
-  count_launch();
-  return cudaGetLastError();
-}
-
-cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st) {
-  ssd_classify_kernel<<<p.n_units * n_row_blocks, kThreads, 0, st>>>(p, n_row_blocks);
   count_launch();
   return cudaGetLastError();
 }

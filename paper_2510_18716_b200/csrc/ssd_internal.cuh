@@ -78,6 +78,7 @@ struct ClassifyParams {
   const __nv_bfloat16* q_cal;  // [n_units, N, 128], unit = (layer, p, head)
   const __nv_bfloat16* k_cal;  // [n_units, L + N, 128]
   float* ratio_part;           // [n_units, n_row_blocks]
+  uint32_t* status;            // device status word (bit 1: a bounded wait of the classifier ran out)
   int n_units, L, N, w;
   float scale_log2;
 };
