@@ -332,6 +332,7 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
       sp.k_full = static_cast<const __nv_bfloat16*>(k_full);
       sp.desc = desc;
       sp.score = c->d_score();
+      sp.status = c->d_status();
       sp.n_seqs = g.n_seqs; sp.H = g.n_heads; sp.L = g.prompt_len; sp.n0 = n0; sp.n_obs = n_obs;
       sp.scale_log2 = c->scale * 1.4426950408889634f;
       if (launch_score(sp, st) != cudaSuccess) return SSD_ERR_CUDA;

@@ -1,11 +1,8 @@
-// One-time compression of a layer (Algorithm 1, semantic branch; Algorithm 2's prefill split):
-//   score  : score[j] = sum over observed image steps t of softmax(q_t K^T)[L + j]   (causal)
+// One-time compression of a layer (Algorithm 1, semantic branch; Algorithm 2's prefill split),
+// the parts that are not a contraction:
 //   select : top-M of score over candidates [0, n0 - R), ties to the lowest index, ascending
 //   gather : copy prompt rows, selected rows and the newest ring rows into the slab
-//
-// This file holds the CUDA-core (fp32 FMA) form of the QK^T tiles: every product of two bf16
-// values is exact in fp32 and sums are taken in a fixed order, so scores are reproducible bit
-// for bit from run to run, which the selection relies on.
+// The scores themselves (QK^T, softmax, column sums) come from the tensor-core kernel.
 #include "ssd_internal.cuh"
 
 namespace ssd {
@@ -13,175 +10,6 @@ namespace ssd {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBR = 32;        // query rows per block (4 per warp)
-constexpr int kBK = 64;        // keys per tile (2 per lane)
-constexpr int kKStride = 65;   // padded row stride of the key tile in 32-bit words
-constexpr float kNegBig = -1.0e30f;
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float lo_f(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float hi_f(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-struct TileSmem {
-  uint32_t k[kBK * kKStride];   // key tile, bf16 pairs
-  float2 q[kBR * 64];           // query rows, pre-scaled by scale*log2(e)
-};
-
-// rows [r0, r0 + kBR) of Q (n_rows total) -> smem, scaled
-__device__ __forceinline__ void load_q_tile(TileSmem& sm, const __nv_bfloat16* Q, int r0, int n_rows,
-                                            float scale_log2) {
-  const uint32_t* Qw = reinterpret_cast<const uint32_t*>(Q);
-  for (int i = threadIdx.x; i < kBR * 64; i += kThreads) {
-    int r = i >> 6, dw = i & 63;
-    uint32_t w = (r0 + r < n_rows) ? Qw[(size_t)(r0 + r) * 64 + dw] : 0u;
-    sm.q[i] = make_float2(lo_f(w) * scale_log2, hi_f(w) * scale_log2);
-  }
-}
-
-// keys [k0, k0 + kBK) of K (n_keys total) -> smem (zero beyond n_keys)
-__device__ __forceinline__ void load_k_tile(TileSmem& sm, const __nv_bfloat16* K, int k0, int n_keys) {
-  const uint4* K4 = reinterpret_cast<const uint4*>(K);
-  for (int i = threadIdx.x; i < kBK * 16; i += kThreads) {
-    int key = i >> 4, c = i & 15;
-    uint4 v = (k0 + key < n_keys) ? K4[(size_t)(k0 + key) * 16 + c] : make_uint4(0, 0, 0, 0);
-    uint32_t* d = sm.k + key * kKStride + c * 4;
-    d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
-  }
-}
-
-// logits (base-2 units) of this warp's 4 rows against keys `lane` and `lane + 32` of the tile
-__device__ __forceinline__ void tile_logits(const TileSmem& sm, int warp, int lane, float (&x)[4][2]) {
-#pragma unroll
-  for (int r = 0; r < 4; ++r) x[r][0] = x[r][1] = 0.f;
-  const uint32_t* ka = sm.k + lane * kKStride;
-  const uint32_t* kb = sm.k + (lane + 32) * kKStride;
-  const float2* qr = sm.q + warp * 4 * 64;
-#pragma unroll 8
-  for (int dw = 0; dw < 64; ++dw) {
-    uint32_t a = ka[dw], b = kb[dw];
-    float al = lo_f(a), ah = hi_f(a), bl = lo_f(b), bh = hi_f(b);
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      float2 qv = qr[r * 64 + dw];
-      x[r][0] = fmaf(al, qv.x, x[r][0]);
-      x[r][0] = fmaf(ah, qv.y, x[r][0]);
-      x[r][1] = fmaf(bl, qv.x, x[r][1]);
-      x[r][1] = fmaf(bh, qv.y, x[r][1]);
-    }
-  }
-}
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// ----------------------------------------------------------------------------- score
-// One CTA per (sequence, semantic head); loops over blocks of 32 observed queries, two passes
-// over the key tiles per block (row max / row sum, then normalised column sums).
-__global__ void __launch_bounds__(kThreads) ssd_score_kernel(const ScoreParams p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
-  float* s_part = reinterpret_cast<float*>(smem_raw + sizeof(TileSmem));  // [8][kBK]
-  float* s_score = s_part + 8 * kBK;                                      // [n0]
-
-  const int pair = blockIdx.x;
-  const int head = pair % p.H;
-  if (!p.desc[head].w) return;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int ctx_all = p.L + p.n0;
-  const __nv_bfloat16* Q = p.q_obs + (size_t)pair * p.n_obs * kHeadDim;
-  const __nv_bfloat16* K = p.k_full + (size_t)pair * ctx_all * kHeadDim;
-
-  for (int j = tid; j < p.n0; j += kThreads) s_score[j] = 0.f;
-  __syncthreads();
-
-  const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
-  for (int r0 = 0; r0 < p.n_obs; r0 += kBR) {
-    load_q_tile(sm, Q, r0, p.n_obs, p.scale_log2);
-    const int rows_here = min(kBR, p.n_obs - r0);
-    const int ctx_max = p.L + t_first + r0 + rows_here - 1;  // context of the block's last row
-    int ctx_r[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      int row = r0 + warp * 4 + r;
-      ctx_r[r] = row < p.n_obs ? p.L + t_first + row : 0;    // keys [0, ctx_r) are visible
-    }
-    float m[4], s[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) { m[r] = kNegBig; s[r] = 0.f; }
-
-    // pass 1: row max and row sum
-    for (int k0 = 0; k0 < ctx_max; k0 += kBK) {
-      __syncthreads();
-      load_k_tile(sm, K, k0, ctx_all);
-      __syncthreads();
-      float x[4][2];
-      tile_logits(sm, warp, lane, x);
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          int key = k0 + lane + 32 * c;
-          if (key < ctx_r[r]) {
-            float mn = fmaxf(m[r], x[r][c]);
-            s[r] = s[r] * ex2(m[r] - mn) + ex2(x[r][c] - mn);
-            m[r] = mn;
-          }
-        }
-      }
-    }
-    float inv[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      float mw = warp_max(m[r]);
-      float sw = warp_sum(s[r] * ex2(m[r] - mw));
-      m[r] = mw;
-      inv[r] = sw > 0.f ? 1.f / sw : 0.f;
-    }
-
-    // pass 2: normalised probabilities, column sums over the block's rows in a fixed order
-    for (int k0 = 0; k0 < ctx_max; k0 += kBK) {
-      __syncthreads();
-      load_k_tile(sm, K, k0, ctx_all);
-      __syncthreads();
-      float x[4][2];
-      tile_logits(sm, warp, lane, x);
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        int key = k0 + lane + 32 * c;
-        float col = 0.f;
-#pragma unroll
-        for (int r = 0; r < 4; ++r)
-          if (key < ctx_r[r]) col += ex2(x[r][c] - m[r]) * inv[r];
-        s_part[warp * kBK + lane + 32 * c] = col;
-      }
-      __syncthreads();
-      if (tid < kBK) {
-        int key = k0 + tid;
-        if (key >= p.L && key < ctx_max) {
-          float tot = 0.f;
-#pragma unroll
-          for (int w = 0; w < 8; ++w) tot += s_part[w * kBK + tid];
-          s_score[key - p.L] += tot;
-        }
-      }
-    }
-    __syncthreads();
-  }
-  float* out = p.score + (size_t)pair * p.n0;
-  for (int j = tid; j < p.n0; j += kThreads) out[j] = s_score[j];
-}
 
 // ----------------------------------------------------------------------------- select
 // One CTA per (sequence, semantic head): radix-select the k-th largest score (scores are
@@ -293,15 +121,6 @@ __global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams
 }
 
 }  // namespace
-
-cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
-  size_t smem = sizeof(TileSmem) + (8 * kBK + (size_t)p.n0) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  ssd_score_kernel<<<p.n_seqs * p.H, kThreads, smem, st>>>(p);
-  count_launch();
-  return cudaGetLastError();
-}
 
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
   ssd_select_kernel<<<p.n_seqs * p.H, kThreads, 0, st>>>(p);

@@ -63,6 +63,7 @@ struct ScoreParams {
   const __nv_bfloat16* k_full; // [n_seqs, H, L + n0, 128]
   const HeadDesc* desc;
   float* score;                // [n_seqs, H, n0]
+  uint32_t* status;            // device status word (bit 2: a bounded wait of the scoring ran out)
   int n_seqs, H, L, n0, n_obs;
   float scale_log2;
 };

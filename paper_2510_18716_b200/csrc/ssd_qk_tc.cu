@@ -7,6 +7,12 @@
 // Used by the head classifier (Sec. 3.3 sparsity metric): per image step t, the attention mass on
 // visual tokens older than the newest w, over the mass on all visual tokens so far.  Only visual
 // columns are touched: the prompt's share of the softmax cancels in the ratio.
+// Used by the sink scoring of ssd_compress (Algorithm 1, AttentionScores and running sum): per
+// block of 128 observed queries, a first sweep over the key tiles gives every row its maximum and
+// exp-sum, a second sweep recomputes the tiles, normalises, and adds the columns up.  The sum over
+// the 32 rows of a warp is a shuffle transpose-reduction; each warp keeps its own score array in
+// shared memory and the four are added in a fixed order at the end, so scores are bitwise
+// reproducible from run to run, which the selection relies on.
 //
 // Operand tiles sit in shared memory in the K-major layout without swizzling: 8 rows x 16 bytes
 // form a contiguous 128-byte core matrix, core matrices follow each other along the head
@@ -248,6 +254,137 @@ __global__ void __launch_bounds__(kRows) ssd_classify_kernel(const ClassifyParam
   }
 }
 
+// ----------------------------------------------------------------------------- score
+// Sum over the 32 lanes of a warp of 32 values each: lane j returns the total of value j.
+__device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) {
+    const bool up = (lane & s) != 0;
+#pragma unroll
+    for (int i = 0; i < s; ++i) {
+      const float keep = up ? a[i + s] : a[i];
+      const float send = up ? a[i] : a[i + s];
+      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+    }
+  }
+  return a[0];
+}
+
+// One CTA per (sequence, semantic head); loops over blocks of 128 observed queries.
+__global__ void __launch_bounds__(kRows) ssd_score_kernel(const ScoreParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ uint64_t s_bar;
+  __shared__ uint32_t s_tmem;
+  const int pair = blockIdx.x;
+  const int head = pair % p.H;
+  if (!p.desc[head].w) return;            // before any tensor-memory allocation
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ctx_all = p.L + p.n0;
+  const __nv_bfloat16* Q = p.q_obs + (size_t)pair * p.n_obs * kHeadDim;
+  const __nv_bfloat16* K = p.k_full + (size_t)pair * ctx_all * kHeadDim;
+  const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
+
+  const uint32_t q_s = smem_u32(smem), k_s = q_s + kTileBytes;
+  float* s_score = reinterpret_cast<float*>(smem + 2 * kTileBytes);   // [4 warps][n0]
+  const uint32_t bar = smem_u32(&s_bar);
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kKeys)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (tid == 0) {
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int j = tid; j < 4 * p.n0; j += kRows) s_score[j] = 0.f;
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  const uint32_t my_tmem = tmem + ((uint32_t)(warp * 32) << 16);
+  float* my_score = s_score + (size_t)warp * p.n0;
+
+  uint32_t parity = 0;
+  bool ok = true;
+  // S tile of keys [k0, k0 + 128) for the current query block; false if the wait ran out
+  auto logits_tile = [&](int k0) -> bool {
+    load_tile(k_s, K, k0, ctx_all, warp, lane, 4);
+    tiles_ready_for_mma();
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      mma_tile(tmem, q_s, k_s, bar);
+    }
+    const bool done = mbar_wait(bar, parity);
+    parity ^= 1u;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    return __all_sync(0xffffffffu, done);
+  };
+  // everyone is done with the key tile and the accumulator; a CTA-wide verdict on the wait
+  auto tile_done = [&](bool fine) -> bool {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    return __syncthreads_and(fine ? 1 : 0) != 0;
+  };
+
+  for (int r0 = 0; r0 < p.n_obs && ok; r0 += kRows) {
+    load_tile(q_s, Q, r0, p.n_obs, warp, lane, 4);
+    const int row = r0 + tid;
+    const int ctx_r = row < p.n_obs ? p.L + t_first + row : 0;        // keys [0, ctx_r) are visible
+    const int last = min(r0 + kRows, p.n_obs) - 1;
+    const int ctx_max = p.L + t_first + last;                        // context of the block's last row
+    const int warp_ctx = p.L + t_first + min(r0 + warp * 32 + 31, last);
+
+    // sweep 1: row maximum and exp-sum
+    RowStats st = {kNegBig, 0.f, 0.f};
+    for (int k0 = 0; k0 < ctx_max && ok; k0 += kKeys) {
+      const bool fine = logits_tile(k0);
+      if (fine) {
+#pragma unroll 1
+        for (int cb = 0; cb < kKeys / 32; ++cb) {
+          const int base = k0 + cb * 32;
+          if (base >= warp_ctx) break;
+          float v[32];
+          tmem_ld32(my_tmem + cb * 32, v);
+          fold32(st, v, base, ctx_r - 1, 0, p.scale_log2);
+        }
+      }
+      ok = tile_done(fine);
+    }
+    const float inv = st.all > 0.f ? 1.f / st.all : 0.f;
+
+    // sweep 2: normalised probabilities, column sums over the block's rows
+    for (int k0 = (p.L / kKeys) * kKeys; k0 < ctx_max && ok; k0 += kKeys) {
+      const bool fine = logits_tile(k0);
+      if (fine) {
+#pragma unroll 1
+        for (int cb = 0; cb < kKeys / 32; ++cb) {
+          const int base = k0 + cb * 32;
+          if (base >= warp_ctx) break;
+          if (base + 32 <= p.L) continue;                 // prompt keys only: not scored
+          float v[32];
+          tmem_ld32(my_tmem + cb * 32, v);
+          const int nv = min(max(ctx_r - base, 0), 32);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv : 0.f;
+          const float col = warp_column_sums(v, lane);
+          const int key = base + lane;
+          if (key >= p.L && key < ctx_max) my_score[key - p.L] += col;
+        }
+      }
+      ok = tile_done(fine);
+    }
+  }
+
+  __syncthreads();
+  float* out = p.score + (size_t)pair * p.n0;
+  for (int j = tid; j < p.n0; j += kRows)
+    out[j] = ok ? (s_score[j] + s_score[p.n0 + j]) + (s_score[2 * p.n0 + j] + s_score[3 * p.n0 + j]) : 0.f;
+  if (tid == 0 && !ok) atomicOr(p.status, 4u);
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kKeys) : "memory");
+  }
+}
+
 }  // namespace
 
 int classify_rows_per_block() { return kRows; }
@@ -257,6 +394,16 @@ cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStrea
   cudaError_t e = cudaFuncSetAttribute(ssd_classify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   ssd_classify_kernel<<<p.n_units * n_row_blocks, kRows, smem, st>>>(p, n_row_blocks);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
+  const size_t smem = 2 * (size_t)kTileBytes + 4 * (size_t)p.n0 * sizeof(float) + 1024;
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  ssd_score_kernel<<<p.n_seqs * p.H, kRows, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
