@@ -79,7 +79,7 @@ class RunResult:
 
 
 def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, full_every_step=False,
-                 n_obs=None, check_planted=False, device="cuda:0") -> RunResult:
+                 n_obs=None, check_planted=False, device="cuda:0", labels_override=None) -> RunResult:
     """Drive the C-ABI path for `layers` x `seqs` of a workload and check every stage.
 
     The cache is created with len(layers) layers and len(seqs) sequences; layer i of the cache holds
@@ -103,7 +103,7 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
         assert np.array_equal(cache.get_labels(), lab_gpu)
         del qc, kc
     else:
-        labels = gen_masks
+        labels = gen_masks if labels_override is None else np.asarray(labels_override, np.uint8).reshape(gen_masks.shape)
         cache.set_head_labels(labels)
 
     errs = []

@@ -193,3 +193,22 @@ def test_argument_errors_launch_nothing():
     cache.close()
     bad = B.make_config(1, 1, 1, 0, 4, 1, 1, 1, head_dim=64)
     assert B.required_bytes(bad) == 0
+
+
+@pytest.mark.parametrize("kind", ["all_spatial", "all_semantic", "random"])
+def test_other_head_partitions(kind):
+    """The paper's ablation assigns heads at random with the same policies (Sec. 4.4); all-spatial is a
+    sliding-window cache for every head and all-semantic a heavy-hitter cache for every head.  The
+    policies do not depend on what the heads' data look like, so parity must hold for any labelling."""
+    for name, layers, seqs in (("tiny", [0], [0]), ("janus1b", [5], [0, 1, 2])):
+        cfg = wl.CONFIGS[name]
+        H = cfg.n_heads
+        if kind == "all_spatial":
+            lab = np.zeros((len(layers), H), np.uint8)
+        elif kind == "all_semantic":
+            lab = np.ones((len(layers), H), np.uint8)
+        else:
+            rng = np.random.default_rng(123)
+            lab = np.stack([rng.permutation(wl.sink_mask(cfg, l)) for l in layers])
+        r = run_workload(cfg, layers, seqs, (cfg.n0 + 1, cfg.n0 + 9, cfg.n_img), classify=False, labels_override=lab)
+        assert r.steps_checked == 3 * len(layers)
