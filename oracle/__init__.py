@@ -221,3 +221,50 @@ def decode_batch(q, K_hist, V_hist, is_semantic, idx, cnt, L, t, W, M, R, scale=
                                   default_scale(D) if scale is None else scale, int(bool(full)),
                                   _p(out, C.c_double))
     return out
+
+
+class RowBufferOverflow(RuntimeError):
+    """Algorithm 2: a token was appended to a row buffer that already holds R tokens."""
+
+
+def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=None):
+    """Algorithm 2 (compression with a row buffer) for ONE semantic (sequence, head), step by step.
+
+    Q [N,D] image queries, K, V [L+N,D] (uint16 bf16).  State: a static set of at most M image
+    tokens with their accumulated attention scores, and a row buffer of at most R tokens.
+      prefill (image step n0):  scores = running sum of attention over steps 1..n0 (Algorithm 1);
+                                static = top-M of them over all n0 tokens; buffer empty.
+      decode step t = n0+1..t_end, in the algorithm's order:
+        append token t-1 to the buffer (overflow is an error); attend over prompt + static + buffer;
+        add the step's attention weights to the scores of the static and buffered tokens;
+        if the buffer holds R tokens: keep the top-M of static + buffer by score (ties: lowest
+        position), in ascending position; empty the buffer.
+    Returns (outs [t_end-n0, D] fp64, history): history[k] = (t, static positions after step t,
+    scores of those positions) for every step.
+    """
+    Q, K, V = _u16(Q), _u16(K), _u16(V)
+    sc = scores(Q[:n0], K[: L + n0], L, n0, scale) if n0 > 0 else np.zeros(0)
+    static = topm(sc, n0, M).tolist()
+    acc = {j: float(sc[j]) for j in static}
+    buf = []
+    outs, hist = [], []
+    for t in range(n0 + 1, t_end + 1):
+        if len(buf) + 1 > R:
+            raise RowBufferOverflow(f"step {t}: row buffer of {R} is full")
+        buf.append(t - 1)
+        acc[t - 1] = 0.0
+        held = static + buf
+        pos = np.array(list(range(L)) + [L + j for j in held], np.int32)
+        out, wts = attend(Q[t - 1], K, V, pos, scale, return_weights=True)
+        for k, j in enumerate(held):
+            acc[j] += float(wts[L + k])
+        outs.append(out)
+        if compress_when_full and len(buf) == R:
+            cand = held                                   # ascending positions by construction
+            s = np.array([acc[j] for j in cand], np.float64)
+            keep = topm(s, len(cand), M)
+            static = [cand[i] for i in keep]
+            acc = {j: acc[j] for j in static}
+            buf = []
+        hist.append((t, list(static), [acc[j] for j in static], list(buf), [acc[j] for j in buf]))
+    return np.array(outs), hist

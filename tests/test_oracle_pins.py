@@ -330,3 +330,64 @@ def test_decode_batch_agrees_with_single_pair_functions():
             assert len(pos) == min(cfg.slots(bool(sem[0, h])), L + t)
             want = oracle.attend(qu[0, h, t - 1], ku[0, h], vu[0, h], pos)
             assert np.array_equal(out[0, h], want)
+
+
+# ------------------------------------------------------------------ Algorithm 2 (row buffer)
+def test_rowbuf_nothing_dropped_is_full_attention_and_running_sum():
+    rng = np.random.default_rng(20)
+    L, N, D, n0, R = 3, 14, 8, 4, 3
+    Q, K, V = rand_bf16(rng, N, D), rand_bf16(rng, L + N, D), rand_bf16(rng, L + N, D)
+    outs, hist = oracle.rowbuf_semantic(Q, K, V, L, n0, N, R, N)          # M = N: nothing is ever dropped
+    for k, t in enumerate(range(n0 + 1, N + 1)):
+        mask = np.arange(L + N) < L + t
+        assert np.allclose(outs[k], _sdpa_fp64(Q[t - 1], K, V, mask), rtol=1e-11, atol=1e-13)
+    # accumulated scores = Algorithm 1's running sum over all steps so far (already pinned above)
+    t, static, acc, buf, bacc = hist[-1]
+    held = static + buf
+    want = oracle.scores(Q[:N], K, L, N)
+    assert held == list(range(N))
+    assert np.allclose(np.array(acc + bacc), want, rtol=1e-12, atol=1e-15)
+
+
+def test_rowbuf_compresses_when_full_and_overflows_otherwise():
+    rng = np.random.default_rng(21)
+    L, N, D, n0, M, R = 2, 20, 8, 6, 4, 3
+    Q, K, V = rand_bf16(rng, N, D), rand_bf16(rng, L + N, D), rand_bf16(rng, L + N, D)
+    outs, hist = oracle.rowbuf_semantic(Q, K, V, L, n0, M, R, N)
+    for t, static, acc, buf, _ in hist:
+        assert len(static) <= M and len(buf) < R and len(static) + len(buf) <= M + R
+        assert static == sorted(set(static)) and all(j < t for j in static + buf)
+        assert len(buf) == (t - n0) % R                       # emptied every R steps
+        assert all(a >= 0 for a in acc)
+    with pytest.raises(oracle.RowBufferOverflow):
+        oracle.rowbuf_semantic(Q, K, V, L, n0, M, R, n0 + R + 1, compress_when_full=False)
+    # brute force of one cycle: scores after R steps and the re-selection
+    sc0 = oracle.scores(Q[:n0], K[: L + n0], L, n0)
+    static = oracle.topm(sc0, n0, M).tolist()
+    acc = {j: sc0[j] for j in static}
+    held = list(static)
+    for t in range(n0 + 1, n0 + R + 1):
+        held.append(t - 1)
+        acc[t - 1] = 0.0
+        pos = np.array(list(range(L)) + [L + j for j in held], np.int32)
+        a = oracle.attention_row(Q[t - 1], K[pos])
+        for k, j in enumerate(held):
+            acc[j] += a[L + k]
+    order = sorted(held, key=lambda j: (-acc[j], j))[:M]
+    assert hist[R - 1][1] == sorted(order)
+    assert np.allclose(hist[R - 1][2], [acc[j] for j in sorted(order)], rtol=1e-12)
+
+
+def test_rowbuf_promotes_a_heavily_attended_buffer_token():
+    # one-hot keys: every decode query looks at the token appended at step n0+1, which must then
+    # displace the least-attended static token at the first compression
+    N, D, L, n0, M, R, c = 12, 128, 0, 6, 3, 3, 128.0
+    K = _onehot_keys(N, D, c, L)
+    Q = np.zeros((N, D))
+    Q[:n0, 0] = c                         # prefill steps look at token 0
+    Q[n0:, n0] = c                        # decode steps look at token n0 (first buffered token)
+    V = np.random.default_rng(22).standard_normal((N, D))
+    outs, hist = oracle.rowbuf_semantic(bf16(Q), bf16(K), bf16(V), L, n0, M, R, n0 + R)
+    t, static, acc, buf, _ = hist[-1]
+    assert n0 in static and 0 in static and buf == []
+    assert abs(acc[static.index(n0)] - R) < 1e-9              # R steps of weight ~1 each
