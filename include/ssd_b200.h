@@ -125,6 +125,27 @@ int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v
  * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
 int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
+/* Row-buffer mode (Algorithm 2, Appendix B).  With the mode on, the ring of a semantic head is the
+ * algorithm's row buffer of R = sink_recent tokens, filled from empty:
+ *   ssd_compress     selects the top-M over all n0 tokens (the buffer starts empty) and records the
+ *                    selected tokens' scores;
+ *   ssd_append       puts the token into the buffer; SSD_ERR_OVERFLOW when the buffer already holds R
+ *                    tokens ("row buffer overflow"): call ssd_recompress first;
+ *   ssd_decode_attn  attends over prompt + static set + buffer and keeps the step's attention weights
+ *                    of the static and buffered tokens of semantic heads; they are added to the tokens'
+ *                    accumulated scores by the layer's next ssd_append or ssd_recompress;
+ *   ssd_recompress   ("row buffer full"): per (sequence, semantic head) keeps the top-M of static set +
+ *                    buffer by accumulated score (ties: lowest position) as the new static set, in
+ *                    ascending position, and empties the buffer.  Asynchronous.
+ * Spatial heads keep exactly their W newest tokens in both modes.  ssd_cache_set_row_buffer switches the
+ * mode and resets every layer to the empty state (call it before ssd_compress).
+ * ssd_cache_get_scores: acc_host [n_seqs, n_heads, M + R] accumulated scores, entry e < M for static
+ * slot e, entry M + r for buffer slot r, including the last decode's weights; -1 for entries that hold no
+ * token or belong to spatial heads.  Synchronises the device. */
+int ssd_cache_set_row_buffer(ssd_cache *cache, int32_t enable);
+int ssd_recompress(ssd_cache *cache, int32_t layer, void *stream);
+int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
+
 /* ssd_decode_attn for callers that cannot allocate.  The paper has no counterpart; this is a
  * packaging variant of the same kernel.  ssd_decode_attn keeps the kernel's scratch (partial sums of
  * heads that two thread blocks share, and per-head arrival counters) inside the buffer given to

@@ -227,7 +227,7 @@ class RowBufferOverflow(RuntimeError):
     """Algorithm 2: a token was appended to a row buffer that already holds R tokens."""
 
 
-def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=None):
+def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=None, choose=None):
     """Algorithm 2 (compression with a row buffer) for ONE semantic (sequence, head), step by step.
 
     Q [N,D] image queries, K, V [L+N,D] (uint16 bf16).  State: a static set of at most M image
@@ -240,7 +240,10 @@ def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=
         if the buffer holds R tokens: keep the top-M of static + buffer by score (ties: lowest
         position), in ascending position; empty the buffer.
     Returns (outs [t_end-n0, D] fp64, history): history[k] = (t, static positions after step t,
-    scores of those positions) for every step.
+    their scores, buffered positions, their scores) for every step.
+    `choose(t, candidates, scores, keep)` may replace the kept candidate indices at a compression (a
+    parity test uses it to follow another implementation's choice where scores tie within a tolerance);
+    by default the oracle's own top-M stands.
     """
     Q, K, V = _u16(Q), _u16(K), _u16(V)
     sc = scores(Q[:n0], K[: L + n0], L, n0, scale) if n0 > 0 else np.zeros(0)
@@ -263,6 +266,8 @@ def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=
             cand = held                                   # ascending positions by construction
             s = np.array([acc[j] for j in cand], np.float64)
             keep = topm(s, len(cand), M)
+            if choose is not None:
+                keep = np.asarray(choose(t, cand, s, keep), np.int32)
             static = [cand[i] for i in keep]
             acc = {j: acc[j] for j in static}
             buf = []

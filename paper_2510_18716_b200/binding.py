@@ -30,6 +30,7 @@ EXPORTS = [
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
+    "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores",
 ]
 
 
@@ -76,6 +77,9 @@ def load():
     L.ssd_append.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_decode_attn.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_decode_attn_static.argtypes = [vp, i32, vp, vp, vp]
+    L.ssd_cache_set_row_buffer.argtypes = [vp, i32]
+    L.ssd_recompress.argtypes = [vp, i32, vp]
+    L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
     L.ssd_cache_max_slots.argtypes = [vp]
@@ -236,6 +240,19 @@ class SsdCache:
         self._check(self.lib.ssd_decode_attn_static(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"),
                                                     _stream()), "ssd_decode_attn_static")
         return out
+
+    # -- Algorithm 2 (row buffer)
+    def set_row_buffer(self, enable: bool = True):
+        self._check(self.lib.ssd_cache_set_row_buffer(self._h, 1 if enable else 0), "ssd_cache_set_row_buffer")
+
+    def recompress(self, layer: int):
+        self._check(self.lib.ssd_recompress(self._h, layer, _stream()), "ssd_recompress")
+
+    def get_scores(self, layer: int) -> np.ndarray:
+        c = self.cfg
+        a = np.empty((c.n_seqs, c.n_heads, c.sink_budget + c.sink_recent), np.float32)
+        self._check(self.lib.ssd_cache_get_scores(self._h, layer, a.ctypes.data), "ssd_cache_get_scores")
+        return a
 
     def step_host(self, layer: int, q_host, k_new_host, v_new_host, out_host):
         """One append + decode of a layer from (pinned) host bf16 tensors; asynchronous."""

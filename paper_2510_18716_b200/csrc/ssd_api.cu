@@ -16,7 +16,7 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Regions {
-  size_t desc, idx, counters, status, partial, score, staging, slab;  // byte offsets
+  size_t desc, idx, counters, status, partial, score, staging, acc, logits, ml, slab;  // byte offsets
   size_t score_bytes, partial_bytes, front_bytes;
 };
 
@@ -50,6 +50,12 @@ static Regions plan_regions(const ssd_config& c) {
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
   r.score = off;     off = align_up(off + r.score_bytes);
   r.staging = off;   off = align_up(off + 4 * pairs_layer * kHeadDim * 2);
+  // row-buffer mode (Algorithm 2): accumulated scores and the last decode's logits of the static and
+  // ring slots, and the last decode's (max, exp-sum), per layer
+  const size_t mr = (size_t)c.sink_budget + c.sink_recent;
+  r.acc = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * mr * 4);
+  r.logits = off;    off = align_up(off + (size_t)c.n_layers * pairs_layer * mr * 4);
+  r.ml = off;        off = align_up(off + (size_t)c.n_layers * pairs_layer * 8);
   r.front_bytes = off;
   r.slab = off;
   return r;
@@ -72,6 +78,9 @@ struct ssd_cache {
   std::vector<int64_t> layer_base;    // [layers] first slot of the layer in the slab
   std::vector<int32_t> n_sink;        // [layers]
   std::vector<int32_t> t_img, n0, prompt_valid, static_valid;  // [layers]
+  bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
+  std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
+  std::vector<uint8_t> pending;       // [layers] last decode's logits not yet added to the scores
   std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
   int prof_n = 0;                     // launches recorded since the last collect
 
@@ -82,6 +91,13 @@ struct ssd_cache {
   }
   uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(base + reg.status); }
+  int mr() const { return cfg.sink_budget + cfg.sink_recent; }
+  size_t layer_scores(int layer) const { return (size_t)layer * cfg.n_seqs * cfg.n_heads * mr(); }
+  float* d_acc(int layer) const { return reinterpret_cast<float*>(base + reg.acc) + layer_scores(layer); }
+  float* d_logits(int layer) const { return reinterpret_cast<float*>(base + reg.logits) + layer_scores(layer); }
+  float2* d_ml(int layer) const { return reinterpret_cast<float2*>(base + reg.ml) + (size_t)layer * cfg.n_seqs * cfg.n_heads; }
+  // tokens in the rings of semantic heads
+  int sem_tokens(int layer) const { return row_buffer ? t_img[layer] - t_base[layer] : t_img[layer]; }
   float* d_partial() const { return reinterpret_cast<float*>(base + reg.partial); }
   float* d_score() const { return reinterpret_cast<float*>(base + reg.score); }
   char* d_staging() const { return base + reg.staging; }
@@ -96,6 +112,7 @@ struct ssd_cache {
     v.prompt_valid = prompt_valid[layer];
     v.static_valid = static_valid[layer];
     v.t_img = t_img[layer];
+    v.t_sem = sem_tokens(layer);
     for (int h = 0; h < cfg.n_heads; ++h) {
       const HeadDesc& d = desc[(size_t)layer * cfg.n_heads + h];
       v.head[h] = HeadRec{d.x, d.y, d.z, d.w};
@@ -163,6 +180,8 @@ int ssd_cache_create(const ssd_config* cfg, void* dev_mem, size_t dev_bytes, ssd
   c->n0.assign(cfg->n_layers, 0);
   c->prompt_valid.assign(cfg->n_layers, 0);
   c->static_valid.assign(cfg->n_layers, 0);
+  c->t_base.assign(cfg->n_layers, 0);
+  c->pending.assign(cfg->n_layers, 0);
   if (cudaMemset(c->base, 0, r.front_bytes) != cudaSuccess ||
       cudaMemset(c->base + r.idx, 0xFF, r.counters - r.idx) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
@@ -248,7 +267,10 @@ int ssd_set_head_labels(ssd_cache* c, const uint8_t* labels_host) {
   }
   c->desc.swap(desc);
   for (size_t i = 0; i < nh; ++i) c->labels[i] = labels_host[i] ? 1 : 0;
-  for (int l = 0; l < g.n_layers; ++l) c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = 0;
+  for (int l = 0; l < g.n_layers; ++l) {
+    c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = c->t_base[l] = 0;
+    c->pending[l] = 0;
+  }
   c->labels_set = true;
   return SSD_OK;
 }
@@ -320,7 +342,9 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (g.prompt_len + n0 < 1) return SSD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int n_cand = n0 - g.sink_recent > 0 ? n0 - g.sink_recent : 0;
+  // the R newest tokens stay in the ring and are not candidates; with a row buffer (Algorithm 2,
+  // prefill) the buffer starts empty and every token is a candidate
+  const int n_cand = c->row_buffer ? n0 : (n0 - g.sink_recent > 0 ? n0 - g.sink_recent : 0);
   const int sv = g.sink_budget < n_cand ? g.sink_budget : n_cand;
   const bool select = c->n_sink[layer] > 0 && sv > 0;
   if (select && n_obs > 0 && !q_obs) return SSD_ERR_INVALID_ARG;
@@ -343,6 +367,8 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
     sl.score = c->d_score();
     sl.desc = desc;
     sl.static_idx = c->d_idx(layer);
+    sl.acc = c->row_buffer ? c->d_acc(layer) : nullptr;
+    sl.mr = c->mr();
     sl.n_seqs = g.n_seqs; sl.H = g.n_heads; sl.M = g.sink_budget; sl.n0 = n0; sl.n_cand = n_cand;
     if (launch_select(sl, st) != cudaSuccess) return SSD_ERR_CUDA;
   }
@@ -350,6 +376,7 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   gp.slab = c->d_slab(layer);
   gp.desc = desc;
   gp.static_idx = c->d_idx(layer);
+  gp.sem_ring = c->row_buffer ? 0 : 1;
   gp.k_full = static_cast<const uint4*>(k_full);
   gp.v_full = static_cast<const uint4*>(v_full);
   gp.n_seqs = g.n_seqs; gp.H = g.n_heads; gp.L = g.prompt_len; gp.M = g.sink_budget; gp.n0 = n0;
@@ -360,6 +387,8 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   c->n0[layer] = n0;
   c->prompt_valid[layer] = g.prompt_len;
   c->static_valid[layer] = select ? sv : 0;
+  c->t_base[layer] = n0;
+  c->pending[layer] = 0;
   return SSD_OK;
 }
 
@@ -369,6 +398,8 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent)
+    return SSD_ERR_OVERFLOW;            // Algorithm 2: row buffer overflow; call ssd_recompress first
   AppendParams p;
   p.slab = c->d_slab(layer);
   p.desc = c->d_desc(layer);
@@ -377,7 +408,15 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
   p.j = c->t_img[layer];
   p.seq_slots = c->seq_slots[layer];
+  p.sem_slot = c->sem_tokens(layer);
+  p.static_valid = c->static_valid[layer];
+  p.pending = c->pending[layer];
+  p.mr = c->mr();
+  p.acc = c->row_buffer ? c->d_acc(layer) : nullptr;
+  p.logits = c->d_logits(layer);
+  p.ml = c->d_ml(layer);
   if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  if (c->row_buffer) c->pending[layer] = 0;
   c->t_img[layer] += 1;
   return SSD_OK;
 }
@@ -396,6 +435,9 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.partial = c->d_partial();
   p.counters = c->d_counters();
   p.status = c->d_status();
+  p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
+  p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
+  p.mr = c->mr();
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
@@ -403,6 +445,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  if (c->row_buffer) c->pending[layer] = 1;
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -463,8 +506,12 @@ int ssd_cache_get_indices(ssd_cache* c, int32_t layer, int32_t* idx_host) {
           int j = sidx[((size_t)s * g.n_heads + h) * (M > 0 ? M : 1) + m];
           o[L + m] = j >= 0 ? L + j : -1;
         }
-      for (int r = 0; r < d.z; ++r)
-        if (t - 1 >= r) o[L + d.y + r] = L + ((t - 1 - r) / d.z) * d.z + r;
+      if (d.w && c->row_buffer) {       // row buffer: filled from slot 0 since the last re-selection
+        for (int r = 0; r < c->sem_tokens(layer) && r < d.z; ++r) o[L + d.y + r] = L + c->t_base[layer] + r;
+      } else {
+        for (int r = 0; r < d.z; ++r)
+          if (t - 1 >= r) o[L + d.y + r] = L + ((t - 1 - r) / d.z) * d.z + r;
+      }
     }
   return SSD_OK;
 }
@@ -476,8 +523,8 @@ int ssd_cache_get_lengths(ssd_cache* c, int32_t layer, int32_t* len_host) {
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   for (int h = 0; h < g.n_heads; ++h) {
     const HeadDesc& d = c->desc[(size_t)layer * g.n_heads + h];
-    len_host[h] = c->prompt_valid[layer] + (d.w ? c->static_valid[layer] : 0) +
-                  (c->t_img[layer] < d.z ? c->t_img[layer] : d.z);
+    const int tok = d.w ? c->sem_tokens(layer) : c->t_img[layer];
+    len_host[h] = c->prompt_valid[layer] + (d.w ? c->static_valid[layer] : 0) + (tok < d.z ? tok : d.z);
   }
   return SSD_OK;
 }
@@ -497,6 +544,7 @@ int32_t ssd_cache_tokens(const ssd_cache* c, int32_t layer) {
 int ssd_cache_rewind(ssd_cache* c, int32_t layer, int32_t t) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return SSD_ERR_INVALID_ARG;
   if (t < c->n0[layer] || t > c->t_img[layer]) return SSD_ERR_INVALID_ARG;
+  if (c->row_buffer) return SSD_ERR_BAD_STATE;   // the static sets have moved on; replay is meaningless
   c->t_img[layer] = t;
   return SSD_OK;
 }
@@ -507,6 +555,74 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
   size_t slots = 0;
   for (int l = 0; l < c->cfg.n_layers; ++l) slots += (size_t)c->seq_slots[l];
   *bytes_per_seq = slots * kSlotBytes;
+  return SSD_OK;
+}
+
+int ssd_cache_set_row_buffer(ssd_cache* c, int32_t enable) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  c->row_buffer = enable != 0;
+  for (int l = 0; l < c->cfg.n_layers; ++l) {
+    c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = c->t_base[l] = 0;
+    c->pending[l] = 0;
+  }
+  return SSD_OK;
+}
+
+int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set || !c->row_buffer) return SSD_ERR_BAD_STATE;
+  const int buffered = c->sem_tokens(layer);
+  if (c->n_sink[layer] > 0 && (buffered > 0 || c->pending[layer])) {
+    RecompressParams p;
+    p.slab = c->d_slab(layer);
+    p.desc = c->d_desc(layer);
+    p.static_idx = c->d_idx(layer);
+    p.acc = c->d_acc(layer);
+    p.logits = c->d_logits(layer);
+    p.ml = c->d_ml(layer);
+    p.pending = c->pending[layer];
+    p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len; p.M = g.sink_budget; p.mr = c->mr();
+    p.static_valid = c->static_valid[layer];
+    p.buffered = buffered;
+    p.t_base = c->t_base[layer];
+    p.seq_slots = c->seq_slots[layer];
+    if (launch_recompress(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+    const int n = c->static_valid[layer] + buffered;
+    c->static_valid[layer] = n < g.sink_budget ? n : g.sink_budget;
+  }
+  c->t_base[layer] = c->t_img[layer];
+  c->pending[layer] = 0;
+  return SSD_OK;
+}
+
+int ssd_cache_get_scores(ssd_cache* c, int32_t layer, float* acc_host) {
+  if (!c || !acc_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set || !c->row_buffer) return SSD_ERR_BAD_STATE;
+  const size_t n = (size_t)g.n_seqs * g.n_heads * c->mr();
+  std::vector<float> lg(n);
+  std::vector<float2> ml((size_t)g.n_seqs * g.n_heads);
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(acc_host, c->d_acc(layer), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(lg.data(), c->d_logits(layer), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(ml.data(), c->d_ml(layer), ml.size() * 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  const int mr = c->mr(), sv = c->static_valid[layer], b = c->sem_tokens(layer);
+  for (int pr = 0; pr < g.n_seqs * g.n_heads; ++pr) {
+    const HeadDesc& d = c->desc[(size_t)layer * g.n_heads + pr % g.n_heads];
+    float* a = acc_host + (size_t)pr * mr;
+    for (int e = 0; e < mr; ++e) {
+      const bool valid = d.w && (e < sv || (e >= d.y && e < d.y + b));
+      if (!valid) { a[e] = -1.f; continue; }
+      // what the next append or re-selection would add first: the last decode's normalised weights
+      if (c->pending[layer]) a[e] += std::exp2(lg[(size_t)pr * mr + e] - ml[pr].x) / ml[pr].y;
+    }
+  }
   return SSD_OK;
 }
 
@@ -531,7 +647,7 @@ int64_t ssd_debug_decode_plan(int32_t n_heads, const int32_t* head_recs, int32_t
   if (chunk <= 0) chunk = decode_chunk_slots();
   LayerView v;
   v.H = n_heads; v.L = prompt_len; v.n_seqs = n_seqs;
-  v.prompt_valid = prompt_valid; v.static_valid = static_valid; v.t_img = t_img;
+  v.prompt_valid = prompt_valid; v.static_valid = static_valid; v.t_img = t_img; v.t_sem = t_img;
   int off = 0;
   for (int h = 0; h < n_heads; ++h) {
     const int32_t* r = head_recs + 4 * h;
@@ -640,9 +756,13 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.partial = reinterpret_cast<float*>(base);
   p.counters = reinterpret_cast<uint32_t*>(base + kStaticPartialBytes);
   p.status = c->d_status();
+  p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
+  p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
+  p.mr = c->mr();
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  if (c->row_buffer) c->pending[layer] = 1;
   return SSD_OK;
 }

@@ -236,8 +236,18 @@ __device__ __forceinline__ void load_stage(const uint4* __restrict__ sb, int n, 
   }
 }
 
+// Where the logits of a chunk go when the scores of semantic heads are being accumulated
+// (Algorithm 2): row = the head's logit row (null: nothing to record), slot s of the chunk is valid
+// slot i0 + s of the head; valid slots below `skip` are prompt slots (not scored) and those from
+// `ring_from` on sit `ring_shift` entries further (unused static capacity in between).
+struct LogitSink {
+  float* row;
+  int i0, skip, ring_from, ring_shift;
+};
+
 // Fold those slots into the running state of this lane's group.
-__device__ __forceinline__ void fold_stage(const Rows& r, int n, int grp, const float2 (&q)[8], State& st) {
+__device__ __forceinline__ void fold_stage(const Rows& r, int n, int grp, int l8, const float2 (&q)[8], State& st,
+                                           const LogitSink& sink) {
 #pragma unroll
   for (int s = 0; s < kPer; s += kU) {
     if (kGroups * s >= n) break;
@@ -248,6 +258,14 @@ __device__ __forceinline__ void fold_stage(const Rows& r, int n, int grp, const 
     for (int off = 4; off >= 1; off >>= 1) {
 #pragma unroll
       for (int u = 0; u < kU; ++u) x[u] += __shfl_xor_sync(0xffffffffu, x[u], off);
+    }
+    if (sink.row != nullptr && l8 == 0) {
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+        const int slot = kGroups * (s + u) + grp;
+        const int li = sink.i0 + slot;
+        if (slot < n && li >= sink.skip) sink.row[li - sink.skip + (li >= sink.ring_from ? sink.ring_shift : 0)] = x[u];
+      }
     }
     float mn = st.m;
 #pragma unroll
@@ -370,6 +388,7 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
       merge4(m, l, acc, __ldcg(G), __ldcg(G + 1), __ldcg(reinterpret_cast<const float4*>(G + 4) + lane));
     }
     write_out4(p.out + (size_t)pair * kHeadDim, l, acc, lane);
+    if (p.ml != nullptr && lane == 0) p.ml[pair] = make_float2(m, l);
     if (lane == 0) p.counters[pair] = 0u;
   }
 }
@@ -473,6 +492,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   int piece_i0 = 0;
   float2 q[8];
   State st;
+  LogitSink sink = {nullptr, 0, 0, 0, 0};
 
 #pragma unroll 1
   while (cons.g < cons.g_end) {
@@ -498,13 +518,19 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
       piece_i0 = cons.i;
       leading = cons.g == g_begin;      // the piece that holds the share's first slot
       begin = false;
+      const HeadRec d = v.head[cons.head];
+      sink.row = (p.logits != nullptr && d.w) ? p.logits + ((size_t)cons.seq * v.H + cons.head) * p.mr : nullptr;
+      sink.skip = v.prompt_valid;
+      sink.ring_from = v.prompt_valid + v.static_valid;
+      sink.ring_shift = d.y - v.static_valid;
     }
+    sink.i0 = cons.i;
     Rows rows;
     load_stage(sb, n, grp, l8, rows);
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
     if (prod.g < prod.g_end) issue(stage);
-    fold_stage(rows, n, grp, q, st);
+    fold_stage(rows, n, grp, l8, q, st, sink);
 
     const int i1 = cons.i + n;
     if (i1 == cons.vh || cons.g + n == cons.g_end) {
@@ -515,6 +541,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
       state_merge_lane(tot, 16);
       if (piece_i0 == 0 && i1 == cons.vh) {
         if (grp == 0) write_out(p.out + ((size_t)cons.seq * v.H + cons.head) * kHeadDim, tot, l8);
+        if (p.ml != nullptr && lane == 0) p.ml[(size_t)cons.seq * v.H + cons.head] = make_float2(tot.m, tot.l);
       } else {
         // post the partial; the worker that posts a head's last piece in this CTA merges them
         float* P = mail + (size_t)(2 * warp + (leading ? 0 : 1)) * kPartialFloats;
@@ -554,6 +581,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
           }
           if (w_lo >= lo_c && w_hi <= hi_c) {              // the whole head lies inside this CTA
             write_out4(p.out + ((size_t)cons.seq * v.H + cons.head) * kHeadDim, l, acc, lane);
+            if (p.ml != nullptr && lane == 0) p.ml[(size_t)cons.seq * v.H + cons.head] = make_float2(m, l);
           } else {                                         // hand the CTA's partial to the finisher
             const int slot = w_lo < lo_c ? 0 : 1;
             float* C = mail + (size_t)(2 * kWarps + slot) * kPartialFloats;
@@ -581,7 +609,25 @@ __global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   if (warp >= p.n_seqs * p.H) return;
   const int seq = warp / p.H, head = warp - seq * p.H;
   const HeadDesc d = p.desc[head];
-  const int ring_slot = p.j % d.z;
+  int ring_slot = p.j % d.z;
+  if (p.acc != nullptr && d.w) {
+    // Algorithm 2: the ring of a semantic head is a row buffer filled from slot 0.  First bring the
+    // scores up to date with the attention of the layer's last decode ("accumulate semantic
+    // attention scores"), then start the new token's score at zero.
+    float* acc = p.acc + (size_t)warp * p.mr;
+    if (p.pending) {
+      const float* lg = p.logits + (size_t)warp * p.mr;
+      const float2 ml = p.ml[warp];
+      const float inv = 1.f / ml.y;
+      const int n = p.static_valid + p.sem_slot;
+      for (int i = lane; i < n; i += 32) {
+        const int c = i < p.static_valid ? i : d.y + (i - p.static_valid);
+        acc[c] += ex2(lg[c] - ml.x) * inv;
+      }
+    }
+    ring_slot = p.sem_slot;
+    if (lane == 0) acc[d.y + ring_slot] = 0.f;
+  }
   uint4* dst = p.slab + ((size_t)seq * p.seq_slots + d.x + p.L + d.y + ring_slot) * kSlotU4;
   const uint4* src = (lane < 16 ? p.k_new : p.v_new) + (size_t)warp * 16 + (lane & 15);
   dst[lane] = *src;

@@ -32,6 +32,10 @@ struct DecodeParams {
   float* partial;           // [max workers * 2, kPartialFloats]
   uint32_t* counters;       // [n_seqs * H], zero between launches
   uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
+  float* logits;            // row-buffer mode: [n_seqs * H, M + R] logits (base 2) of the static and
+                            // ring slots of semantic heads, for the score accumulation; else null
+  float2* ml;               // row-buffer mode: [n_seqs * H] final (max, exp-sum) of each head; else null
+  int mr;                   // M + R
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
   LayerView view;           // layout and occupancy of the layer
@@ -45,11 +49,20 @@ struct AppendParams {
   int n_seqs, H, L;
   int j;                    // image index of the token being appended
   int seq_slots;
+  // row-buffer mode (Algorithm 2); acc == nullptr otherwise
+  int sem_slot;             // ring slot of semantic heads for this token (tokens buffered so far)
+  int static_valid;         // valid static slots of semantic heads
+  int pending;              // 1: the logits of the layer's last decode are not yet in the scores
+  int mr;                   // M + R
+  float* acc;               // [n_seqs * H, M + R] accumulated attention scores
+  const float* logits;      // [n_seqs * H, M + R]
+  const float2* ml;         // [n_seqs * H]
 };
 
 struct GatherParams {
   uint4* slab;
   const HeadDesc* desc;
+  int sem_ring;              // 0: leave the rings of semantic heads empty (row-buffer mode)
   const int32_t* static_idx; // [n_seqs, H, M] image indices, ascending, -1 padded
   const uint4* k_full;       // [n_seqs, H, L + n0, 16] uint4
   const uint4* v_full;
@@ -72,6 +85,8 @@ struct SelectParams {
   const float* score;          // [n_seqs, H, n0]
   const HeadDesc* desc;
   int32_t* static_idx;         // [n_seqs, H, M]
+  float* acc;                  // row-buffer mode: [n_seqs * H, mr], gets the selected tokens' scores; else null
+  int mr;
   int n_seqs, H, M, n0, n_cand;
 };
 
@@ -89,6 +104,21 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
+struct RecompressParams {
+  uint4* slab;
+  const HeadDesc* desc;
+  int32_t* static_idx;         // [n_seqs, H, M] image indices of the static slots (updated)
+  float* acc;                  // [n_seqs * H, mr] accumulated scores (updated)
+  const float* logits;         // pending logits of the last decode
+  const float2* ml;
+  int pending;
+  int n_seqs, H, L, M, mr;
+  int static_valid;            // valid static slots before the call
+  int buffered;                // tokens in the row buffer
+  int t_base;                  // image index of the buffer's first token
+  int seq_slots;
+};
+cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st);
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st);
 int classify_rows_per_block();
 int decode_max_workers();

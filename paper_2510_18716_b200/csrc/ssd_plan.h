@@ -35,17 +35,24 @@ struct LayerView {
   int32_t H, L, n_seqs, seq_slots;  // seq_slots = physical slots per sequence in this layer
   int32_t prompt_valid;             // 0 or L
   int32_t static_valid;             // valid static slots of semantic heads
-  int32_t t_img;                    // image tokens held; a ring holds min(t_img, z) of them
+  int32_t t_img;                    // image tokens held; a spatial ring holds min(t_img, z) of them
+  int32_t t_sem;                    // same count for semantic rings: t_img, or the tokens buffered since
+                                    // the last re-selection when the ring is used as a row buffer
   int32_t contig;                   // 1 if every head's valid slots are one run from its first slot
   int32_t max_vh;                   // most valid slots any head holds
   int32_t cum[kPlanMaxHeads + 1];   // exclusive prefix of valid slots per head
   HeadRec head[kPlanMaxHeads];
 };
 
+// Ring slots of a head that hold a token.
+SSD_HD int ring_valid(const LayerView& v, const HeadRec& d) {
+  const int t = d.w ? v.t_sem : v.t_img;
+  return t < d.z ? t : d.z;
+}
+
 SSD_HD int head_valid(const LayerView& v, int h) {
   const HeadRec d = v.head[h];
-  const int rv = v.t_img < d.z ? v.t_img : d.z;
-  return v.prompt_valid + (d.w ? v.static_valid : 0) + rv;
+  return v.prompt_valid + (d.w ? v.static_valid : 0) + ring_valid(v, d);
 }
 
 // Fill the fields derived from the others: cum[], max_vh, contig.
@@ -192,7 +199,7 @@ template <class Emit>
 SSD_HD void chunk_runs(const LayerView& v, int h, int i, int n, Emit emit) {
   const HeadRec d = v.head[h];
   const int sv = d.w ? v.static_valid : 0;
-  const int rv = v.t_img < d.z ? v.t_img : d.z;
+  const int rv = ring_valid(v, d);
   const int l0[3] = {0, v.prompt_valid, v.prompt_valid + sv};  // logical start of each run
   const int ln[3] = {v.prompt_valid, sv, rv};
   const int p0[3] = {0, v.L, v.L + d.y};                       // physical start of each run

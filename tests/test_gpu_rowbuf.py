@@ -1,0 +1,125 @@
+"""GPU parity of the row-buffer mode (Algorithm 2): append into the buffer, attend over prompt +
+static set + buffer, accumulate the attention scores of semantic heads, re-select when the buffer is
+full -- against the fp64 oracle, step by step, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_18716_b200 import binding as B
+from paper_2510_18716_b200 import workloads as wl
+
+from parity_util import BAND, check_outputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, layer, seqs, t_end):
+    dev = torch.device("cuda:0")
+    L, n0, M, R, W, H, S = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.window, cfg.n_heads, len(seqs)
+    labels = wl.sink_mask(cfg, layer)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=S), device=dev)
+    cache.set_row_buffer(True)
+    cache.set_head_labels(labels)
+    q, k, v, _ = wl.gen_layer(cfg, layer, seqs, device=dev)
+    qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+
+    # the oracle runs each semantic pair on its own, following the GPU's choice inside the tie band
+    gpu_sets = {}          # (s, h, t) -> static image indices after the compression at step t
+    n_band = [0]
+
+    def chooser(s, h):
+        def choose(t, cand, sc, keep):
+            got = gpu_sets[(s, h, t)]
+            want = [cand[i] for i in keep]
+            if got == want:
+                return keep
+            n_band[0] += 1
+            kth = np.sort(sc)[::-1][len(keep) - 1]
+            sure_in = {cand[i] for i in np.nonzero(sc > kth * (1 + BAND))[0]}
+            band = {cand[i] for i in np.nonzero(np.abs(sc - kth) <= BAND * abs(kth))[0]}
+            assert sure_in <= set(got) <= (sure_in | band) and len(got) == len(want)
+            return [cand.index(j) for j in got]
+        return choose
+
+    # GPU pass first (records outputs, sets and scores), then the oracle replays it
+    outs = []
+    for t in range(n0 + 1, t_end + 1):
+        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
+        outs.append(cache.decode_attn(0, q[:, :, t - 1].contiguous()).float().cpu().numpy().astype(np.float64))
+        if (t - n0) % R == 0:
+            cache.recompress(0)
+            gi = cache.get_indices(0)
+            for s in range(S):
+                for h in range(H):
+                    if labels[h]:
+                        st = gi[s, h, L:L + M]
+                        gpu_sets[(s, h, t)] = (st[st >= 0] - L).tolist()
+                        ring = gi[s, h, L + M:L + M + R]
+                        assert (ring == -1).all(), "the buffer is empty after a re-selection"
+            assert (cache.get_lengths(0)[labels == 1] == L + min(M, t)).all()
+    assert cache.device_status() == 0
+
+    for s in range(S):
+        for h in range(H):
+            if labels[h]:
+                want, hist = oracle.rowbuf_semantic(qu[s, h], ku[s, h], vu[s, h], L, n0, M, R, t_end,
+                                                    choose=chooser(s, h))
+                for i, t in enumerate(range(n0 + 1, t_end + 1)):
+                    err = np.abs(outs[i][s, h] - want[i])
+                    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (s, h, t, err.max())
+            else:
+                for i, t in enumerate(range(n0 + 1, t_end + 1)):
+                    pos = oracle.retained_set(False, L, t, W, R)
+                    want = oracle.attend(qu[s, h, t - 1], ku[s, h], vu[s, h], pos)
+                    err = np.abs(outs[i][s, h] - want)
+                    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (s, h, t, err.max())
+    cache.close()
+    return n_band[0]
+
+
+def test_rowbuf_tiny_every_step():
+    cfg = wl.CONFIGS["tiny"]
+    _run(cfg, 0, [0], cfg.n_img)
+
+
+def test_rowbuf_janus1b_slice():
+    cfg = wl.CONFIGS["janus1b"]
+    _run(cfg, 3, [0, 1], cfg.n0 + 3 * cfg.sink_recent + 5)
+
+
+def test_rowbuf_scores_match_oracle_before_reselection():
+    cfg = wl.CONFIGS["tiny"]
+    dev = torch.device("cuda:0")
+    L, n0, M, R, H = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.n_heads
+    labels = wl.sink_mask(cfg, 0)
+    cache = B.SsdCache(B.config_from_workload(cfg), device=dev)
+    cache.set_row_buffer(True)
+    cache.set_head_labels(labels)
+    q, k, v, _ = wl.gen_layer(cfg, 0, [0], device=dev)
+    qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+    for t in range(n0 + 1, n0 + R + 1):
+        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
+        cache.decode_attn(0, q[:, :, t - 1].contiguous())
+    acc = cache.get_scores(0)
+    gi = cache.get_indices(0)
+    for h in range(H):
+        if not labels[h]:
+            assert (acc[0, h] == -1).all()
+            continue
+        _, hist = oracle.rowbuf_semantic(qu[0, h], ku[0, h], vu[0, h], L, n0, M, R, n0 + R, compress_when_full=False)
+        _, static, sacc, buf, bacc = hist[-1]
+        assert (gi[0, h, L:L + M] - L).tolist() == static
+        assert (gi[0, h, L + M:L + M + R] - L).tolist() == buf
+        assert np.allclose(acc[0, h, :M], sacc, rtol=2e-4, atol=1e-6)
+        assert np.allclose(acc[0, h, M:M + R], bacc, rtol=2e-4, atol=1e-6)
+    # one more token without a re-selection: the buffer is full
+    x = k[:, :, L + n0 + R].contiguous()
+    with pytest.raises(B.SsdError) as e:
+        cache.append(0, x, x)
+    assert e.value.code == B.SSD_ERR_OVERFLOW
+    cache.recompress(0)
+    cache.append(0, x, x)                      # accepted again
+    cache.close()
