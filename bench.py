@@ -178,7 +178,7 @@ def run_reference(args, cfg):
 
 
 # ----------------------------------------------------------------------------- our arm
-def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0):
+def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0, row_buffer=False):
     """Create, classify, load and compress every layer; returns the cache and per-layer step inputs."""
     from paper_2510_18716_b200 import binding as B
     from paper_2510_18716_b200 import dist as D
@@ -190,6 +190,8 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
     else:
         ccfg = B.config_from_workload(cfg)
         cache = B.SsdCache(ccfg, n_sink_heads_total=cfg.n_layers * cfg.n_sink_heads, device=device)
+        if row_buffer:
+            cache.set_row_buffer(True)
         mine = D.shard_calibration(cfg.n_cal, rank, world)
         qs, ks = [], []
         for layer in range(cfg.n_layers):
@@ -374,6 +376,34 @@ def run_ours(args, cfg):
         del fcache, fsteps, fst
         torch.cuda.empty_cache()
 
+    # ---- Algorithm 2 (row buffer): append + decode with score accumulation, re-selection every R steps
+    rowbuf = None
+    if not args.no_row_buffer and cfg.n_sink_heads > 0:
+        R = cfg.sink_recent
+        Kb = 2 * R
+        rcache, rsteps = build_cache(cfg, device, rank * S, rank, world, t_steps=Kb + R, row_buffer=True)
+        rstate = {"i": 0}
+
+        def rb_step():
+            i = rstate["i"]
+            for layer in range(cfg.n_layers):
+                qq, kk, vv = rsteps[layer]
+                rcache.append(layer, kk[i], vv[i])
+                rcache.decode_attn(layer, qq[i], out)
+            rstate["i"] += 1
+            if rstate["i"] % R == 0:
+                for layer in range(cfg.n_layers):
+                    rcache.recompress(layer)
+
+        for _ in range(R):            # one whole cycle as warm-up, so the timed region starts on an empty buffer
+            rb_step()
+        ms_b = max_over_ranks(timed(rb_step, Kb, barrier))
+        rowbuf = {"value": cfg.images_per_step * world / (ms_b / Kb * 1e-3), "unit": UNIT, "ms_per_step": ms_b / Kb,
+                  "steps": Kb, "reselect_every": R, "device_status": rcache.device_status()}
+        rcache.close()
+        del rcache, rsteps
+        torch.cuda.empty_cache()
+
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -403,7 +433,7 @@ def run_ours(args, cfg):
                        "kv_bytes_per_seq": kv_bytes_per_seq},
             "sequence_tokens_per_s": value * 2 if S > 1 else value,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "full_cache": full,
+            "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -421,6 +451,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (small profiling case)")
     ap.add_argument("--no-full-cache", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-row-buffer", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = wl.CONFIGS[args.workload]
