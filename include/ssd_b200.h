@@ -125,6 +125,14 @@ int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v
  * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
 int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
+/* ssd_append followed by ssd_decode_attn for the same layer, in one kernel launch (Algorithm 1's
+ * Append and the attention that consumes its output).  Same arguments, results and errors as the two
+ * calls; the newest token's rows are read from k_new / v_new by the attention and stored into the
+ * ring by the same kernel.  k_new, v_new, q, out 16-byte aligned.  In row-buffer mode the call issues
+ * the two launches.  Asynchronous. */
+int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new,
+                      const void *q, void *out, void *stream);
+
 /* Row-buffer mode (Algorithm 2, Appendix B).  With the mode on, the ring of a semantic head is the
  * algorithm's row buffer of R = sink_recent tokens, filled from empty:
  *   ssd_compress     selects the top-M over all n0 tokens (the buffer starts empty) and records the

@@ -30,7 +30,7 @@ EXPORTS = [
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
-    "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores",
+    "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
 ]
 
 
@@ -77,6 +77,7 @@ def load():
     L.ssd_append.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_decode_attn.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_decode_attn_static.argtypes = [vp, i32, vp, vp, vp]
+    L.ssd_append_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_set_row_buffer.argtypes = [vp, i32]
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
@@ -228,6 +229,17 @@ class SsdCache:
             out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
         self._check(self.lib.ssd_decode_attn(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"), _stream()),
                     "ssd_decode_attn")
+        return out
+
+    def append_decode(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor,
+                      out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """append + decode_attn of one layer in a single launch."""
+        c = self.cfg
+        shp = (c.n_seqs, c.n_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
+        self._check(self.lib.ssd_append_decode(self._h, layer, _dev(k_new, shp, "k_new"), _dev(v_new, shp, "v_new"),
+                                               _dev(q, shp, "q"), _dev(out, shp, "out"), _stream()), "ssd_append_decode")
         return out
 
     def decode_attn_static(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -438,6 +438,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
   p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
   p.mr = c->mr();
+  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
@@ -446,6 +447,49 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   if (c->row_buffer) c->pending[layer] = 1;
+  if (timed) {
+    cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
+    c->prof_n += 1;
+  }
+  return SSD_OK;
+}
+
+int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new, const void* q, void* out,
+                      void* stream) {
+  if (!c || !k_new || !v_new || !q || !out) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->row_buffer) {                 // the row buffer's append also maintains the scores: two launches
+    const int rc = ssd_append(c, layer, k_new, v_new, stream);
+    return rc != SSD_OK ? rc : ssd_decode_attn(c, layer, q, out, stream);
+  }
+  if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
+       reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
+    return SSD_ERR_INVALID_ARG;
+  DecodeParams p;
+  p.slab = c->d_slab(layer);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.partial = c->d_partial();
+  p.counters = c->d_counters();
+  p.status = c->d_status();
+  p.logits = nullptr; p.ml = nullptr; p.mr = c->mr();
+  p.k_new = static_cast<const unsigned char*>(k_new);
+  p.v_new = static_cast<const unsigned char*>(v_new);
+  p.new_j = c->t_img[layer];
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  p.split = Split{0, 0, 0, 0, 0.f};
+  c->t_img[layer] += 1;                // the view describes the layer with the token in place
+  c->fill_view(layer, p.view);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
+  if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
+  if (launch_decode(p, st) != cudaSuccess) {
+    c->t_img[layer] -= 1;
+    return SSD_ERR_CUDA;
+  }
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -469,9 +513,7 @@ int ssd_step_host(ssd_cache* c, int32_t layer, const void* q_host, const void* k
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }
-  int rc = ssd_append(c, layer, s + nb, s + 2 * nb, stream);
-  if (rc != SSD_OK) return rc;
-  rc = ssd_decode_attn(c, layer, s, s + 3 * nb, stream);
+  int rc = ssd_append_decode(c, layer, s + nb, s + 2 * nb, s, s + 3 * nb, stream);
   if (rc != SSD_OK) return rc;
   if (cudaMemcpyAsync(out_host, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
     cudaGetLastError();
@@ -759,6 +801,7 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
   p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
   p.mr = c->mr();
+  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);

@@ -28,6 +28,11 @@
 //     order, and no streaming warp executes a global fence or atomic.  A worker whose last head
 //     runs past the CTA's range takes that piece first, which hides the global merge's latency
 //     behind the rest of the streaming.
+// Fused append (ssd_append_decode): the newest token's K/V rows are taken from the caller's
+// k_new / v_new instead of the slab (the chunk that holds the token's ring slot is copied around
+// that slot, and the two rows are copied into its place in the stage), and the worker that
+// consumes that chunk writes the rows into the slab for later steps.  Nothing reads that slab slot
+// during the launch, so no ordering is needed, and the per-layer append launch disappears.
 // Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
 // waits (bounded again) for its other copies in flight and leaves.
 #include "ssd_internal.cuh"
@@ -323,6 +328,15 @@ __device__ __forceinline__ void head_workers(const Split& sp, int wk, int g0, in
   while (w_hi + 1 < sp.W && share_start(sp, w_hi + 1) < g1) ++w_hi;
 }
 
+// Fused append: valid-slot index, inside head h, of the token being appended (its ring slot holds
+// stale bytes in the slab), and that slot's index from the head's first slot.
+__device__ __forceinline__ void new_token_slot(const LayerView& v, int h, int new_j, int& valid_idx, int& phys) {
+  const HeadRec d = v.head[h];
+  const int r = new_j % d.z;
+  valid_idx = v.prompt_valid + (d.w ? v.static_valid : 0) + r;
+  phys = v.L + d.y + r;
+}
+
 // The finisher warp of a CTA carries the (at most two) heads that cross the CTA's own range
 // through global memory: it waits for the CTA's merged partial of such a head (left in a shared-
 // memory mailbox by the worker that completed it), stores it in global scratch, counts arrivals
@@ -468,12 +482,28 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
       // the asynchronous writes that follow
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + (begin ? kQBytes : 0)));
-      if (v.contig) {
-        bulk_g2s(dst, hbase + (size_t)prod.i * kSlotBytes, (uint32_t)n * kSlotBytes, bar);
+      // valid slots [a, a + len) of the head into the stage from slot `at` on
+      auto copy_range = [&](int a, int len, int at) {
+        if (len <= 0) return;
+        if (v.contig) {
+          bulk_g2s(dst + (uint32_t)at * kSlotBytes, hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
+        } else {
+          chunk_runs(v, prod.head, a, len, [&](int src, int d, int l) {
+            bulk_g2s(dst + (uint32_t)(at + d) * kSlotBytes, hbase + (size_t)src * kSlotBytes, (uint32_t)l * kSlotBytes, bar);
+          });
+        }
+      };
+      int fresh = -1, fresh_phys = 0;
+      if (p.new_j >= 0) new_token_slot(v, prod.head, p.new_j, fresh, fresh_phys);
+      if (fresh >= prod.i && fresh < prod.i + n) {
+        // the newest token: its rows come from the caller's arrays, the slab is copied around it
+        const size_t row = ((size_t)prod.seq * v.H + prod.head) * kQBytes;
+        copy_range(prod.i, fresh - prod.i, 0);
+        bulk_g2s(dst + (uint32_t)(fresh - prod.i) * kSlotBytes, p.k_new + row, kQBytes, bar);
+        bulk_g2s(dst + (uint32_t)(fresh - prod.i) * kSlotBytes + kQBytes, p.v_new + row, kQBytes, bar);
+        copy_range(fresh + 1, prod.i + n - fresh - 1, fresh + 1 - prod.i);
       } else {
-        chunk_runs(v, prod.head, prod.i, n, [&](int src, int d, int len) {
-          bulk_g2s(dst + (uint32_t)d * kSlotBytes, hbase + (size_t)src * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
-        });
+        copy_range(prod.i, n, 0);
       }
       if (begin)
         bulk_g2s(dst + kChunk * kSlotBytes, p.q + ((size_t)prod.seq * v.H + prod.head) * kHeadDim, kQBytes, bar);
@@ -527,6 +557,17 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     sink.i0 = cons.i;
     Rows rows;
     load_stage(sb, n, grp, l8, rows);
+    if (p.new_j >= 0) {
+      // fused append: the chunk that carries the newest token also stores it in the slab
+      int fresh, fresh_phys;
+      new_token_slot(v, cons.head, p.new_j, fresh, fresh_phys);
+      const int s_new = fresh - cons.i;
+      if (s_new >= 0 && s_new < n) {
+        uint4* dstrow = const_cast<uint4*>(p.slab) +
+                        ((size_t)cons.seq * v.seq_slots + v.head[cons.head].x + fresh_phys) * kSlotU4;
+        dstrow[lane] = sb[s_new * kSlotU4 + lane];
+      }
+    }
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
     if (prod.g < prod.g_end) issue(stage);

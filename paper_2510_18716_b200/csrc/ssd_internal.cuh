@@ -36,6 +36,10 @@ struct DecodeParams {
                             // ring slots of semantic heads, for the score accumulation; else null
   float2* ml;               // row-buffer mode: [n_seqs * H] final (max, exp-sum) of each head; else null
   int mr;                   // M + R
+  // fused append: the newest token's rows are not in the slab yet (null / -1 when it is)
+  const unsigned char* k_new;  // [n_seqs, H, 128] bf16: K row of image token new_j
+  const unsigned char* v_new;
+  int new_j;                // image index of that token; the view already counts it
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
   LayerView view;           // layout and occupancy of the layer

@@ -212,3 +212,45 @@ def test_other_head_partitions(kind):
             lab = np.stack([rng.permutation(wl.sink_mask(cfg, l)) for l in layers])
         r = run_workload(cfg, layers, seqs, (cfg.n0 + 1, cfg.n0 + 9, cfg.n_img), classify=False, labels_override=lab)
         assert r.steps_checked == 3 * len(layers)
+
+
+@pytest.mark.parametrize("case", ["tiny_compressed", "tiny_ring_from_zero", "janus7b_slice"])
+def test_fused_append_decode_matches_the_two_calls(case):
+    """ssd_append_decode must give the bits of ssd_append + ssd_decode_attn at every step, and leave
+    the same cache behind (later steps read the token that the fused kernel stored)."""
+    dev = torch.device("cuda:0")
+    if case == "janus7b_slice":
+        cfg, seqs, n_steps = wl.CONFIGS["janus7b"], [0, 1, 2, 3, 4], 30
+    else:
+        cfg, seqs, n_steps = wl.CONFIGS["tiny"], [0], 32
+    L, n0 = cfg.prompt_len, cfg.n0
+    q, k, v, _ = wl.gen_layer(cfg, 0, seqs, device=dev)
+    caches = []
+    for _ in range(2):
+        c = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=len(seqs)), device=dev)
+        c.set_head_labels(wl.sink_mask(cfg, 0))
+        if case == "tiny_ring_from_zero":
+            t0 = 0                       # no compress: prompt slots unused, rings fill from empty
+        else:
+            t0 = n0
+            c.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(c)
+    two, fused = caches
+    for t in range(t0 + 1, t0 + n_steps + 1):
+        kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
+        two.append(0, kt, vt)
+        want = two.decode_attn(0, qt)
+        got = fused.append_decode(0, kt, vt, qt)
+        assert torch.equal(got, want), f"step {t}"
+        assert fused.tokens(0) == two.tokens(0) == t
+    assert np.array_equal(fused.get_indices(0), two.get_indices(0))
+    # the fused cache is a full substitute: switch roles for a few more steps
+    for t in range(t0 + n_steps + 1, min(t0 + n_steps + 4, cfg.n_img) + 1):
+        kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
+        fused.append(0, kt, vt)
+        a = fused.decode_attn(0, qt)
+        b = two.append_decode(0, kt, vt, qt)
+        assert torch.equal(a, b), f"step {t} after switching roles"
+    assert fused.device_status() == 0 and two.device_status() == 0
+    for c in caches:
+        c.close()
