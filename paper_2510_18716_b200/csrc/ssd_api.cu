@@ -78,6 +78,10 @@ struct ssd_cache {
   std::vector<int64_t> layer_base;    // [layers] first slot of the layer in the slab
   std::vector<int32_t> n_sink;        // [layers]
   std::vector<int32_t> t_img, n0, prompt_valid, static_valid;  // [layers]
+  // Layer whose slab the library's latest launch may write (append, fused append, compress,
+  // re-selection), -1 if none, -2 if unknown: a decode launch of ANOTHER layer may prefetch its slab
+  // before that launch has completed.
+  int last_writer = -2;
   bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
   std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
   std::vector<uint8_t> pending;       // [layers] last decode's logits not yet added to the scores
@@ -389,6 +393,7 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   c->static_valid[layer] = select ? sv : 0;
   c->t_base[layer] = n0;
   c->pending[layer] = 0;
+  c->last_writer = -2;
   return SSD_OK;
 }
 
@@ -416,6 +421,7 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   p.logits = c->d_logits(layer);
   p.ml = c->d_ml(layer);
   if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  c->last_writer = layer;
   if (c->row_buffer) c->pending[layer] = 0;
   c->t_img[layer] += 1;
   return SSD_OK;
@@ -439,6 +445,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
   p.mr = c->mr();
   p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
+  p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
@@ -446,6 +453,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  c->last_writer = -1;
   if (c->row_buffer) c->pending[layer] = 1;
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
@@ -479,6 +487,7 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   p.k_new = static_cast<const unsigned char*>(k_new);
   p.v_new = static_cast<const unsigned char*>(v_new);
   p.new_j = c->t_img[layer];
+  p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->t_img[layer] += 1;                // the view describes the layer with the token in place
@@ -490,6 +499,7 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
     c->t_img[layer] -= 1;
     return SSD_ERR_CUDA;
   }
+  c->last_writer = layer;
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -636,6 +646,7 @@ int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
   }
   c->t_base[layer] = c->t_img[layer];
   c->pending[layer] = 0;
+  c->last_writer = -2;
   return SSD_OK;
 }
 
@@ -802,10 +813,12 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
   p.mr = c->mr();
   p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
+  p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  c->last_writer = -1;
   if (c->row_buffer) c->pending[layer] = 1;
   return SSD_OK;
 }

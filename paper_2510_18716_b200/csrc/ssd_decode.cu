@@ -131,10 +131,14 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 
 // Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
 // may start while its predecessor in the stream is still running, once the predecessor has allowed
-// it; it must then wait for the predecessor to complete before touching memory.  Both kernels of
-// the decode step allow their successor at once and wait just before their first global access,
-// so launch latency and the index planning overlap with the predecessor's tail.  Every kernel of
-// the chain waits for its predecessor's completion, so stream order is preserved transitively.
+// it; it must then wait for the predecessor to complete before touching memory the predecessor may
+// write, or that anything earlier may have written and not yet flushed.  Both kernels of the decode
+// step wait just before their first such access and allow their successor right after that wait.
+// So launch latency, CTA start-up and the index planning overlap with the predecessor's tail; every
+// kernel of the chain waits for its predecessor's completion, which preserves stream order
+// transitively; and when a kernel starts, everything before its predecessor has completed (the
+// predecessor passed its own wait before allowing it), which is what makes the slab prefetch of the
+// decode kernel's prologue safe.
 __device__ __forceinline__ void pdl_allow_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -374,6 +378,7 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   unsigned heads = __ballot_sync(FULL, r_pair >= 0);
   if (!heads) return;
   pdl_wait_predecessor();                // the scratch below may still be in use by the previous launch
+  pdl_allow_successor();
   for (unsigned h = heads; h; h &= h - 1) {
     const int slot = __ffs(h) - 1;       // 0: began in an earlier CTA, 1: begins here and runs on
     if (!mbar_wait(cta_bar0 + 8 * slot, 0)) {
@@ -412,7 +417,6 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   const LayerView& v = p.view;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = lane >> 3, l8 = lane & 7;
-  pdl_allow_successor();
 
   const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
   const uint32_t cta_bar0 = smem_u32(smem + kRingBytes) + kWarps * kStages * 8;
@@ -470,14 +474,20 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   Walk cons = prod;
   int ahead = 0;   // chunks issued and not yet consumed
 
-  // lane 0 starts the copies of the producer's current chunk into `stage`; every lane advances
-  auto issue = [&](int stage) {
-    const int n = walk_chunk(prod, kChunk);
-    if (lane == 0) {
-      const bool begin = prod.i == 0 || prod.g == g_begin;
-      const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
-      const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
-                                   ((size_t)prod.seq * v.seq_slots + v.head[prod.head].x) * kSlotBytes;
+  // Lane 0 starts copies of the chunk at walk position `w` into `stage`.  what & 1: the slab part
+  // (and the barrier's byte count for the whole chunk); what & 2: the caller's inputs that travel with
+  // the chunk (the head's query row with its first chunk, the newest token's rows in place of its slot).
+  auto copy_chunk = [&](const Walk& w, int stage, int what) {
+    const int n = walk_chunk(w, kChunk);
+    if (lane != 0) return;
+    const bool begin = w.i == 0 || w.g == g_begin;
+    const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
+    const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
+                                 ((size_t)w.seq * v.seq_slots + v.head[w.head].x) * kSlotBytes;
+    int fresh = -1, fresh_phys = 0;
+    if (p.new_j >= 0) new_token_slot(v, w.head, p.new_j, fresh, fresh_phys);
+    const bool has_fresh = fresh >= w.i && fresh < w.i + n;
+    if (what & 1) {
       // order the warp's reads of this stage (made visible to this lane by __syncwarp) before
       // the asynchronous writes that follow
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -488,33 +498,60 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
         if (v.contig) {
           bulk_g2s(dst + (uint32_t)at * kSlotBytes, hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
         } else {
-          chunk_runs(v, prod.head, a, len, [&](int src, int d, int l) {
+          chunk_runs(v, w.head, a, len, [&](int src, int d, int l) {
             bulk_g2s(dst + (uint32_t)(at + d) * kSlotBytes, hbase + (size_t)src * kSlotBytes, (uint32_t)l * kSlotBytes, bar);
           });
         }
       };
-      int fresh = -1, fresh_phys = 0;
-      if (p.new_j >= 0) new_token_slot(v, prod.head, p.new_j, fresh, fresh_phys);
-      if (fresh >= prod.i && fresh < prod.i + n) {
-        // the newest token: its rows come from the caller's arrays, the slab is copied around it
-        const size_t row = ((size_t)prod.seq * v.H + prod.head) * kQBytes;
-        copy_range(prod.i, fresh - prod.i, 0);
-        bulk_g2s(dst + (uint32_t)(fresh - prod.i) * kSlotBytes, p.k_new + row, kQBytes, bar);
-        bulk_g2s(dst + (uint32_t)(fresh - prod.i) * kSlotBytes + kQBytes, p.v_new + row, kQBytes, bar);
-        copy_range(fresh + 1, prod.i + n - fresh - 1, fresh + 1 - prod.i);
+      if (has_fresh) {                   // the slab is copied around the newest token's slot
+        copy_range(w.i, fresh - w.i, 0);
+        copy_range(fresh + 1, w.i + n - fresh - 1, fresh + 1 - w.i);
       } else {
-        copy_range(prod.i, n, 0);
+        copy_range(w.i, n, 0);
       }
-      if (begin)
-        bulk_g2s(dst + kChunk * kSlotBytes, p.q + ((size_t)prod.seq * v.H + prod.head) * kHeadDim, kQBytes, bar);
     }
-    advance(prod, n);
+    if (what & 2) {
+      const size_t row = ((size_t)w.seq * v.H + w.head) * kQBytes;
+      if (has_fresh) {
+        bulk_g2s(dst + (uint32_t)(fresh - w.i) * kSlotBytes, p.k_new + row, kQBytes, bar);
+        bulk_g2s(dst + (uint32_t)(fresh - w.i) * kSlotBytes + kQBytes, p.v_new + row, kQBytes, bar);
+      }
+      if (begin) bulk_g2s(dst + kChunk * kSlotBytes, reinterpret_cast<const unsigned char*>(p.q) + row, kQBytes, bar);
+    }
+  };
+  // the producer's current chunk, whole; every lane advances
+  auto issue = [&](int stage) {
+    copy_chunk(prod, stage, 3);
+    advance(prod, walk_chunk(prod, kChunk));
     ++ahead;
   };
 
-  pdl_wait_predecessor();                // everything above read only the launch parameters
+  // Prologue.  Everything above read only the launch parameters.  The slab holds nothing that the
+  // preceding launch writes when that launch worked on another layer (p.early), so the first
+  // chunks' slab copies may start while it is still running; the caller's inputs (q, new rows) and
+  // every write wait until it has completed.
+  if (!p.early) {
+    pdl_wait_predecessor();
+    pdl_allow_successor();
+  }
+  const Walk prod0 = prod;
+  int n_pro = 0;
 #pragma unroll 1
-  for (int s = 0; s < kStages && prod.g < prod.g_end; ++s) issue(s);
+  for (; n_pro < kStages && prod.g < prod.g_end; ++n_pro) {
+    copy_chunk(prod, n_pro, p.early ? 1 : 3);
+    advance(prod, walk_chunk(prod, kChunk));
+    ++ahead;
+  }
+  if (p.early) {
+    pdl_wait_predecessor();
+    pdl_allow_successor();
+    Walk redo = prod0;
+#pragma unroll 1
+    for (int s = 0; s < n_pro; ++s) {
+      copy_chunk(redo, s, 2);
+      advance(redo, walk_chunk(redo, kChunk));
+    }
+  }
 
   int stage = 0;
   uint32_t parity = 0;
@@ -645,8 +682,8 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
 
 __global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  pdl_allow_successor();
   pdl_wait_predecessor();
+  pdl_allow_successor();
   if (warp >= p.n_seqs * p.H) return;
   const int seq = warp / p.H, head = warp - seq * p.H;
   const HeadDesc d = p.desc[head];

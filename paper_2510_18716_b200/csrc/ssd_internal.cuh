@@ -40,6 +40,7 @@ struct DecodeParams {
   const unsigned char* k_new;  // [n_seqs, H, 128] bf16: K row of image token new_j
   const unsigned char* v_new;
   int new_j;                // image index of that token; the view already counts it
+  int early;                // 1: the launch before this one on the stream does not write this layer's slab
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
   LayerView view;           // layout and occupancy of the layer
