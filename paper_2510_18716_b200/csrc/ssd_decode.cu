@@ -477,6 +477,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   // Lane 0 starts copies of the chunk at walk position `w` into `stage`.  what & 1: the slab part
   // (and the barrier's byte count for the whole chunk); what & 2: the caller's inputs that travel with
   // the chunk (the head's query row with its first chunk, the newest token's rows in place of its slot).
+  int pf_key = -1, pf_fresh = -1, pf_phys = 0;     // producer side: newest token's slot in the current head
   auto copy_chunk = [&](const Walk& w, int stage, int what) {
     const int n = walk_chunk(w, kChunk);
     if (lane != 0) return;
@@ -484,8 +485,11 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
     const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
                                  ((size_t)w.seq * v.seq_slots + v.head[w.head].x) * kSlotBytes;
-    int fresh = -1, fresh_phys = 0;
-    if (p.new_j >= 0) new_token_slot(v, w.head, p.new_j, fresh, fresh_phys);
+    if (p.new_j >= 0 && pf_key != w.seq * v.H + w.head) {      // once per head, not per chunk
+      pf_key = w.seq * v.H + w.head;
+      new_token_slot(v, w.head, p.new_j, pf_fresh, pf_phys);
+    }
+    const int fresh = pf_fresh;
     const bool has_fresh = fresh >= w.i && fresh < w.i + n;
     if (what & 1) {
       // order the warp's reads of this stage (made visible to this lane by __syncwarp) before
@@ -560,6 +564,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   float2 q[8];
   State st;
   LogitSink sink = {nullptr, 0, 0, 0, 0};
+  int fresh = -1, fresh_phys = 0;                   // consumer side: newest token's slot in the current head
 
 #pragma unroll 1
   while (cons.g < cons.g_end) {
@@ -590,14 +595,13 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
       sink.skip = v.prompt_valid;
       sink.ring_from = v.prompt_valid + v.static_valid;
       sink.ring_shift = d.y - v.static_valid;
+      if (p.new_j >= 0) new_token_slot(v, cons.head, p.new_j, fresh, fresh_phys);
     }
     sink.i0 = cons.i;
     Rows rows;
     load_stage(sb, n, grp, l8, rows);
     if (p.new_j >= 0) {
       // fused append: the chunk that carries the newest token also stores it in the slab
-      int fresh, fresh_phys;
-      new_token_slot(v, cons.head, p.new_j, fresh, fresh_phys);
       const int s_new = fresh - cons.i;
       if (s_new >= 0 && s_new < n) {
         uint4* dstrow = const_cast<uint4*>(p.slab) +
