@@ -31,8 +31,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # DRAM bytes (read + written) of one ssd_decode_kernel launch on a janus7b layer, from the ncu capture
 # summarised in profiles/ssd_decode_kernel_janus7b_layer.md.  Reported only while the kernel's sources
 # still hash to what was captured; otherwise `traffic` is null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "bytes_per_launch": 163.20e6,
-                  "sha256": "a2124ff9dcbf2ab96075a4300fc1db22f6ee23de10b80ed01842a813914304cf"}
+DECODE_TRAFFIC = {"workload": "janus7b", "bytes_per_launch": 162.81e6,
+                  "sha256": "7993692ac2b01944ce25df5e056f3d649f2c608c28c8c849ae68ca9f38a765d2"}
 
 
 def decode_traffic(cfg):
