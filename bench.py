@@ -178,7 +178,8 @@ def run_reference(args, cfg):
 
 
 # ----------------------------------------------------------------------------- our arm
-def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0, row_buffer=False):
+def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0, row_buffer=False,
+                classify=True):
     """Create, classify, load and compress every layer; returns the cache and per-layer step inputs."""
     from paper_2510_18716_b200 import binding as B
     from paper_2510_18716_b200 import dist as D
@@ -192,7 +193,9 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
         cache = B.SsdCache(ccfg, n_sink_heads_total=cfg.n_layers * cfg.n_sink_heads, device=device)
         if row_buffer:
             cache.set_row_buffer(True)
-        mine = D.shard_calibration(cfg.n_cal, rank, world)
+        if not classify:
+            cache.set_head_labels(np.stack([wl.sink_mask(cfg, l) for l in range(cfg.n_layers)]))
+        mine = D.shard_calibration(cfg.n_cal, rank, world) if classify else None
         qs, ks = [], []
         for layer in range(cfg.n_layers):
             if mine:
@@ -201,10 +204,11 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
                 ks.append(k)
         qc = torch.stack(qs) if mine else None
         kc = torch.stack(ks) if mine else None
-        labels = D.classify_sharded(cache, qc, kc, cfg.n_cal, N, cfg.tau)
-        want = np.stack([wl.sink_mask(cfg, l) for l in range(cfg.n_layers)])
-        if not np.array_equal(labels, want):
-            raise RuntimeError("classifier did not recover the generator's head split")
+        if classify:
+            labels = D.classify_sharded(cache, qc, kc, cfg.n_cal, N, cfg.tau)
+            want = np.stack([wl.sink_mask(cfg, l) for l in range(cfg.n_layers)])
+            if not np.array_equal(labels, want):
+                raise RuntimeError("classifier did not recover the generator's head split")
         del qc, kc, qs, ks
     steps_in = []
     seqs = list(range(seq_lo, seq_lo + S))
@@ -458,6 +462,50 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Large-batch sweep on the 7B shape (batch x compression ratio x sink-head fraction): one JSON line
+    per point, timed on `--layers` layers (default 6; every layer has the same shape, so the step time
+    scales with the layer count) with the generator's head split installed directly."""
+    import dataclasses
+    from paper_2510_18716_b200 import binding as B
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    B.load()
+    n_layers = args.layers if args.layers > 0 else 6
+    K = min(args.steps, 40)
+    points = []
+    for batch in (32, 64, 128):
+        points.append((batch, 1, 0.0))
+        for ratio in (2, 5, 10):
+            for frac in (0.25, 0.5, 0.75):
+                points.append((batch, ratio, frac))
+    for batch, ratio, frac in points:
+        cfg = dataclasses.replace(wl.sweep(batch, ratio, frac), n_layers=n_layers)
+        full = ratio == 1
+        if full:
+            cfg = dataclasses.replace(cfg, n0=288)
+        S, H = cfg.n_seqs, cfg.n_heads
+        cache, steps_in = build_cache(cfg, device, 0, 0, 1, full_cache=full, t_steps=K + 4, classify=False)
+        out = torch.empty((S, H, 128), dtype=torch.bfloat16, device=device)
+        st = Stepper(cfg, cache, steps_in, out)
+        for _ in range(3):
+            st.step()
+        ms = timed(st.step, K, lambda: None) / K
+        slots = sum(int(cache.get_lengths(l).sum()) for l in range(n_layers)) / n_layers
+        bytes_layer = S * (slots * 512 + H * 2 * 256 + H * 2 * 512)
+        line = {"sweep": cfg.name, "batch": batch, "n_seqs": S, "ratio": ratio, "sink_frac": frac,
+                "window": cfg.window, "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent,
+                "layers_timed": n_layers, "us_per_layer": ms / n_layers * 1e3,
+                "ms_per_step_30_layers": ms / n_layers * 30, "image_tokens_per_s": batch / (ms / n_layers * 30 * 1e-3),
+                "gbs": bytes_layer / (ms / n_layers * 1e-3) / 1e9,
+                "kv_bytes_per_seq_30_layers": cache.kv_bytes_per_seq() // n_layers * 30,
+                "slots_per_head_mean": slots / H, "status": cache.device_status()}
+        print(json.dumps(line), flush=True)
+        cache.close()
+        del cache, steps_in, st
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -469,8 +517,12 @@ def main():
     ap.add_argument("--no-full-cache", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-row-buffer", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="large-batch sweep on the 7B shape: one JSON line per point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.sweep:
+        run_sweep(args)
+        return
     cfg = wl.CONFIGS[args.workload]
     if args.layers > 0:
         import dataclasses
