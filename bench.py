@@ -428,15 +428,15 @@ def run_ours(args, cfg):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        layers = sorted({0, cfg.n_layers - 1})
+        layers = sorted({0, cfg.n_layers // 2, cfg.n_layers - 1})
         data = oracle_sample(cfg, layers, 0, device)
         oracle_time_steps(cfg, data, n0 + 1, 1)
-        n_cpu = 4
+        n_cpu = min(N - n0, 288)
         secs = oracle_time_steps(cfg, data, n0 + 1, n_cpu)
         scale = cfg.n_layers / len(layers)
         cpu_ms = secs / n_cpu * scale * 1e3
         cpu = {"value": cfg.images_per_step / (cpu_ms * 1e-3), "unit": UNIT, "cores": oracle.threads(),
-               "kind": "oracle", "ms_per_step": cpu_ms,
+               "kind": "oracle", "ms_per_step": cpu_ms, "seconds_timed": secs,
                "sample": (f"{n_cpu} decode steps over layers {layers} of {cfg.n_layers}, all {S} sequences x {H} "
                           f"heads; time scaled by {scale:g} (extrapolated)")}
 

@@ -123,3 +123,11 @@ def test_rowbuf_scores_match_oracle_before_reselection():
     cache.recompress(0)
     cache.append(0, x, x)                      # accepted again
     cache.close()
+
+
+def test_per_step_eviction_is_a_row_buffer_of_one():
+    """Algorithm 1 taken literally re-selects at every step; that is the row buffer with R = 1 and a
+    re-selection after each step (the evicted token is dropped after the step's attention)."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], sink_recent=1, name="tiny_r1")
+    _run(cfg, 0, [0], cfg.n0 + 20)
