@@ -160,3 +160,43 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
     assert cache.device_status() == 0, "a decode warp gave up a bounded wait"
     cache.close()
     return res
+
+
+def run_sampled(cfg: wl.Workload, layer: int, sample, steps, device="cuda:0"):
+    """Full launch size on the GPU (all cfg.n_seqs sequences of one layer, the launch configuration the
+    benchmark times); the oracle recomputes only the sampled (sequence, head) pairs one by one: their
+    selected index sets (exact outside the tie band) and their outputs at the given image steps."""
+    dev = torch.device(device)
+    L, N, n0, W, M, R, H, S = (cfg.prompt_len, cfg.n_img, cfg.n0, cfg.window, cfg.sink_budget, cfg.sink_recent,
+                               cfg.n_heads, cfg.n_seqs)
+    labels = wl.sink_mask(cfg, layer)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1), device=device)
+    cache.set_head_labels(labels)
+    q, k, v, _ = wl.gen_layer(cfg, layer, list(range(S)), device=dev)
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+    gi = cache.get_indices(0)
+    n_cand = max(n0 - R, 0)
+    picked = {}
+    for (s, h) in sample:
+        qu, ku, vu = wl.to_u16(q[s, h]), wl.to_u16(k[s, h]), wl.to_u16(v[s, h])
+        sem = np.array([[labels[h]]], np.uint8)
+        gidx = np.full((1, 1, M), -1, np.int32)
+        if labels[h]:
+            st = gi[s, h, L:L + M]
+            gidx[0, 0] = np.where(st >= 0, st - L, -1)
+            sc, oidx, ocnt = oracle.select_batch(qu[None, None, :n0], ku[None, None, : L + n0], sem, L, n0, M, R)
+            check_index_sets(gidx, sc, oidx, ocnt, sem, n_cand, M)
+        picked[(s, h)] = (qu, ku, vu, sem, gidx, (gidx >= 0).sum(-1).astype(np.int32))
+    steps = sorted(steps)
+    for t in range(n0 + 1, steps[-1] + 1):
+        kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
+        if t not in steps:
+            cache.append_decode(0, kt, vt, qt) if t % 2 else cache.append(0, kt, vt)
+            continue
+        out = bf16_to_f64(cache.append_decode(0, kt, vt, qt))
+        for (s, h), (qu, ku, vu, sem, gidx, gcnt) in picked.items():
+            want = oracle.decode_batch(qu[None, None, t - 1], ku[None, None], vu[None, None], sem, gidx, gcnt, L, t, W, M, R)
+            err = np.abs(out[s, h] - want[0, 0])
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (s, h, t, err.max())
+    assert cache.device_status() == 0
+    cache.close()

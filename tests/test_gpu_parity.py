@@ -254,3 +254,26 @@ def test_fused_append_decode_matches_the_two_calls(case):
     assert fused.device_status() == 0 and two.device_status() == 0
     for c in caches:
         c.close()
+
+
+def _sample_pairs(cfg, layer, n, seed):
+    rng = np.random.default_rng(seed)
+    labels = wl.sink_mask(cfg, layer)
+    sem_heads, spa_heads = np.nonzero(labels)[0], np.nonzero(labels == 0)[0]
+    pairs = []
+    for i in range(n):
+        heads = sem_heads if (i % 2 == 0 and len(sem_heads)) else spa_heads
+        pairs.append((int(rng.integers(0, cfg.n_seqs)), int(rng.choice(heads))))
+    return pairs
+
+
+def test_hires7b_full_launch_size_sampled_pairs():
+    cfg = wl.CONFIGS["hires7b"]
+    from parity_util import run_sampled
+    run_sampled(cfg, 7, _sample_pairs(cfg, 7, 6, 1), (cfg.n0 + 1, cfg.n0 + 70))
+
+
+def test_sweep_batch128_full_launch_size_sampled_pairs():
+    cfg = wl.sweep(128, 5, 0.5)
+    from parity_util import run_sampled
+    run_sampled(cfg, 2, _sample_pairs(cfg, 2, 8, 2), (cfg.n0 + 1, cfg.n0 + 26))
