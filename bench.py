@@ -408,8 +408,7 @@ def run_ours(args, cfg):
             i = rstate["i"]
             for layer in range(cfg.n_layers):
                 qq, kk, vv = rsteps[layer]
-                rcache.append(layer, kk[i], vv[i])
-                rcache.decode_attn(layer, qq[i], out)
+                rcache.append_decode(layer, kk[i], vv[i], qq[i], out)
             rstate["i"] += 1
             if rstate["i"] % R == 0:
                 for layer in range(cfg.n_layers):

@@ -14,7 +14,7 @@ from parity_util import BAND, check_outputs
 pytestmark = pytest.mark.gpu
 
 
-def _run(cfg, layer, seqs, t_end):
+def _run(cfg, layer, seqs, t_end, fused=False):
     dev = torch.device("cuda:0")
     L, n0, M, R, W, H, S = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.window, cfg.n_heads, len(seqs)
     labels = wl.sink_mask(cfg, layer)
@@ -46,8 +46,13 @@ def _run(cfg, layer, seqs, t_end):
     # GPU pass first (records outputs, sets and scores), then the oracle replays it
     outs = []
     for t in range(n0 + 1, t_end + 1):
-        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
-        outs.append(cache.decode_attn(0, q[:, :, t - 1].contiguous()).float().cpu().numpy().astype(np.float64))
+        kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
+        if fused and t % 3:              # mostly the single launch, now and then the two calls
+            o = cache.append_decode(0, kt, vt, qt)
+        else:
+            cache.append(0, kt, vt)
+            o = cache.decode_attn(0, qt)
+        outs.append(o.float().cpu().numpy().astype(np.float64))
         if (t - n0) % R == 0:
             cache.recompress(0)
             gi = cache.get_indices(0)
@@ -79,14 +84,16 @@ def _run(cfg, layer, seqs, t_end):
     return n_band[0]
 
 
-def test_rowbuf_tiny_every_step():
+@pytest.mark.parametrize("fused", [False, True])
+def test_rowbuf_tiny_every_step(fused):
     cfg = wl.CONFIGS["tiny"]
-    _run(cfg, 0, [0], cfg.n_img)
+    _run(cfg, 0, [0], cfg.n_img, fused)
 
 
-def test_rowbuf_janus1b_slice():
+@pytest.mark.parametrize("fused", [False, True])
+def test_rowbuf_janus1b_slice(fused):
     cfg = wl.CONFIGS["janus1b"]
-    _run(cfg, 3, [0, 1], cfg.n0 + 3 * cfg.sink_recent + 5)
+    _run(cfg, 3, [0, 1], cfg.n0 + 3 * cfg.sink_recent + 5, fused)
 
 
 def test_rowbuf_scores_match_oracle_before_reselection():
@@ -101,8 +108,12 @@ def test_rowbuf_scores_match_oracle_before_reselection():
     qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
     cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
     for t in range(n0 + 1, n0 + R + 1):
-        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
-        cache.decode_attn(0, q[:, :, t - 1].contiguous())
+        kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
+        if t % 2:
+            cache.append_decode(0, kt, vt, qt)
+        else:
+            cache.append(0, kt, vt)
+            cache.decode_attn(0, qt)
     acc = cache.get_scores(0)
     gi = cache.get_indices(0)
     for h in range(H):
@@ -130,4 +141,4 @@ def test_per_step_eviction_is_a_row_buffer_of_one():
     re-selection after each step (the evicted token is dropped after the step's attention)."""
     import dataclasses
     cfg = dataclasses.replace(wl.CONFIGS["tiny"], sink_recent=1, name="tiny_r1")
-    _run(cfg, 0, [0], cfg.n0 + 20)
+    _run(cfg, 0, [0], cfg.n0 + 20, fused=True)
