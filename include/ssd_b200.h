@@ -81,6 +81,7 @@ int ssd_cache_free(ssd_cache *cache);
  * visual tokens so far); label = s > tau.
  *   q_cal [n_layers, n_cal_seqs, n_heads, n_img, head_dim]   queries of image steps 1..n_img
  *   k_cal [n_layers, n_cal_seqs, n_heads, prompt_len + n_img, head_dim]
+ *     (device, bf16, dense, 16-byte aligned: read by the TMA unit; SSD_ERR_INVALID_ARG otherwise)
  *   s_out_host      [n_layers * n_heads] float  (may be NULL)
  *   labels_out_host [n_layers * n_heads] uint8, 1 = semantic (may be NULL)
  * Installs the labels in the cache (fixing the per-head layout) and SYNCHRONISES the stream.
@@ -103,6 +104,7 @@ int ssd_set_head_labels(ssd_cache *cache, const uint8_t *labels_host);
  * compress it (Algorithm 1; Algorithm 2's prefill split when n0 == 0).
  *   q_obs  [n_seqs, n_heads, n_obs, head_dim]  queries of image steps n0-n_obs+1 .. n0
  *   k_full, v_full [n_seqs, n_heads, prompt_len + n0, head_dim]
+ *     (device, bf16, dense, 16-byte aligned; SSD_ERR_INVALID_ARG otherwise)
  * Semantic heads: score[j] = sum over the observed steps of the post-softmax attention on image
  * token j (causal, softmax over prompt + image tokens); keep the min(M, n0-R) best-scoring
  * tokens among j in [0, n0-R) (ties: lowest j), stored in ascending j, plus the R newest tokens.

@@ -282,6 +282,7 @@ int ssd_set_head_labels(ssd_cache* c, const uint8_t* labels_host) {
 int ssd_classify_partial(ssd_cache* c, const void* q_cal, const void* k_cal, int32_t n_cal_seqs, int32_t n_img,
                          double* ratio_sums_host, void* stream) {
   if (!c || !q_cal || !k_cal || !ratio_sums_host) return SSD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q_cal) | reinterpret_cast<uintptr_t>(k_cal)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (n_cal_seqs < 1 || n_img < 1 || n_img > g.max_image_tokens) return SSD_ERR_INVALID_ARG;
   const int rpb = classify_rows_per_block();
@@ -340,6 +341,8 @@ int ssd_classify_heads(ssd_cache* c, const void* q_cal, const void* k_cal, int32
 int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_full, const void* v_full, int32_t n0,
                  int32_t n_obs, void* stream) {
   if (!c || !k_full || !v_full) return SSD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q_obs) | reinterpret_cast<uintptr_t>(k_full) | reinterpret_cast<uintptr_t>(v_full)) % 16 != 0)
+    return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (n0 < 0 || n0 > g.max_image_tokens || n_obs < 0 || n_obs > n0) return SSD_ERR_INVALID_ARG;

@@ -1,8 +1,7 @@
 // The dense contraction of the method on the 5th-generation tensor cores: logit tiles
 //   S[128 query rows, 128 keys] = Q_tile K_tile^T   (bf16 x bf16 -> fp32, head dimension 128)
 // computed by tcgen05.mma with both operands in shared memory and the accumulator in tensor
-// memory (TMEM), and consumed in place: every thread owns one query row (one TMEM lane) and reads
-// its 128 logits with tcgen05.ld, so the softmax statistics of a row need no cross-thread step.
+// memory (TMEM), and consumed in place with tcgen05.ld.
 //
 // Used by the head classifier (Sec. 3.3 sparsity metric): per image step t, the attention mass on
 // visual tokens older than the newest w, over the mass on all visual tokens so far.  Only visual
@@ -10,29 +9,46 @@
 // Used by the sink scoring of ssd_compress (Algorithm 1, AttentionScores and running sum): per
 // block of 128 observed queries, a first sweep over the key tiles gives every row its maximum and
 // exp-sum, a second sweep recomputes the tiles, normalises, and adds the columns up.  The sum over
-// the 32 rows of a warp is a shuffle transpose-reduction; each warp keeps its own score array in
-// shared memory and the four are added in a fixed order at the end, so scores are bitwise
-// reproducible from run to run, which the selection relies on.
+// the 32 rows of a warp is a shuffle transpose-reduction; each TMEM lane quadrant keeps its own
+// score array in shared memory and the four are added in a fixed order at the end, so scores are
+// bitwise reproducible from run to run, which the selection relies on.
 //
-// Operand tiles sit in shared memory in the K-major layout without swizzling: 8 rows x 16 bytes
-// form a contiguous 128-byte core matrix, core matrices follow each other along the head
-// dimension (128 bytes apart) and groups of 8 rows follow each other 2048 bytes apart.  Tiles are
-// written with 16-byte cp.async (zero fill past the end of the tensor).  One CTA = one block of
-// 128 query rows of one (layer, sequence, head); several CTAs per SM overlap each other's loads,
-// MMAs and exponentials.  Every mbarrier wait is bounded and failures end in the status word.
+// A CTA is a pipeline of three roles that meet only at mbarriers:
+//   warp 0, one lane   producer: TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the query tile
+//                      of a row block and the key tiles, the latter into a ring of kStages buffers;
+//   warp 1, one lane   issues the 8 tcgen05.mma of a tile into one of kAccs TMEM accumulators and
+//                      commits them to the barriers that free the key stage and publish the tile;
+//   warps 2..9         read the accumulator (tcgen05.ld), hand it back as soon as it is in registers
+//                      and do the exponentials.  A query row (one TMEM lane) belongs to two threads,
+//                      one per half of the tile's columns; the halves of a row's softmax statistics
+//                      meet through shared memory.
+// so the loads and the MMAs of tile k+1 run under the exponentials of tile k.  Two CTAs share an SM
+// (2 x 96 KB of tiles, 2 x 256 TMEM columns).  Operand tiles are two TMA boxes of 128 rows x 64
+// elements in the K-major 128-byte-swizzled layout (8-row groups 1024 bytes apart); rows past the
+// end of a tensor are zero-filled by the TMA unit.  Every mbarrier wait is bounded: a wait that
+// runs out raises the CTA's abort flag, after which no role waits any more, all of them run to the
+// end of their loops, the CTA reports through the status word and frees its tensor memory.
+#include <cuda.h>
+
 #include "ssd_internal.cuh"
 
 namespace ssd {
 
 namespace {
 
-constexpr int kRows = 128;                 // query rows per CTA = TMEM lanes = threads
+constexpr int kRows = 128;                 // query rows per block = TMEM lanes
 constexpr int kKeys = 128;                 // keys per tile = TMEM columns of one accumulator
-constexpr int kTileBytes = 128 * kHeadDim * 2;   // 32 KB per operand tile
-constexpr int kLbo = 128;                  // bytes between core matrices along the head dimension
-constexpr int kSbo = 2048;                 // bytes between groups of 8 rows
+constexpr int kBoxBytes = 128 * 64 * 2;    // one TMA box: 128 rows x 64 bf16
+constexpr int kTileBytes = 2 * kBoxBytes;  // 32 KB per operand tile (two boxes along the head dimension)
+constexpr int kStages = 2;                 // key tiles in flight
+constexpr int kAccs = 2;                   // TMEM accumulators
+constexpr int kEpiWarps = 8;
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kTcThreads = 64 + kEpiThreads;
+constexpr int kTmemCols = kAccs * kKeys;   // 256: a power of two, as the allocator wants
 constexpr float kNegBig = -1.0e30f;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+static_assert(kHeadDim == 128, "two 64-element boxes per tile row");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -43,9 +59,15 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// ---- mbarrier with a bounded wait
+// ---- mbarriers; every wait is bounded and gives up at once when the CTA's abort flag is up
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -65,56 +87,87 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  bool ok = mbar_try_wait(bar, parity);
-  if (!ok) {
-    const unsigned long long t0 = global_ns();
-    do {
+__device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+  if (*abort) return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
 #pragma unroll 1
-      for (int i = 0; i < 64 && !ok; ++i) ok = mbar_try_wait(bar, parity);
-    } while (!ok && global_ns() - t0 < kWaitLimitNs);
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort = 1;
+      return false;
+    }
   }
-  return ok;
+}
+
+// The barriers of a CTA's pipeline, one after another in shared memory; `base` is the address of the first.
+struct PipeBars {
+  uint64_t b[2 + 2 * kStages + 2 * kAccs];
+};
+struct Pipe {
+  uint32_t base;
+  __device__ __forceinline__ uint32_t q_full() const { return base; }
+  __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
+  __device__ __forceinline__ uint32_t full(int s) const { return base + 16 + 8 * s; }
+  __device__ __forceinline__ uint32_t empty(int s) const { return base + 16 + 8 * (kStages + s); }
+  __device__ __forceinline__ uint32_t acc_full(int a) const { return base + 16 + 8 * (2 * kStages + a); }
+  __device__ __forceinline__ uint32_t acc_empty(int a) const { return base + 16 + 8 * (2 * kStages + kAccs + a); }
+};
+__device__ __forceinline__ Pipe pipe_make(PipeBars& bars, bool init) {
+  Pipe p;
+  p.base = smem_u32(&bars.b[0]);
+  if (init) {
+    mbar_init(p.q_full(), 1);
+    mbar_init(p.q_empty(), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(p.full(s), 1);
+      mbar_init(p.empty(s), 1);
+    }
+    for (int a = 0; a < kAccs; ++a) {
+      mbar_init(p.acc_full(a), 1);
+      mbar_init(p.acc_empty(a), kEpiWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  return p;
 }
 
 // ---- operand tiles
-// Copy rows [row0, row0 + 128) of a row-major [n_rows, 128] bf16 matrix into a tile (zero rows past
-// n_rows).  A warp moves 8 rows x 64 bytes per step: full 32-byte sectors on the global side,
-// conflict-free 128-byte runs on the shared side.
-__device__ __forceinline__ void load_tile(uint32_t tile_s, const __nv_bfloat16* __restrict__ src, int row0, int n_rows,
-                                          int warp, int lane, int n_warps) {
-  const int r8 = lane & 7, c4 = lane >> 3;
-  for (int it = warp; it < 16 * 4; it += n_warps) {
-    const int rg = it >> 2, cg = it & 3;          // group of 8 rows, group of 4 chunks
-    const int r = rg * 8 + r8, c = cg * 4 + c4;   // row in tile, 16-byte chunk in row
-    const int grow = row0 + r;
-    const bool in = grow < n_rows;
-    const __nv_bfloat16* g = src + (size_t)(in ? grow : 0) * kHeadDim + c * 8;
-    const uint32_t dst = tile_s + (uint32_t)(rg * kSbo + c * kLbo + r8 * 16);
-    const int bytes = in ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(g), "r"(bytes) : "memory");
-  }
+// One box of a tile: rows [y, y + 128) x elements [x, x + 64) of unit z of a [units, rows, 128] bf16
+// tensor.  x is 0 or 64 (128 bytes), so the copy starts on the boundary the TMA unit wants.
+__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
 }
-__device__ __forceinline__ void tiles_ready_for_mma() {
-  asm volatile("cp.async.wait_all;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> tensor-core reads
+__device__ __forceinline__ void tma_tile(uint32_t dst, const CUtensorMap* map, int row0, int unit, uint32_t bar) {
+  mbar_expect_tx(bar, kTileBytes);
+  tma_box(dst, map, 0, row0, unit, bar);
+  tma_box(dst + kBoxBytes, map, 64, row0, unit, bar);
 }
 
-// Shared-memory matrix descriptor of a K-major, unswizzled operand starting at byte address `addr`.
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte-swizzled layout starting at
+// byte address `addr`: groups of 8 rows 1024 bytes apart, descriptor version 1.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  const uint32_t lo = ((addr >> 4) & 0x3fffu) | ((uint32_t)(kLbo >> 4) << 16);
-  const uint32_t hi = (uint32_t)(kSbo >> 4) | (1u << 14);        // descriptor version 1, no swizzle
+  const uint32_t lo = ((addr >> 4) & 0x3fffu) | (1u << 16);
+  const uint32_t hi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
   return ((uint64_t)hi << 32) | lo;
 }
 // Instruction descriptor: D = fp32, A = B = bf16, both K-major, N = 128, M = 128.
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kKeys >> 3) << 17) |
                                 ((uint32_t)(kRows >> 4) << 24);
 
-// One thread: S[128 x 128] (TMEM columns [tmem_d, tmem_d + 128)) = A_tile B_tile^T, then signal `bar`.
-__device__ __forceinline__ void mma_tile(uint32_t tmem_d, uint32_t a_s, uint32_t b_s, uint32_t bar) {
+// One thread: S[128 x 128] (TMEM columns [tmem_d, tmem_d + 128)) = A_tile B_tile^T.  A step of 16
+// elements along the head dimension is 32 bytes inside a swizzled row; the second box follows the first.
+__device__ __forceinline__ void mma_tile(uint32_t tmem_d, uint32_t a_s, uint32_t b_s) {
 #pragma unroll
   for (int k = 0; k < kHeadDim / 16; ++k) {
-    const uint64_t da = smem_desc(a_s + k * 2 * kLbo), db = smem_desc(b_s + k * 2 * kLbo);
+    const uint32_t off = (uint32_t)((k >> 2) * kBoxBytes + (k & 3) * 32);
+    const uint64_t da = smem_desc(a_s + off), db = smem_desc(b_s + off);
     const uint32_t accumulate = k > 0 ? 1u : 0u;
     asm volatile(
         "{\n"
@@ -124,6 +177,9 @@ __device__ __forceinline__ void mma_tile(uint32_t tmem_d, uint32_t a_s, uint32_t
         "}\n" ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc), "r"(accumulate)
         : "memory");
   }
+}
+// The barrier gets one arrival when every tcgen05.mma this thread has issued so far is complete.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
@@ -145,113 +201,245 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
 }
 
-// Running softmax statistics of one row over the visual keys: exp-sum over all visible keys and over
-// the "far" ones (older than the newest w), both relative to the running maximum m (base-2 units).
+// ---- the three roles.  Each keeps its own count of tiles (t) and query blocks (qn); stage, accumulator
+// and barrier phase follow from the counts, so the roles agree as long as they walk the same schedule.
+struct Producer {
+  Pipe p;
+  volatile int* abort;
+  uint32_t q_s, k_s;
+  const CUtensorMap *tq, *tk;
+  int t = 0, qn = 0;
+  int q_last = -1, k_last = -1;       // counts of the last copies actually issued (-1: none)
+  __device__ __forceinline__ void query_block(int row0, int unit) {
+    pipe_wait(p.q_empty(), ((qn & 1) ^ 1), abort);        // the MMAs of the previous block are done with it
+    if (!*abort) {
+      tma_tile(q_s, tq, row0, unit, p.q_full());
+      q_last = qn;
+    }
+    ++qn;
+  }
+  __device__ __forceinline__ void key_tile(int row0, int unit) {
+    const int s = t % kStages;
+    pipe_wait(p.empty(s), ((t / kStages) & 1) ^ 1, abort);
+    if (!*abort) {
+      tma_tile(k_s + s * kTileBytes, tk, row0, unit, p.full(s));
+      k_last = t;
+    }
+    ++t;
+  }
+  // After an abort: give the copies still in flight their time to land before the CTA ends.
+  __device__ __forceinline__ void drain() {
+    if (!*abort) return;
+    const unsigned long long t0 = global_ns();
+    bool done = false;
+    while (!done && global_ns() - t0 < kWaitLimitNs) {
+      done = q_last < 0 || mbar_try_wait(p.q_full(), q_last & 1);
+      for (int d = 0; d < kStages; ++d) {
+        const int tt = k_last - d;     // the stages hold the last kStages tiles issued
+        if (tt >= 0) done = mbar_try_wait(p.full(tt % kStages), (tt / kStages) & 1) && done;
+      }
+    }
+  }
+};
+
+struct Issuer {
+  Pipe p;
+  volatile int* abort;
+  uint32_t q_s, k_s, tmem;
+  int t = 0, qn = 0;
+  __device__ __forceinline__ void query_block() { pipe_wait(p.q_full(), qn & 1, abort); }
+  __device__ __forceinline__ void key_tile() {
+    const int s = t % kStages, a = t % kAccs;
+    pipe_wait(p.full(s), (t / kStages) & 1, abort);
+    pipe_wait(p.acc_empty(a), ((t / kAccs) & 1) ^ 1, abort);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (!*abort) {
+      mma_tile(tmem + a * kKeys, q_s, k_s + s * kTileBytes);
+      mma_commit(p.empty(s));
+      mma_commit(p.acc_full(a));
+    }
+    ++t;
+  }
+  __device__ __forceinline__ void end_block() {
+    if (!*abort) mma_commit(p.q_empty());
+    ++qn;
+  }
+};
+
+struct Consumer {
+  Pipe p;
+  volatile int* abort;
+  uint32_t tmem_lane;        // TMEM address of this warp's lane quadrant, column 0
+  int lane;
+  int t = 0;
+  // waits for the tile; returns the TMEM address of this warp's lanes of its accumulator
+  __device__ __forceinline__ uint32_t tile() {
+    const int a = t % kAccs;
+    pipe_wait(p.acc_full(a), (t / kAccs) & 1, abort);
+    __syncwarp();              // the lanes left the wait one by one; tcgen05.ld wants them together
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    return tmem_lane + a * kKeys;
+  }
+  // this warp has read all it wants from the tile's accumulator
+  __device__ __forceinline__ void release() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) mbar_arrive(p.acc_empty(t % kAccs));
+    ++t;
+  }
+};
+
+// ---- softmax statistics
+// Running statistics of one row over its column half: exp-sum over all visible keys and over the
+// "far" ones (older than the newest w), both relative to the running maximum m (base-2 units).
 struct RowStats {
   float m, all, far;
 };
 
-// Fold 32 logits (raw dot products; x = v * scale) of keys base .. base + 31 into the statistics of
-// the row whose newest visible key is `row` and whose newest far key is `row - w`.
-__device__ __forceinline__ void fold32(RowStats& st, const float (&v)[32], int base, int row, int w, float scale) {
-  const int nv = min(max(row - base + 1, 0), 32);          // visible: first nv
-  const int nf = min(max(row - w - base + 1, 0), 32);      // far: first nf
-  if (nv == 0) return;
+// Fold 32 logits (raw dot products; x = v * scale) into the statistics of a row that sees the first
+// nv of them, the first nf of which are far.  Without kMasked the row sees all 32 and they are
+// either all far or none (all_far); without kFar the far sum is not kept.
+template <bool kMasked, bool kFar>
+__device__ __forceinline__ void fold32(RowStats& st, const float (&v)[32], int nv, int nf, bool all_far, float scale) {
+  if (kMasked && nv <= 0) return;
   float gmax = kNegBig;
 #pragma unroll
-  for (int j = 0; j < 32; ++j) gmax = fmaxf(gmax, j < nv ? v[j] : kNegBig);
+  for (int j = 0; j < 32; ++j) gmax = fmaxf(gmax, (!kMasked || j < nv) ? v[j] : kNegBig);
   const float mn = fmaxf(st.m, gmax * scale);
   const float corr = ex2(st.m - mn);
   float sa = 0.f, sf = 0.f;
 #pragma unroll
   for (int j = 0; j < 32; ++j) {
-    const float e = j < nv ? ex2(fmaf(v[j], scale, -mn)) : 0.f;
+    const float e = (!kMasked || j < nv) ? ex2(fmaf(v[j], scale, -mn)) : 0.f;
     sa += e;
-    sf += j < nf ? e : 0.f;
+    if (kMasked && kFar) sf += j < nf ? e : 0.f;
   }
+  if (!kMasked && kFar) sf = all_far ? sa : 0.f;
   st.all = st.all * corr + sa;
-  st.far = st.far * corr + sf;
+  if (kFar) st.far = st.far * corr + sf;
   st.m = mn;
 }
 
-// ----------------------------------------------------------------------------- classify
-// One CTA per (unit, block of 128 image steps), unit = (layer, calibration sequence, head).
-__global__ void __launch_bounds__(kRows) ssd_classify_kernel(const ClassifyParams p, int n_row_blocks) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  __shared__ uint64_t s_bar;
-  __shared__ uint32_t s_tmem;
-  __shared__ float s_ratio[4];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int unit = blockIdx.x / n_row_blocks, rb = blockIdx.x - unit * n_row_blocks;
-  const __nv_bfloat16* Q = p.q_cal + (size_t)unit * p.N * kHeadDim;
-  const __nv_bfloat16* K = p.k_cal + ((size_t)unit * (p.L + p.N) + p.L) * kHeadDim;   // visual keys
-  const int r0 = rb * kRows;
-  const int row = r0 + tid;                 // image index of this thread's query; step t = row + 1
-  const int last_row = min(r0 + kRows, p.N) - 1;
+__device__ __forceinline__ int clamp32(int x) { return min(max(x, 0), 32); }
 
-  const uint32_t q_s = smem_u32(smem), k_s = q_s + kTileBytes;
-  const uint32_t bar = smem_u32(&s_bar);
+// What every CTA does first: barriers, abort flag, tensor memory.  Returns the 1024-byte aligned
+// shared-memory address of the tiles (query tile, then the key stages).
+__device__ __forceinline__ uint32_t cta_setup(unsigned char* smem, PipeBars& bars, uint32_t* s_tmem, int* s_abort, Pipe& pipe) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) *s_abort = 0;
+  pipe = pipe_make(bars, tid == 0);
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kKeys)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid == 0) {
-    mbar_init(bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  load_tile(q_s, Q, r0, p.N, warp, lane, 4);
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem = s_tmem;
-  const uint32_t my_tmem = tmem + ((uint32_t)(warp * 32) << 16);
-
-  RowStats st = {kNegBig, 0.f, 0.f};
-  uint32_t parity = 0;
-  bool ok = true;
-  for (int k0 = 0; k0 <= last_row; k0 += kKeys) {
-    load_tile(k_s, K, k0, p.N, warp, lane, 4);
-    tiles_ready_for_mma();
-    __syncthreads();
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      mma_tile(tmem, q_s, k_s, bar);
-    }
-    ok = mbar_wait(bar, parity);
-    parity ^= 1u;
+  return (smem_u32(smem) + 1023u) & ~1023u;
+}
+__device__ __forceinline__ void cta_teardown(uint32_t tmem) {
+  if (threadIdx.x < 32) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (__all_sync(0xffffffffu, ok)) {
-      const int warp_last = min(r0 + warp * 32 + 31, last_row);
-#pragma unroll 1
-      for (int cb = 0; cb < kKeys / 32; ++cb) {
-        const int base = k0 + cb * 32;
-        if (base > warp_last) break;          // no row of this warp sees these keys
-        float v[32];
-        tmem_ld32(my_tmem + cb * 32, v);
-        if (row < p.N) fold32(st, v, base, row, p.w, p.scale_log2);
-      }
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------- classify
+// One CTA = one block of 128 query rows of one unit (layer, calibration sequence, head); its key
+// tiles are those up to the diagonal.  Blocks of a unit are launched longest first.
+__global__ void __launch_bounds__(kTcThreads, 2)
+ssd_classify_kernel(const ClassifyParams p, int n_row_blocks, const __grid_constant__ CUtensorMap tq,
+                    const __grid_constant__ CUtensorMap tk) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ PipeBars s_bars;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ float s_ratio[4];
+  __shared__ float s_half[3][kRows];        // statistics of the rows' upper column halves
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int unit = blockIdx.x / n_row_blocks;
+  const int rb = n_row_blocks - 1 - (blockIdx.x - unit * n_row_blocks);
+  const int r0 = rb * kRows;
+  const int last_row = min(r0 + kRows, p.N) - 1;
+  const int n_tiles = last_row / kKeys + 1;   // keys 0 .. last_row
+
+  Pipe pipe;
+  const uint32_t q_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe), k_s = q_s + kTileBytes;
+  const uint32_t tmem = s_tmem;
+
+  const int quad = warp & 3, half = (warp - 2) >> 2;   // TMEM lane quadrant; which half of a tile's columns
+  const int rl = quad * 32 + lane;                     // row inside the block
+  const int row = r0 + rl;                             // image index of this thread's query; step t = row + 1
+  RowStats st = {kNegBig, 0.f, 0.f};
+
+  if (warp == 0) {
+    if (lane == 0) {
+      Producer pr;
+      pr.p = pipe; pr.abort = &s_abort; pr.q_s = q_s; pr.k_s = k_s; pr.tq = &tq; pr.tk = &tk;
+      pr.query_block(r0, unit);
+      for (int ti = 0; ti < n_tiles; ++ti) pr.key_tile(p.L + ti * kKeys, unit);   // visual keys only
+      pr.drain();
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    // everyone is done with the key tile and the accumulator; a CTA-wide verdict on the wait
-    if (!__syncthreads_and(ok ? 1 : 0)) {
-      ok = false;
-      break;
+  } else if (warp == 1) {
+    if (lane == 0) {
+      Issuer is;
+      is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem;
+      is.query_block();
+      for (int ti = 0; ti < n_tiles; ++ti) is.key_tile();
+      is.end_block();
+    }
+  } else {
+    Consumer co;
+    co.p = pipe; co.abort = &s_abort; co.tmem_lane = tmem + ((uint32_t)(quad * 32) << 16); co.lane = lane;
+    const int lo_row = r0 + quad * 32;                  // this warp's rows: lo_row .. lo_row + 31
+    const int warp_last = min(lo_row + 31, last_row);
+    for (int ti = 0; ti < n_tiles; ++ti) {
+      const uint32_t acc = co.tile();
+      bool released = false;
+#pragma unroll 1
+      for (int cb = 2 * half; cb < 2 * half + 2; ++cb) {
+        const int base = ti * kKeys + cb * 32;
+        if (base > warp_last || lo_row > last_row) break;   // no row of this warp sees these keys
+        float v[32];
+        tmem_ld32(acc + cb * 32, v);
+        if (cb == 2 * half + 1) {
+          co.release();
+          released = true;
+        }
+        const bool all_far = base + 31 <= lo_row - p.w, none_far = base > lo_row + 31 - p.w;
+        if (base + 31 <= lo_row && (all_far || none_far)) {
+          fold32<false, true>(st, v, 32, 0, all_far, p.scale_log2);
+        } else if (row < p.N) {
+          fold32<true, true>(st, v, clamp32(row - base + 1), clamp32(row - p.w - base + 1), false, p.scale_log2);
+        }
+      }
+      if (!released) co.release();
+    }
+    if (half == 1) {
+      s_half[0][rl] = st.m;
+      s_half[1][rl] = st.all;
+      s_half[2][rl] = st.far;
     }
   }
-
-  float ratio = (ok && row < p.N && st.all > 0.f) ? st.far / st.all : 0.f;
+  __syncthreads();
+  const bool ok = s_abort == 0;
+  if (warp >= 2 && half == 0) {
+    // the two halves of every row meet
+    const float m2 = s_half[0][rl], mn = fmaxf(st.m, m2);
+    const float c1 = ex2(st.m - mn), c2 = ex2(m2 - mn);
+    const float all = st.all * c1 + s_half[1][rl] * c2, far = st.far * c1 + s_half[2][rl] * c2;
+    float ratio = (ok && row < p.N && all > 0.f) ? far / all : 0.f;
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) ratio += __shfl_xor_sync(0xffffffffu, ratio, o);
-  if (lane == 0) s_ratio[warp] = ratio;
+    for (int o = 16; o >= 1; o >>= 1) ratio += __shfl_xor_sync(0xffffffffu, ratio, o);
+    if (lane == 0) s_ratio[quad] = ratio;
+  }
   __syncthreads();
   if (tid == 0) {
     p.ratio_part[(size_t)unit * n_row_blocks + rb] = (s_ratio[0] + s_ratio[1]) + (s_ratio[2] + s_ratio[3]);
     if (!ok) atomicOr(p.status, 2u);
   }
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kKeys) : "memory");
-  }
+  cta_teardown(tmem);
 }
 
 // ----------------------------------------------------------------------------- score
@@ -270,119 +458,191 @@ __device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
   return a[0];
 }
 
+// The tiles of a scoring CTA, in the order all three roles walk them: for every block of 128
+// observed queries, the key tiles of sweep 1 (from key 0) and then of sweep 2 (from the tile that
+// holds the first image key), both up to the context of the block's last row.
+struct ScoreBlock {
+  int r0, last, ctx_max, k_first2;
+};
+__device__ __forceinline__ ScoreBlock score_block(const ScoreParams& p, int r0) {
+  ScoreBlock b;
+  b.r0 = r0;
+  b.last = min(r0 + kRows, p.n_obs) - 1;
+  b.ctx_max = p.L + (p.n0 - p.n_obs + 1) + b.last;   // keys [0, ctx_max) are visible to the block's last row
+  b.k_first2 = (p.L / kKeys) * kKeys;
+  return b;
+}
+
 // One CTA per (sequence, semantic head); loops over blocks of 128 observed queries.
-__global__ void __launch_bounds__(kRows) ssd_score_kernel(const ScoreParams p) {
+__global__ void __launch_bounds__(kTcThreads, 2)
+ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, const __grid_constant__ CUtensorMap tk) {
   extern __shared__ __align__(1024) unsigned char smem[];
-  __shared__ uint64_t s_bar;
+  __shared__ PipeBars s_bars;
   __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ float s_half[2][2][2][kRows];   // [block parity][column half][m, exp-sum][row]: sweep-1 statistics
   const int pair = blockIdx.x;
   const int head = pair % p.H;
   if (!p.desc[head].w) return;            // before any tensor-memory allocation
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int ctx_all = p.L + p.n0;
-  const __nv_bfloat16* Q = p.q_obs + (size_t)pair * p.n_obs * kHeadDim;
-  const __nv_bfloat16* K = p.k_full + (size_t)pair * ctx_all * kHeadDim;
   const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
 
-  const uint32_t q_s = smem_u32(smem), k_s = q_s + kTileBytes;
-  float* s_score = reinterpret_cast<float*>(smem + 2 * kTileBytes);   // [4 warps][n0]
-  const uint32_t bar = smem_u32(&s_bar);
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kKeys)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (tid == 0) {
-    mbar_init(bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  for (int j = tid; j < 4 * p.n0; j += kRows) s_score[j] = 0.f;
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  Pipe pipe;
+  const uint32_t q_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe), k_s = q_s + kTileBytes;
   const uint32_t tmem = s_tmem;
-  const uint32_t my_tmem = tmem + ((uint32_t)(warp * 32) << 16);
-  float* my_score = s_score + (size_t)warp * p.n0;
+  // [4 lane quadrants][n0], behind the tiles
+  float* s_score = reinterpret_cast<float*>(smem + (q_s - smem_u32(smem)) + (1 + kStages) * kTileBytes);
 
-  uint32_t parity = 0;
-  bool ok = true;
-  // S tile of keys [k0, k0 + 128) for the current query block; false if the wait ran out
-  auto logits_tile = [&](int k0) -> bool {
-    load_tile(k_s, K, k0, ctx_all, warp, lane, 4);
-    tiles_ready_for_mma();
-    __syncthreads();
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      mma_tile(tmem, q_s, k_s, bar);
+  if (warp == 0) {
+    if (lane == 0) {
+      Producer pr;
+      pr.p = pipe; pr.abort = &s_abort; pr.q_s = q_s; pr.k_s = k_s; pr.tq = &tq; pr.tk = &tk;
+      for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
+        const ScoreBlock b = score_block(p, r0);
+        pr.query_block(r0, pair);
+        for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) pr.key_tile(k0, pair);
+        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) pr.key_tile(k0, pair);
+      }
+      pr.drain();
     }
-    const bool done = mbar_wait(bar, parity);
-    parity ^= 1u;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    return __all_sync(0xffffffffu, done);
-  };
-  // everyone is done with the key tile and the accumulator; a CTA-wide verdict on the wait
-  auto tile_done = [&](bool fine) -> bool {
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    return __syncthreads_and(fine ? 1 : 0) != 0;
-  };
+  } else if (warp == 1) {
+    if (lane == 0) {
+      Issuer is;
+      is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem;
+      for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
+        const ScoreBlock b = score_block(p, r0);
+        is.query_block();
+        for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
+        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
+        is.end_block();
+      }
+    }
+  } else {
+    const int quad = warp & 3, half = (warp - 2) >> 2;   // TMEM lane quadrant; which half of a tile's columns
+    const int rl = quad * 32 + lane;                     // row inside a block of queries
+    Consumer co;
+    co.p = pipe; co.abort = &s_abort; co.tmem_lane = tmem + ((uint32_t)(quad * 32) << 16); co.lane = lane;
+    float* my_score = s_score + (size_t)quad * p.n0;     // the two warps of a quadrant write disjoint keys
+    for (int j = tid - 64; j < 4 * p.n0; j += kEpiThreads) s_score[j] = 0.f;   // ordered before its use by the barrier below
 
-  for (int r0 = 0; r0 < p.n_obs && ok; r0 += kRows) {
-    load_tile(q_s, Q, r0, p.n_obs, warp, lane, 4);
-    const int row = r0 + tid;
-    const int ctx_r = row < p.n_obs ? p.L + t_first + row : 0;        // keys [0, ctx_r) are visible
-    const int last = min(r0 + kRows, p.n_obs) - 1;
-    const int ctx_max = p.L + t_first + last;                        // context of the block's last row
-    const int warp_ctx = p.L + t_first + min(r0 + warp * 32 + 31, last);
+    int blk = 0;
+    for (int r0 = 0; r0 < p.n_obs; r0 += kRows, ++blk) {
+      const ScoreBlock b = score_block(p, r0);
+      const int row = r0 + rl;
+      const int ctx_r = row < p.n_obs ? p.L + t_first + row : 0;          // keys [0, ctx_r) are visible
+      const int lo_row = r0 + quad * 32;
+      const bool warp_full = lo_row + 31 <= b.last;                       // all 32 rows of the warp exist
+      const int lo_ctx = p.L + t_first + lo_row;                          // context of the warp's first row
+      const int warp_ctx = p.L + t_first + min(lo_row + 31, b.last);      // and of its last
 
-    // sweep 1: row maximum and exp-sum
-    RowStats st = {kNegBig, 0.f, 0.f};
-    for (int k0 = 0; k0 < ctx_max && ok; k0 += kKeys) {
-      const bool fine = logits_tile(k0);
-      if (fine) {
+      // sweep 1: row maximum and exp-sum
+      RowStats st = {kNegBig, 0.f, 0.f};
+      for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) {
+        const uint32_t acc = co.tile();
+        bool released = false;
 #pragma unroll 1
-        for (int cb = 0; cb < kKeys / 32; ++cb) {
+        for (int cb = 2 * half; cb < 2 * half + 2; ++cb) {
           const int base = k0 + cb * 32;
           if (base >= warp_ctx) break;
           float v[32];
-          tmem_ld32(my_tmem + cb * 32, v);
-          fold32(st, v, base, ctx_r - 1, 0, p.scale_log2);
+          tmem_ld32(acc + cb * 32, v);
+          if (cb == 2 * half + 1) {
+            co.release();
+            released = true;
+          }
+          if (warp_full && base + 32 <= lo_ctx) fold32<false, false>(st, v, 32, 0, false, p.scale_log2);
+          else fold32<true, false>(st, v, clamp32(ctx_r - base), 0, false, p.scale_log2);
         }
+        if (!released) co.release();
       }
-      ok = tile_done(fine);
-    }
-    const float inv = st.all > 0.f ? 1.f / st.all : 0.f;
+      // both threads of a row get the statistics of the whole row
+      float (*xch)[2][kRows] = s_half[blk & 1];
+      xch[half][0][rl] = st.m;
+      xch[half][1][rl] = st.all;
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+      {
+        const float m2 = xch[half ^ 1][0][rl], l2 = xch[half ^ 1][1][rl];
+        const float mn = fmaxf(st.m, m2);
+        // the same expression in both threads (operands ordered by column half), so they agree bit for bit
+        const float lo_m = half ? m2 : st.m, hi_m = half ? st.m : m2;
+        const float lo_l = half ? l2 : st.all, hi_l = half ? st.all : l2;
+        st.all = lo_l * ex2(lo_m - mn) + hi_l * ex2(hi_m - mn);
+        st.m = mn;
+      }
+      const float inv = st.all > 0.f ? 1.f / st.all : 0.f;
 
-    // sweep 2: normalised probabilities, column sums over the block's rows
-    for (int k0 = (p.L / kKeys) * kKeys; k0 < ctx_max && ok; k0 += kKeys) {
-      const bool fine = logits_tile(k0);
-      if (fine) {
+      // sweep 2: normalised probabilities, column sums over the block's rows
+      for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) {
+        const uint32_t acc = co.tile();
+        bool released = false;
 #pragma unroll 1
-        for (int cb = 0; cb < kKeys / 32; ++cb) {
+        for (int cb = 2 * half; cb < 2 * half + 2; ++cb) {
           const int base = k0 + cb * 32;
           if (base >= warp_ctx) break;
           if (base + 32 <= p.L) continue;                 // prompt keys only: not scored
           float v[32];
-          tmem_ld32(my_tmem + cb * 32, v);
-          const int nv = min(max(ctx_r - base, 0), 32);
+          tmem_ld32(acc + cb * 32, v);
+          if (cb == 2 * half + 1) {
+            co.release();
+            released = true;
+          }
+          if (warp_full && base + 32 <= lo_ctx) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv : 0.f;
+            for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv;
+          } else {
+            const int nv = clamp32(ctx_r - base);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv : 0.f;
+          }
           const float col = warp_column_sums(v, lane);
           const int key = base + lane;
-          if (key >= p.L && key < ctx_max) my_score[key - p.L] += col;
+          if (key >= p.L && key < b.ctx_max) my_score[key - p.L] += col;
         }
+        if (!released) co.release();
       }
-      ok = tile_done(fine);
     }
   }
 
   __syncthreads();
+  const bool ok = s_abort == 0;
   float* out = p.score + (size_t)pair * p.n0;
-  for (int j = tid; j < p.n0; j += kRows)
+  for (int j = tid; j < p.n0; j += kTcThreads)
     out[j] = ok ? (s_score[j] + s_score[p.n0 + j]) + (s_score[2 * p.n0 + j] + s_score[3 * p.n0 + j]) : 0.f;
   if (tid == 0 && !ok) atomicOr(p.status, 4u);
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kKeys) : "memory");
-  }
+  cta_teardown(tmem);
+}
+
+// ---- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tensor_map_encoder() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// Map of a [units, rows, 128] bf16 tensor, read in boxes of 128 rows x 64 elements with the 128-byte
+// swizzle; rows past `rows` read as zeros.
+cudaError_t make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t units) {
+  EncodeTiledFn enc = tensor_map_encoder();
+  if (!enc) return cudaErrorNotSupported;
+  if (rows == 0 || units == 0 || rows >> 31 || units >> 31) return cudaErrorInvalidValue;
+  const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, rows, units};
+  const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, rows * kHeadDim * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -390,20 +650,27 @@ __global__ void __launch_bounds__(kRows) ssd_score_kernel(const ScoreParams p) {
 int classify_rows_per_block() { return kRows; }
 
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st) {
-  const int smem = 2 * kTileBytes + 1024;
-  cudaError_t e = cudaFuncSetAttribute(ssd_classify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const int smem = (1 + kStages) * kTileBytes + 1024;
+  CUtensorMap tq, tk;
+  cudaError_t e = make_tile_map(&tq, p.q_cal, (uint64_t)p.N, (uint64_t)p.n_units);
+  if (e == cudaSuccess) e = make_tile_map(&tk, p.k_cal, (uint64_t)p.L + p.N, (uint64_t)p.n_units);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ssd_classify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  ssd_classify_kernel<<<p.n_units * n_row_blocks, kRows, smem, st>>>(p, n_row_blocks);
+  ssd_classify_kernel<<<p.n_units * n_row_blocks, kTcThreads, smem, st>>>(p, n_row_blocks, tq, tk);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
-  const size_t smem = 2 * (size_t)kTileBytes + 4 * (size_t)p.n0 * sizeof(float) + 1024;
-  if (smem > 227 * 1024) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = (1 + kStages) * (size_t)kTileBytes + 4 * (size_t)p.n0 * sizeof(float) + 1024;
+  if (smem + 8192 > 227 * 1024) return cudaErrorInvalidValue;   // 8 KB left for the kernel's static arrays
+  CUtensorMap tq, tk;
+  const uint64_t pairs = (uint64_t)p.n_seqs * p.H;
+  cudaError_t e = make_tile_map(&tq, p.q_obs, (uint64_t)p.n_obs, pairs);
+  if (e == cudaSuccess) e = make_tile_map(&tk, p.k_full, (uint64_t)p.L + p.n0, pairs);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  ssd_score_kernel<<<p.n_seqs * p.H, kRows, smem, st>>>(p);
+  ssd_score_kernel<<<p.n_seqs * p.H, kTcThreads, smem, st>>>(p, tq, tk);
   count_launch();
   return cudaGetLastError();
 }
