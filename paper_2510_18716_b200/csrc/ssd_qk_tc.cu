@@ -533,7 +533,8 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
       const int lo_row = r0 + quad * 32;
       const bool warp_full = lo_row + 31 <= b.last;                       // all 32 rows of the warp exist
       const int lo_ctx = p.L + t_first + lo_row;                          // context of the warp's first row
-      const int warp_ctx = p.L + t_first + min(lo_row + 31, b.last);      // and of its last
+      // and of its last; 0 (nothing to do in either sweep) when the block ends before the warp's rows
+      const int warp_ctx = lo_row <= b.last ? p.L + t_first + min(lo_row + 31, b.last) : 0;
 
       // sweep 1: row maximum and exp-sum
       RowStats st = {kNegBig, 0.f, 0.f};
