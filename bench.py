@@ -6,7 +6,7 @@
 Prints ONE JSON line.  A "step" is one decoded image token for every sequence: for each layer,
 ssd_append of the new K/V then ssd_decode_attn.  `value` is decoded image tokens per second
 (one per CFG pair per step) over the whole job with inputs resident in HBM; `e2e` is the same
-through ssd_step_host with pinned HOST buffers (copies inside the timed region).  Under torchrun
+through ssd_step_host_layers with pinned HOST buffers (copies inside the timed region).  Under torchrun
 each rank owns its own block of sequences (weak scaling, no data-path collective); time is the max
 over ranks.  `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample.
 """
@@ -347,12 +347,14 @@ def run_ours(args, cfg):
                              "launches_timed": int(len(dec_ms)), "ms_per_step_while_timing_launches": ms_r / Kr},
                 "frac_of_8TBs_nominal": achieved / 8000.0}
 
-    # ---- end to end: the same step through ssd_step_host with pinned host buffers
+    # ---- end to end: the same step through ssd_step_host_layers with pinned host buffers: one call
+    # per step takes every layer's q, k_new, v_new from the host and returns every layer's output
     pool = 4
-    hq = [[steps_in[l][0][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
-    hk = [[steps_in[l][1][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
-    hv = [[steps_in[l][2][i].cpu().pin_memory() for i in range(pool)] for l in range(cfg.n_layers)]
-    ho = [torch.empty((S, H, 128), dtype=torch.bfloat16).pin_memory() for _ in range(cfg.n_layers)]
+    stack = lambda j, i: torch.stack([steps_in[l][j][i] for l in range(cfg.n_layers)]).cpu().pin_memory()
+    hq = [stack(0, i) for i in range(pool)]
+    hk = [stack(1, i) for i in range(pool)]
+    hv = [stack(2, i) for i in range(pool)]
+    ho = torch.empty((cfg.n_layers, S, H, 128), dtype=torch.bfloat16).pin_memory()
     state = {"i": 0}
 
     def host_step():
@@ -360,8 +362,7 @@ def run_ours(args, cfg):
             for layer in range(cfg.n_layers):
                 cache.rewind(layer, n0)
         i = state["i"] % pool
-        for layer in range(cfg.n_layers):
-            cache.step_host(layer, hq[layer][i], hk[layer][i], hv[layer][i], ho[layer])
+        cache.step_host_layers(0, hq[i], hk[i], hv[i], ho)
         state["i"] += 1
 
     Ke = max(4, min(K, 16))

@@ -183,6 +183,23 @@ int ssd_decode_attn_static(ssd_cache *cache, int32_t layer, const void *q, void 
 int ssd_step_host(ssd_cache *cache, int32_t layer, const void *q_host, const void *k_new_host,
                   const void *v_new_host, void *out_host, void *stream);
 
+/* The same for n_layers consecutive layers in one call, with the copies running beside the kernels:
+ * layers move in groups of 4 (one copy per tensor and group); a group's inputs are copied on a
+ * stream of the library's own while the group before it is attended to, and its outputs go back
+ * on another while the next group runs (a ring of 3 staging slots inside the cache buffer; the
+ * streams and events are created at the first call).
+ *   q_host, k_new_host, v_new_host, out_host [n_layers, n_seqs, n_heads, head_dim] bf16 on the
+ *   host, pinned (pageable memory works but serialises the copies); entry i belongs to layer
+ *   first_layer + i.
+ * The kernels are ordered after the work already on `stream`, and `stream` is made to wait for the
+ * last copy, so the results are on the host once `stream` has drained; until then the host buffers
+ * must stay untouched.  The INPUT copies do not wait for earlier work on `stream` (so that the next
+ * step's inputs travel under this step's kernels): the input buffers must hold their values when
+ * the call is made.  SSD_ERR_OVERFLOW (nothing enqueued) if any of the layers is full.
+ * Asynchronous. */
+int ssd_step_host_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *q_host,
+                         const void *k_new_host, const void *v_new_host, void *out_host, void *stream);
+
 /* Absolute positions held by each slot of a layer, for inspection and index-set parity:
  * idx_host [n_seqs, n_heads, max_slots] int32 with max_slots = ssd_cache_max_slots(); slots are
  * ordered prompt, static (ascending position), ring (physical ring order); -1 = empty or unused.

@@ -26,7 +26,7 @@ SSD_ERR_LIMIT = -6
 EXPORTS = [
     "ssd_status_string", "ssd_cache_required_bytes", "ssd_cache_create", "ssd_cache_free",
     "ssd_classify_heads", "ssd_classify_partial", "ssd_set_head_labels", "ssd_compress", "ssd_append",
-    "ssd_decode_attn", "ssd_step_host", "ssd_cache_get_indices", "ssd_cache_max_slots",
+    "ssd_decode_attn", "ssd_step_host", "ssd_step_host_layers", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
@@ -82,6 +82,7 @@ def load():
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    L.ssd_step_host_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
     L.ssd_cache_max_slots.argtypes = [vp]
     L.ssd_cache_max_slots.restype = i32
@@ -272,6 +273,16 @@ class SsdCache:
             assert (not t.is_cuda) and t.dtype == torch.bfloat16 and t.is_contiguous()
         self._check(self.lib.ssd_step_host(self._h, layer, q_host.data_ptr(), k_new_host.data_ptr(),
                                            v_new_host.data_ptr(), out_host.data_ptr(), _stream()), "ssd_step_host")
+
+    def step_host_layers(self, first_layer: int, q_host, k_new_host, v_new_host, out_host):
+        """Append + decode of q_host.shape[0] consecutive layers from (pinned) host bf16 tensors
+        [n_layers, n_seqs, n_heads, head_dim], copies overlapped with the kernels; asynchronous."""
+        n = q_host.shape[0]
+        for t in (q_host, k_new_host, v_new_host, out_host):
+            assert (not t.is_cuda) and t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape[0] == n
+        self._check(self.lib.ssd_step_host_layers(self._h, first_layer, n, q_host.data_ptr(), k_new_host.data_ptr(),
+                                                  v_new_host.data_ptr(), out_host.data_ptr(), _stream()),
+                    "ssd_step_host_layers")
 
     # -- inspection
     def max_slots(self) -> int:

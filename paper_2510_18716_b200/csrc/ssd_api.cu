@@ -15,6 +15,12 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 
 static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
+// ssd_step_host_layers moves layers in groups of kHostGroup (one copy per tensor and group: a copy
+// of one layer's 0.5 MB costs about as much in set-up as in transfer) through a ring of kHostSlots
+// staging slots; a slot holds q, k_new, v_new and out of a whole group.
+constexpr int kHostGroup = 4;
+constexpr int kHostSlots = 3;
+
 struct Regions {
   size_t desc, idx, counters, status, partial, score, staging, acc, logits, ml, slab;  // byte offsets
   size_t score_bytes, partial_bytes, front_bytes;
@@ -49,7 +55,7 @@ static Regions plan_regions(const ssd_config& c) {
   r.partial = off;   off = align_up(off + r.partial_bytes);
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
   r.score = off;     off = align_up(off + r.score_bytes);
-  r.staging = off;   off = align_up(off + 4 * pairs_layer * kHeadDim * 2);
+  r.staging = off;   off = align_up(off + (size_t)kHostSlots * kHostGroup * 4 * pairs_layer * kHeadDim * 2);
   // row-buffer mode (Algorithm 2): accumulated scores and the last decode's logits of the static and
   // ring slots, and the last decode's (max, exp-sum), per layer
   const size_t mr = (size_t)c.sink_budget + c.sink_recent;
@@ -85,6 +91,11 @@ struct ssd_cache {
   bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
   std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
   std::vector<uint8_t> pending;       // [layers] last decode's logits not yet added to the scores
+  // ssd_step_host_layers: copy streams and per-slot events, created at its first call
+  cudaStream_t h_in = nullptr, h_out = nullptr;
+  cudaEvent_t h_fork = nullptr, h_loaded[kHostSlots] = {}, h_done[kHostSlots] = {}, h_stored[kHostSlots] = {};
+  long h_groups = 0;                  // groups sent through the staging ring so far
+  bool h_foreign = false;             // ssd_step_host has used the staging area since
   std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
   int prof_n = 0;                     // launches recorded since the last collect
 
@@ -104,7 +115,9 @@ struct ssd_cache {
   int sem_tokens(int layer) const { return row_buffer ? t_img[layer] - t_base[layer] : t_img[layer]; }
   float* d_partial() const { return reinterpret_cast<float*>(base + reg.partial); }
   float* d_score() const { return reinterpret_cast<float*>(base + reg.score); }
-  char* d_staging() const { return base + reg.staging; }
+  char* d_staging(int slot = 0) const {
+    return base + reg.staging + (size_t)slot * kHostGroup * 4 * cfg.n_seqs * cfg.n_heads * kHeadDim * 2;
+  }
   uint4* d_slab(int layer) const { return reinterpret_cast<uint4*>(base + reg.slab) + (size_t)layer_base[layer] * kSlotU4; }
   int max_slots() const {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
@@ -203,8 +216,39 @@ static void destroy_events(ssd_cache* c) {
   c->prof_n = 0;
 }
 
+static void destroy_host_pipe(ssd_cache* c) {
+  if (c->h_in) cudaStreamDestroy(c->h_in);
+  if (c->h_out) cudaStreamDestroy(c->h_out);
+  if (c->h_fork) cudaEventDestroy(c->h_fork);
+  for (int i = 0; i < kHostSlots; ++i) {
+    if (c->h_loaded[i]) cudaEventDestroy(c->h_loaded[i]);
+    if (c->h_done[i]) cudaEventDestroy(c->h_done[i]);
+    if (c->h_stored[i]) cudaEventDestroy(c->h_stored[i]);
+    c->h_loaded[i] = c->h_done[i] = c->h_stored[i] = nullptr;
+  }
+  c->h_in = c->h_out = nullptr;
+  c->h_fork = nullptr;
+}
+
+static bool make_host_pipe(ssd_cache* c) {
+  if (c->h_in) return true;
+  bool ok = cudaStreamCreateWithFlags(&c->h_in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&c->h_out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&c->h_fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < kHostSlots; ++i)
+    ok = cudaEventCreateWithFlags(&c->h_loaded[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->h_done[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->h_stored[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    destroy_host_pipe(c);
+  }
+  return ok;
+}
+
 int ssd_cache_free(ssd_cache* c) {
   if (c) destroy_events(c);
+  if (c) destroy_host_pipe(c);
   delete c;
   return SSD_OK;
 }
@@ -520,6 +564,7 @@ int ssd_step_host(ssd_cache* c, int32_t layer, const void* q_host, const void* k
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t nb = (size_t)g.n_seqs * g.n_heads * kHeadDim * 2;
   char* s = c->d_staging();
+  c->h_foreign = true;
   if (cudaMemcpyAsync(s, q_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(s + nb, k_new_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(s + 2 * nb, v_new_host, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) {
@@ -529,6 +574,70 @@ int ssd_step_host(ssd_cache* c, int32_t layer, const void* q_host, const void* k
   int rc = ssd_append_decode(c, layer, s + nb, s + 2 * nb, s, s + 3 * nb, stream);
   if (rc != SSD_OK) return rc;
   if (cudaMemcpyAsync(out_host, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  return SSD_OK;
+}
+
+int ssd_step_host_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, const void* q_host, const void* k_new_host,
+                         const void* v_new_host, void* out_host, void* stream) {
+  if (!c || !q_host || !k_new_host || !v_new_host || !out_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  for (int i = 0; i < n_layers; ++i)
+    if (c->t_img[first_layer + i] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;   // before anything is enqueued
+  if (!make_host_pipe(c)) return SSD_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t nb = (size_t)g.n_seqs * g.n_heads * kHeadDim * 2;
+  const char* qh = static_cast<const char*>(q_host);
+  const char* kh = static_cast<const char*>(k_new_host);
+  const char* vh = static_cast<const char*>(v_new_host);
+  char* oh = static_cast<char*>(out_host);
+  bool ok = true;
+  auto chk = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
+  // The copies into a staging slot wait only for the kernels that last read that slot (events of the
+  // ring, which carries on from call to call), not for the caller's stream as a whole: the next
+  // step's inputs travel while this step's last kernels run.  If ssd_step_host has used the staging
+  // area in between, the copy-in stream first waits for everything on the caller's stream.
+  if (c->h_foreign) {
+    chk(cudaEventRecord(c->h_fork, st));
+    chk(cudaStreamWaitEvent(c->h_in, c->h_fork, 0));
+    c->h_foreign = false;
+  }
+  int rc = SSD_OK;
+  const size_t gb = (size_t)kHostGroup * nb;            // a slot is [q | k_new | v_new | out], each of a group
+  for (int i0 = 0; ok && rc == SSD_OK && i0 < n_layers; i0 += kHostGroup) {
+    const long grp = c->h_groups++;
+    const int slot = (int)(grp % kHostSlots);
+    const int cnt = n_layers - i0 < kHostGroup ? n_layers - i0 : kHostGroup;
+    char* s = c->d_staging(slot);
+    // inputs of a slot may be overwritten once the kernels that read them are done
+    if (grp >= kHostSlots) chk(cudaStreamWaitEvent(c->h_in, c->h_done[slot], 0));
+    chk(cudaMemcpyAsync(s, qh + (size_t)i0 * nb, cnt * nb, cudaMemcpyHostToDevice, c->h_in));
+    chk(cudaMemcpyAsync(s + gb, kh + (size_t)i0 * nb, cnt * nb, cudaMemcpyHostToDevice, c->h_in));
+    chk(cudaMemcpyAsync(s + 2 * gb, vh + (size_t)i0 * nb, cnt * nb, cudaMemcpyHostToDevice, c->h_in));
+    chk(cudaEventRecord(c->h_loaded[slot], c->h_in));
+    chk(cudaStreamWaitEvent(st, c->h_loaded[slot], 0));
+    // the slot's outputs may be overwritten once its previous contents have gone to the host
+    // (kHostSlots groups ago: long done, so this does not stall the kernels)
+    if (grp >= kHostSlots) chk(cudaStreamWaitEvent(st, c->h_stored[slot], 0));
+    if (!ok) break;
+    for (int j = 0; j < cnt && rc == SSD_OK; ++j)
+      rc = ssd_append_decode(c, first_layer + i0 + j, s + gb + j * nb, s + 2 * gb + j * nb, s + j * nb,
+                             s + 3 * gb + j * nb, stream);
+    if (rc != SSD_OK) break;
+    chk(cudaEventRecord(c->h_done[slot], st));
+    chk(cudaStreamWaitEvent(c->h_out, c->h_done[slot], 0));
+    chk(cudaMemcpyAsync(oh + (size_t)i0 * nb, s + 3 * gb, cnt * nb, cudaMemcpyDeviceToHost, c->h_out));
+    chk(cudaEventRecord(c->h_stored[slot], c->h_out));
+  }
+  // join: the caller's stream is not done before the outputs are on the host (the kernels have
+  // already waited for the inputs)
+  for (int slot = 0; slot < kHostSlots; ++slot) cudaStreamWaitEvent(st, c->h_stored[slot], 0);
+  if (rc != SSD_OK) return rc;
+  if (!ok) {
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }

@@ -169,6 +169,48 @@ def test_step_host_matches_device_path():
         assert torch.equal(a, b)
 
 
+def test_step_host_layers_matches_device_path():
+    """Fourteen layers (four groups: more than the staging ring holds, the last group short) from
+    pinned host arrays in one call, several steps in a row, against per-layer calls on device
+    tensors: bit-identical outputs."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], n_layers=14, n_seqs=2)
+    dev = torch.device("cuda:0")
+    L, n0, nl, steps = cfg.prompt_len, cfg.n0, cfg.n_layers, 5
+    data = [wl.gen_layer(cfg, l, range(cfg.n_seqs), device=dev) for l in range(nl)]
+    labels = np.concatenate([wl.sink_mask(cfg, l) for l in range(nl)])
+    caches = []
+    for _ in range(2):
+        cache = B.SsdCache(B.config_from_workload(cfg))
+        cache.set_head_labels(labels)
+        for l, (q, k, v, _) in enumerate(data):
+            cache.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(cache)
+    dev_cache, host_cache = caches
+    for t in range(n0 + 1, n0 + 1 + steps):
+        qs = torch.stack([data[l][0][:, :, t - 1] for l in range(nl)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        want = torch.stack([dev_cache.append_decode(l, ks[l], vs[l], qs[l]) for l in range(nl)]).cpu()
+        hq, hk, hv = (x.cpu().pin_memory() for x in (qs, ks, vs))
+        ho = torch.zeros_like(hq).pin_memory()
+        host_cache.step_host_layers(0, hq, hk, hv, ho)
+        torch.cuda.synchronize()
+        assert torch.equal(ho, want)
+    # a sub-range of layers, and the full-layer guard
+    hq1, hk1, hv1 = (x[2:4].contiguous().pin_memory() for x in (hq, hk, hv))   # the layers' own step inputs
+    ho1 = torch.zeros_like(hq1).pin_memory()
+    host_cache.step_host_layers(2, hq1, hk1, hv1, ho1)
+    torch.cuda.synchronize()
+    assert host_cache.tokens(2) == host_cache.tokens(0) + 1 and host_cache.tokens(4) == host_cache.tokens(0)
+    lib = B.load()
+    assert lib.ssd_step_host_layers(host_cache._h, 13, 2, hq1.data_ptr(), hk1.data_ptr(), hv1.data_ptr(), ho1.data_ptr(),
+                                    None) == B.SSD_ERR_INVALID_ARG
+    assert host_cache.device_status() == 0
+    for c in caches:
+        c.close()
+
+
 def test_argument_errors_launch_nothing():
     cfg = B.make_config(2, 2, 4, 8, 16, 4, 4, 2)
     cache = B.SsdCache(cfg)
