@@ -135,6 +135,19 @@ int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, v
 int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new,
                       const void *q, void *out, void *stream);
 
+/* ssd_append_decode for n_layers consecutive layers in ONE launch (a whole decode step when the
+ * inputs of all layers exist up front, as in a benchmark of this path or a host-driven replay; in a
+ * model, layer l+1's query depends on layer l's output and the per-layer call is the one to use).
+ *   k_new, v_new, q, out [n_layers, n_seqs, n_heads, head_dim] bf16 on the device, 16-byte
+ *   aligned; entry i belongs to layer first_layer + i.
+ * Results are those of the per-layer call up to the rounding order of the softmax sums (a head is
+ * summed by one warp here, by up to several there).  The work is handed out head by head from a
+ * counter in the cache buffer, so the layers need not have the same layout or occupancy.
+ * SSD_ERR_LIMIT if n_layers > 64 (issue several calls), SSD_ERR_OVERFLOW (nothing launched) if any
+ * of the layers is full, SSD_ERR_BAD_STATE in row-buffer mode.  Asynchronous. */
+int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *k_new,
+                             const void *v_new, const void *q, void *out, void *stream);
+
 /* Row-buffer mode (Algorithm 2, Appendix B).  With the mode on, the ring of a semantic head is the
  * algorithm's row buffer of R = sink_recent tokens, filled from empty:
  *   ssd_compress     selects the top-M over all n0 tokens (the buffer starts empty) and records the

@@ -26,7 +26,7 @@ SSD_ERR_LIMIT = -6
 EXPORTS = [
     "ssd_status_string", "ssd_cache_required_bytes", "ssd_cache_create", "ssd_cache_free",
     "ssd_classify_heads", "ssd_classify_partial", "ssd_set_head_labels", "ssd_compress", "ssd_append",
-    "ssd_decode_attn", "ssd_step_host", "ssd_step_host_layers", "ssd_cache_get_indices", "ssd_cache_max_slots",
+    "ssd_decode_attn", "ssd_append_decode_layers", "ssd_step_host", "ssd_step_host_layers", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
@@ -82,6 +82,7 @@ def load():
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    L.ssd_append_decode_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_step_host_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
     L.ssd_cache_max_slots.argtypes = [vp]
@@ -241,6 +242,19 @@ class SsdCache:
             out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
         self._check(self.lib.ssd_append_decode(self._h, layer, _dev(k_new, shp, "k_new"), _dev(v_new, shp, "v_new"),
                                                _dev(q, shp, "q"), _dev(out, shp, "out"), _stream()), "ssd_append_decode")
+        return out
+
+    def append_decode_layers(self, first_layer: int, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor,
+                             out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """append + decode_attn of q.shape[0] consecutive layers in one launch; tensors
+        [n_layers, n_seqs, n_heads, head_dim]."""
+        c = self.cfg
+        shp = (q.shape[0], c.n_seqs, c.n_heads, c.head_dim)
+        if out is None:
+            out = torch.empty(shp, dtype=torch.bfloat16, device=q.device)
+        self._check(self.lib.ssd_append_decode_layers(self._h, first_layer, shp[0], _dev(k_new, shp, "k_new"),
+                                                      _dev(v_new, shp, "v_new"), _dev(q, shp, "q"), _dev(out, shp, "out"),
+                                                      _stream()), "ssd_append_decode_layers")
         return out
 
     def decode_attn_static(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:

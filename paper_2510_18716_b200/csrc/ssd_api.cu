@@ -50,7 +50,7 @@ static Regions plan_regions(const ssd_config& c) {
   r.desc = off;      off = align_up(off + (size_t)c.n_layers * c.n_heads * sizeof(HeadDesc));
   r.idx = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * (c.sink_budget > 0 ? c.sink_budget : 1) * 4);
   r.counters = off;  off = align_up(off + pairs_layer * 4);
-  r.status = off;    off = align_up(off + 4);
+  r.status = off;    off = align_up(off + 132);   // status word, and at +128 the unit counter of the all-layers launch
   r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
   r.partial = off;   off = align_up(off + r.partial_bytes);
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
@@ -106,6 +106,7 @@ struct ssd_cache {
   }
   uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(base + reg.status); }
+  uint32_t* d_work() const { return reinterpret_cast<uint32_t*>(base + reg.status + 128); }   // unit counter of the all-layers launch
   int mr() const { return cfg.sink_budget + cfg.sink_recent; }
   size_t layer_scores(int layer) const { return (size_t)layer * cfg.n_seqs * cfg.n_heads * mr(); }
   float* d_acc(int layer) const { return reinterpret_cast<float*>(base + reg.acc) + layer_scores(layer); }
@@ -551,6 +552,49 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
   }
+  return SSD_OK;
+}
+
+int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, const void* k_new, const void* v_new,
+                             const void* q, void* out, void* stream) {
+  if (!c || !k_new || !v_new || !q || !out) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
+  if (n_layers > kMaxLayersPerLaunch) return SSD_ERR_LIMIT;
+  if (!c->labels_set || c->row_buffer) return SSD_ERR_BAD_STATE;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
+       reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
+    return SSD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_layers; ++i)
+    if (c->t_img[first_layer + i] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DecodeLayersParams p;
+  p.slab = reinterpret_cast<uint4*>(c->base + c->reg.slab);
+  p.q = static_cast<const unsigned char*>(q);
+  p.k_new = static_cast<const unsigned char*>(k_new);
+  p.v_new = static_cast<const unsigned char*>(v_new);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.status = c->d_status();
+  p.work = c->d_work();
+  p.n_layers = n_layers; p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
+  p.scale_log2 = c->scale * 1.4426950408889634f;
+  for (int i = 0; i < n_layers; ++i) {
+    const int layer = first_layer + i;
+    LayerState& ls = p.layer[i];
+    ls.first_slot = c->layer_base[layer];
+    ls.desc = c->d_desc(layer);
+    ls.seq_slots = c->seq_slots[layer];
+    ls.prompt_valid = c->prompt_valid[layer];
+    ls.static_valid = c->static_valid[layer];
+    ls.new_j = c->t_img[layer];
+    ls.t_img = c->t_img[layer] + 1;
+  }
+  if (cudaMemsetAsync(p.work, 0, 4, st) != cudaSuccess || launch_decode_layers(p, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  for (int i = 0; i < n_layers; ++i) c->t_img[first_layer + i] += 1;
+  c->last_writer = -2;                 // several layers' slabs were written
   return SSD_OK;
 }
 

@@ -684,6 +684,204 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   }
 }
 
+// ------------------------------------------------------------------ a whole step in one launch
+// Fused append + decode of every layer.  With all layers in one launch there are tens of thousands
+// of heads to go round, so no head needs to be cut: the unit of work is one whole head of one
+// (layer, sequence), units are handed out in stream order from a global counter to whichever warp
+// asks next (warps on slower SMs simply take fewer), and a head is finished in the registers of the
+// warp that streamed it.  No partials, no mailboxes, no finisher, no barrier after start-up.  A
+// warp's copy pipeline runs on across unit boundaries: the next unit is claimed while the current
+// one streams, and its first chunks are in flight before the current head's arithmetic ends.
+struct Unit {
+  const unsigned char* hbase;   // the head's first slot
+  size_t row;                   // byte offset of the head's row in q, k_new, v_new (and out)
+  int vh;                       // slots that hold a token
+  int pv, sv;                   // of which prompt slots and static slots (the rest is the ring)
+  int y;                        // static capacity (slots between the prompt and the ring)
+  int fresh;                    // valid-slot index of the token being appended
+  int phys;                     // and its slot counted from the head's first slot
+  int contig;                   // the valid slots are one physical run
+};
+
+__device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Unit& U) {
+  const int pairs = p.n_seqs * p.H;
+  const int layer = u / pairs, pair = u - layer * pairs;
+  const int seq = pair / p.H, head = pair - seq * p.H;
+  const LayerState& ls = p.layer[layer];
+  const HeadDesc d = __ldg(ls.desc + head);
+  const int r = ls.new_j % d.z;
+  U.pv = ls.prompt_valid;
+  U.sv = d.w ? ls.static_valid : 0;
+  U.y = d.y;
+  U.vh = U.pv + U.sv + (ls.t_img < d.z ? ls.t_img : d.z);
+  U.fresh = U.pv + U.sv + r;
+  U.phys = p.L + d.y + r;
+  U.contig = (U.pv == p.L && U.sv == d.y) ? 1 : 0;
+  U.hbase = reinterpret_cast<const unsigned char*>(p.slab) +
+            ((size_t)ls.first_slot + (size_t)seq * ls.seq_slots + d.x) * kSlotBytes;
+  U.row = ((size_t)layer * pairs + pair) * kQBytes;
+}
+
+constexpr int kLayersSmemBytes = kRingBytes + kWarps * kStages * 8 + kWarps * 4 * 4;
+
+__global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const __grid_constant__ DecodeLayersParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = lane >> 3, l8 = lane & 7;
+  const uint32_t FULL = 0xffffffffu;
+  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
+  const uint32_t ring_s = smem_u32(ring);
+  const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
+  volatile int* fifo = reinterpret_cast<volatile int*>(smem + kRingBytes + kWarps * kStages * 8) + warp * 4;
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    mbar_init_fence();
+  }
+  __syncwarp();
+  const int n_units = p.n_layers * p.n_seqs * p.H;
+
+  // unit ids come from the counter; lane 0 asks for the next one long before it is needed
+  int raw_next = 0;
+  auto ask = [&]() {
+    if (lane == 0) raw_next = (int)atomicAdd(p.work, 1u);
+  };
+  ask();
+  int u = __shfl_sync(FULL, raw_next, 0);
+  if (u >= n_units) return;
+  ask();
+
+  Unit PU, CU;                 // the producer's and the consumer's current head
+  int pi = 0, ci = 0;          // and their positions in it
+  int produced = 0, consumed = 0, ahead = 0;
+  bool feeding = true;
+  unit_load(p, u, PU);
+  if (lane == 0) fifo[0] = u;
+  produced = 1;
+  __syncwarp();
+
+  // Lane 0 starts the copies of the producer's next chunk into `stage`; every lane advances.
+  auto issue = [&](int stage) {
+    const int n = PU.vh - pi < kChunk ? PU.vh - pi : kChunk;
+    if (lane == 0) {
+      const bool begin = pi == 0;
+      const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
+      const bool has_fresh = PU.fresh >= pi && PU.fresh < pi + n;
+      // order the warp's reads of this stage (made visible to this lane by __syncwarp) before
+      // the asynchronous writes that follow
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + (begin ? kQBytes : 0)));
+      // valid slots [a, a + len) of the head into the stage from slot `at` on
+      auto copy_range = [&](int a, int len, int at) {
+        if (len <= 0) return;
+        if (PU.contig) {
+          bulk_g2s(dst + (uint32_t)at * kSlotBytes, PU.hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
+          return;
+        }
+        const int l0[3] = {0, PU.pv, PU.pv + PU.sv};          // logical start of each run
+        const int l1[3] = {PU.pv, PU.pv + PU.sv, PU.vh};      // and end
+        const int p0[3] = {0, p.L, p.L + PU.y};               // physical start
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+          const int lo = a > l0[r] ? a : l0[r], hi = a + len < l1[r] ? a + len : l1[r];
+          if (hi > lo)
+            bulk_g2s(dst + (uint32_t)(at + lo - a) * kSlotBytes, PU.hbase + (size_t)(p0[r] + lo - l0[r]) * kSlotBytes,
+                     (uint32_t)(hi - lo) * kSlotBytes, bar);
+        }
+      };
+      if (has_fresh) {                   // the slab is copied around the newest token's slot
+        copy_range(pi, PU.fresh - pi, 0);
+        copy_range(PU.fresh + 1, pi + n - PU.fresh - 1, PU.fresh + 1 - pi);
+        bulk_g2s(dst + (uint32_t)(PU.fresh - pi) * kSlotBytes, p.k_new + PU.row, kQBytes, bar);
+        bulk_g2s(dst + (uint32_t)(PU.fresh - pi) * kSlotBytes + kQBytes, p.v_new + PU.row, kQBytes, bar);
+      } else {
+        copy_range(pi, n, 0);
+      }
+      if (begin) bulk_g2s(dst + kChunk * kSlotBytes, p.q + PU.row, kQBytes, bar);
+    }
+    pi += n;
+    ++ahead;
+    if (pi == PU.vh) {                   // on to the unit asked for earlier, and ask for the one after
+      const int nu = __shfl_sync(FULL, raw_next, 0);
+      if (nu < n_units) {
+        ask();
+        unit_load(p, nu, PU);
+        pi = 0;
+        if (lane == 0) fifo[produced & 3] = nu;
+        ++produced;
+        __syncwarp();
+      } else {
+        feeding = false;
+      }
+    }
+  };
+
+#pragma unroll 1
+  for (int s = 0; s < kStages && feeding; ++s) issue(s);
+
+  int stage = 0;
+  uint32_t parity = 0;
+  float2 q[8];
+  State st;
+  const LogitSink sink = {nullptr, 0, 0, 0, 0};
+  bool begin = true;
+
+#pragma unroll 1
+  for (;;) {
+    if (begin) {
+      if (consumed == produced) break;
+      unit_load(p, fifo[consumed & 3], CU);
+      ++consumed;
+      ci = 0;
+    }
+    const int n = CU.vh - ci < kChunk ? CU.vh - ci : kChunk;
+    if (!mbar_wait(bar0 + 8 * stage, parity)) {
+      // give up: flag it, let the copies still in flight land (bounded), and leave
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int k = 0; k < ahead; ++k) {
+        mbar_wait(bar0 + 8 * stage, parity);
+        if (++stage == kStages) { stage = 0; parity ^= 1u; }
+      }
+      return;
+    }
+    const uint4* sb = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageBytes);
+    if (begin) {
+      const uint4 qa = sb[kChunk * kSlotU4 + l8], qb = sb[kChunk * kSlotU4 + 8 + l8];
+      const float2 sc = make_float2(p.scale_log2, p.scale_log2);
+      q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
+      q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
+      q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
+      q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
+      state_init(st);
+      begin = false;
+    }
+    Rows rows;
+    load_stage(sb, n, grp, l8, rows);
+    {
+      // the chunk that carries the newest token also stores it in the slab
+      const int s_new = CU.fresh - ci;
+      if (s_new >= 0 && s_new < n) {
+        uint4* dstrow = reinterpret_cast<uint4*>(const_cast<unsigned char*>(CU.hbase)) + (size_t)CU.phys * kSlotU4;
+        dstrow[lane] = sb[s_new * kSlotU4 + lane];
+      }
+    }
+    __syncwarp();          // every lane has its rows in registers: the stage may be refilled
+    --ahead;
+    if (feeding) issue(stage);
+    fold_stage(rows, n, grp, l8, q, st, sink);
+    ci += n;
+    if (ci == CU.vh) {
+      // the head is complete: merge the four groups and write the output row
+      State tot = st;
+      state_merge_lane(tot, 8);
+      state_merge_lane(tot, 16);
+      if (grp == 0) write_out(reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<unsigned char*>(p.out) + CU.row), tot, l8);
+      begin = true;
+    }
+    if (++stage == kStages) { stage = 0; parity ^= 1u; }
+  }
+}
+
 __global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   pdl_wait_predecessor();
@@ -765,6 +963,32 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
   e = cudaLaunchKernelEx(&cfg, ssd_decode_kernel, p);
   count_launch();
   return e;
+}
+
+cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
+  static bool smem_set[64] = {};
+  static int n_sm[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < 64;
+  int sms = cached ? n_sm[dev] : 0;
+  if (!cached || !smem_set[dev]) {
+    e = cudaFuncSetAttribute(ssd_decode_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLayersSmemBytes);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (cached) {
+      smem_set[dev] = true;
+      n_sm[dev] = sms;
+    }
+  }
+  const long units = (long)p.n_layers * p.n_seqs * p.H;
+  if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  const long want = (units + kWarps - 1) / kWarps;            // no more CTAs than there are units for
+  const int grid = (int)(want < sms ? want : sms);
+  ssd_decode_layers_kernel<<<grid, kWarps * 32, kLayersSmemBytes, st>>>(p);
+  count_launch();
+  return cudaGetLastError();
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st) {

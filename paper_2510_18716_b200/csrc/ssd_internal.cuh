@@ -46,6 +46,30 @@ struct DecodeParams {
   LayerView view;           // layout and occupancy of the layer
 };
 
+// One launch for a whole step (every layer's fused append + decode).
+constexpr int kMaxLayersPerLaunch = 64;
+struct LayerState {
+  long long first_slot;     // the layer's first slot in the slab
+  const HeadDesc* desc;     // [H] layout records of the layer (device)
+  int seq_slots;            // physical slots per sequence
+  int prompt_valid;         // 0 or L
+  int static_valid;         // valid static slots of semantic heads
+  int t_img;                // image tokens held, the one being appended included
+  int new_j;                // image index of the token being appended
+};
+struct DecodeLayersParams {
+  uint4* slab;              // slot 0 of the slab
+  const unsigned char* q;   // [n_layers, n_seqs, H, 128] bf16
+  const unsigned char* k_new;
+  const unsigned char* v_new;
+  __nv_bfloat16* out;       // [n_layers, n_seqs, H, 128]
+  uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
+  uint32_t* work;           // next unit to hand out; zero at launch
+  int n_layers, n_seqs, H, L;
+  float scale_log2;
+  LayerState layer[kMaxLayersPerLaunch];
+};
+
 struct AppendParams {
   uint4* slab;
   const HeadDesc* desc;
@@ -105,6 +129,7 @@ struct ClassifyParams {
 };
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
+cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st);
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);

@@ -1,0 +1,113 @@
+"""The one-launch-per-step form (ssd_append_decode_layers) against the per-layer calls and the oracle.
+
+A head is summed by a single warp there and by up to several here, so the two GPU paths agree up to
+the rounding order of the softmax sums, not bit for bit; both must meet the oracle's bar, and both
+must leave the same cache behind."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_18716_b200 import binding as B
+from paper_2510_18716_b200 import workloads as wl
+
+from parity_util import check_outputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _labels(cfg, kind, n_layers):
+    H = cfg.n_heads
+    if kind == "generator":
+        return np.stack([wl.sink_mask(cfg, l) for l in range(n_layers)])
+    # layers that differ in layout: the generator's split, all spatial, all semantic, a random one
+    rng = np.random.default_rng(5)
+    rows = [wl.sink_mask(cfg, 0), np.zeros(H, np.uint8), np.ones(H, np.uint8), rng.integers(0, 2, H).astype(np.uint8)]
+    return np.stack([rows[l % 4] for l in range(n_layers)])
+
+
+@pytest.mark.parametrize("case", ["tiny_mixed_layouts", "tiny_ring_from_zero", "janus7b_slice"])
+def test_layers_launch_matches_per_layer_calls_and_oracle(case):
+    dev = torch.device("cuda:0")
+    if case == "janus7b_slice":
+        cfg, nl, seqs, n_steps, kind = wl.CONFIGS["janus7b"], 3, list(range(6)), 20, "generator"
+    else:
+        cfg, nl, seqs, n_steps, kind = wl.CONFIGS["tiny"], 4, [0, 1], 32, "mixed"
+    L, N, n0, W, M, R, H, S = (cfg.prompt_len, cfg.n_img, cfg.n0, cfg.window, cfg.sink_budget, cfg.sink_recent,
+                               cfg.n_heads, len(seqs))
+    labels = _labels(cfg, kind, nl)
+    data = [wl.gen_layer(cfg, l, seqs, device=dev) for l in range(nl)]
+    compressed = case != "tiny_ring_from_zero"
+    t0 = n0 if compressed else 0
+    caches = []
+    for _ in range(2):
+        c = B.SsdCache(B.config_from_workload(cfg, n_layers=nl, n_seqs=S), device=dev)
+        c.set_head_labels(labels)
+        if compressed:
+            for l, (q, k, v, _) in enumerate(data):
+                c.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(c)
+    per_layer, fused = caches
+    gidx, gcnt = [], []
+    for l in range(nl):
+        gi = fused.get_indices(l)
+        idx = np.full((S, H, M), -1, np.int32)
+        for h in range(H):
+            if labels[l][h]:
+                st = gi[:, h, L:L + M]
+                idx[:, h] = np.where(st >= 0, st - L, -1)
+        gidx.append(idx)
+        gcnt.append((idx >= 0).sum(-1).astype(np.int32))
+    oracle_steps = {t0 + 1, t0 + n_steps // 2, t0 + n_steps}
+    for t in range(t0 + 1, t0 + n_steps + 1):
+        qs = torch.stack([data[l][0][:, :, t - 1] for l in range(nl)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        want = torch.stack([per_layer.append_decode(l, ks[l], vs[l], qs[l]) for l in range(nl)])
+        got = fused.append_decode_layers(0, ks, vs, qs)
+        d = (got.float() - want.float()).abs()
+        assert torch.isfinite(got.float()).all()
+        assert d.max().item() <= 2e-2 and d.mean().item() <= 5e-4, f"step {t}: {d.max().item()} {d.mean().item()}"
+        for l in range(nl):
+            assert fused.tokens(l) == per_layer.tokens(l) == t
+        if t in oracle_steps and compressed:
+            for l in range(nl):
+                q, k, v, _ = data[l]
+                sem = labels[l][None, :].repeat(S, 0).astype(np.uint8)
+                ref = oracle.decode_batch(wl.to_u16(q)[:, :, t - 1], wl.to_u16(k), wl.to_u16(v), sem, gidx[l], gcnt[l],
+                                          L, t, W, M, R)
+                check_outputs(got[l], ref, f"layer {l} step {t}")
+    for l in range(nl):
+        assert np.array_equal(fused.get_indices(l), per_layer.get_indices(l))
+    # the cache it leaves is a full substitute: per-layer calls on it continue bit for bit
+    t = t0 + n_steps + 1
+    if t <= N:
+        for l in range(nl):
+            kt, vt, qt = (x.contiguous() for x in (data[l][1][:, :, L + t - 1], data[l][2][:, :, L + t - 1],
+                                                   data[l][0][:, :, t - 1]))
+            assert torch.equal(fused.append_decode(l, kt, vt, qt), per_layer.append_decode(l, kt, vt, qt))
+    assert fused.device_status() == 0 and per_layer.device_status() == 0
+    for c in caches:
+        c.close()
+
+
+def test_layers_launch_argument_errors():
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], n_layers=2)
+    dev = torch.device("cuda:0")
+    c = B.SsdCache(B.config_from_workload(cfg, n_layers=2, n_seqs=1), device=dev)
+    x = torch.zeros((2, 1, cfg.n_heads, 128), dtype=torch.bfloat16, device=dev)
+    lib = B.load()
+    args = (x.data_ptr(), x.data_ptr(), x.data_ptr(), x.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    before = B.kernel_launch_count()
+    assert lib.ssd_append_decode_layers(c._h, 0, 2, *args) == B.SSD_ERR_BAD_STATE      # no labels yet
+    c.set_head_labels(np.stack([wl.sink_mask(cfg, l) for l in range(2)]))
+    assert lib.ssd_append_decode_layers(c._h, 1, 2, *args) == B.SSD_ERR_INVALID_ARG    # past the last layer
+    assert lib.ssd_append_decode_layers(c._h, 0, 0, *args) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_append_decode_layers(c._h, 0, 2, x.data_ptr() + 2, *args[1:]) == B.SSD_ERR_INVALID_ARG   # misaligned
+    c.set_row_buffer(True)
+    assert lib.ssd_append_decode_layers(c._h, 0, 2, *args) == B.SSD_ERR_BAD_STATE
+    c.set_row_buffer(False)
+    assert B.kernel_launch_count() == before
+    c.close()

@@ -230,6 +230,16 @@ def test_argument_errors_launch_nothing():
     with pytest.raises(B.SsdError) as e:
         cache.compress(0, None, kf, kf, 17, 0)               # n0 beyond max_image_tokens
     assert e.value.code == B.SSD_ERR_INVALID_ARG
+    # the tensor-core kernels read their inputs through the TMA unit: misaligned tensors are refused
+    lib = B.load()
+    kok = torch.zeros((2, 4, 8 + 8, 128), dtype=torch.bfloat16, device=dev)
+    pad = torch.zeros(2 * 4 * 16 * 128 + 8, dtype=torch.bfloat16, device=dev)
+    off = pad.data_ptr() + 2                                # 2-byte aligned only
+    st = torch.cuda.current_stream().cuda_stream
+    assert lib.ssd_compress(cache._h, 0, kok.data_ptr(), off, kok.data_ptr(), 8, 8, st) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_compress(cache._h, 0, off, kok.data_ptr(), kok.data_ptr(), 8, 8, st) == B.SSD_ERR_INVALID_ARG
+    sums = np.zeros(2 * 4, np.float64)
+    assert lib.ssd_classify_partial(cache._h, off, kok.data_ptr(), 1, 8, sums.ctypes.data, st) == B.SSD_ERR_INVALID_ARG
     assert B.kernel_launch_count() == before
     assert cache.kv_bytes_per_seq() == ((8 + 4) * 4 + (8 + 6) * 4) * 512
     cache.close()
