@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload janus7b] [--impl reference]
 
 Prints ONE JSON line.  A "step" is one decoded image token for every sequence: for each layer,
-ssd_append of the new K/V then ssd_decode_attn.  `value` is decoded image tokens per second
-(one per CFG pair per step) over the whole job with inputs resident in HBM; `e2e` is the same
+append the new K/V and attend.  `value` is decoded image tokens per second (one per CFG pair per
+step) over the whole job with inputs resident in HBM and the step issued as one launch
+(ssd_append_decode_layers); `per_layer` is the same step as one launch per layer; `e2e` is the same
 through ssd_step_host_layers with pinned HOST buffers (copies inside the timed region).  Under torchrun
 each rank owns its own block of sequences (weak scaling, no data-path collective); time is the max
 over ranks.  `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample.
@@ -28,11 +29,13 @@ sys.path.insert(0, ROOT)
 
 from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 
-# DRAM bytes (read + written) of one ssd_decode_kernel launch on a janus7b layer, from the ncu capture
-# summarised in profiles/ssd_decode_kernel_janus7b_layer.md.  Reported only while the kernel's sources
-# still hash to what was captured; otherwise `traffic` is null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "bytes_per_launch": 162.81e6,
-                  "sha256": "7993692ac2b01944ce25df5e056f3d649f2c608c28c8c849ae68ca9f38a765d2"}
+# DRAM bytes (read + written) from the ncu captures summarised under profiles/: one ssd_decode_kernel
+# launch on a janus7b layer, and one ssd_decode_layers_kernel launch per layer it covers (captured on
+# 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
+# Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
+# null until the counters are taken again.
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.83e6, "per_layer_of_step": 160.85e6,
+                  "sha256": "f230d96f3e2a86c5ed55eaf19eead62edea9e2450c4e68145cb27b99a82baf00"}
 
 
 def decode_traffic(cfg):
@@ -43,7 +46,7 @@ def decode_traffic(cfg):
             h.update(fh.read())
     if h.hexdigest() != DECODE_TRAFFIC["sha256"] or not cfg.name.startswith(DECODE_TRAFFIC["workload"]):
         return None
-    return DECODE_TRAFFIC["bytes_per_launch"]
+    return DECODE_TRAFFIC
 
 
 METRIC = "decoded image tokens/sec (attention+cache ops)"
@@ -256,7 +259,9 @@ class Stepper:
         i = self.i
         if one_launch:
             q, k, v = self.cache.step_all
-            self.cache.append_decode_layers(0, k[i], v[i], q[i], self.out_all)
+            for l0 in range(0, self.cfg.n_layers, 64):         # the call takes up to 64 layers
+                l1 = min(l0 + 64, self.cfg.n_layers)
+                self.cache.append_decode_layers(l0, k[i, l0:l1], v[i, l0:l1], q[i, l0:l1], self.out_all[l0:l1])
             self.i += 1
             return
         for layer in range(self.cfg.n_layers):
@@ -311,18 +316,26 @@ def run_ours(args, cfg):
     out = torch.empty((S, H, 128), dtype=torch.bfloat16, device=device)
     stepper = Stepper(cfg, cache, steps_in, out)
 
-    # ---- device-resident timing (the headline `value`)
+    # ---- device-resident timing (the headline `value`): the whole step as one launch
+    # (ssd_append_decode_layers: every layer's append + attention, heads handed out from a counter)
+    one_step = lambda: stepper.step(one_launch=True)
     for _ in range(W):
-        stepper.step()
+        one_step()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
     l0 = B.kernel_launch_count()
-    ms = timed(stepper.step, K, barrier)
+    ms = timed(one_step, K, barrier)
     launches = B.kernel_launch_count() - l0
     ms = max_over_ranks(ms)
     ms_per_step = ms / K
     value = cfg.images_per_step * world / (ms_per_step * 1e-3)
+
+    # ---- the same step as one launch per layer (ssd_append_decode; what a model calls, since layer
+    # l+1's inputs depend on layer l's output); consecutive launches overlap by programmatic dependent launch
+    for _ in range(3):
+        stepper.step()
+    ms_layers = max_over_ranks(timed(stepper.step, K, barrier)) / K
     # the same steps again with a CUDA event on either side of every decode launch (the events stand
     # between the kernels, so these launches do not overlap with their neighbours)
     Kr = min(K, 50)
@@ -331,39 +344,47 @@ def run_ours(args, cfg):
     dec_ms = cache.profile_collect()
     cache.profile_enable(0)
     clocks = sampler.stop()
-    # the same step as two launches per layer (ssd_append, ssd_decode_attn), for comparison
+    # and as two launches per layer (ssd_append, ssd_decode_attn), for comparison
     Kt = min(K, 50)
     two_step = lambda: stepper.step(fused=False)
     two_step()
     ms_two = max_over_ranks(timed(two_step, Kt, barrier)) / Kt
 
-    # the whole step as one launch (ssd_append_decode_layers)
-    one_step = lambda: stepper.step(one_launch=True)
-    for _ in range(3):
-        one_step()
-    ms_one = max_over_ranks(timed(one_step, K, barrier)) / K
-
-    # ---- roofline of the dominant kernel (decode): algorithmic bytes per launch / mean launch time
+    # ---- roofline of the dominant kernel: algorithmic bytes per launch / launch duration (CUDA events)
     slots_layer = int(sum(int(cache.get_lengths(l).sum()) for l in range(cfg.n_layers))) / cfg.n_layers
     # K+V rows of the valid slots, q in and out, and the fused append's 512 B per head read and written
     bytes_launch = S * (slots_layer * 512 + H * 2 * 256 + H * 2 * 512)
+    bytes_step = bytes_launch * cfg.n_layers
     peak, peak_kind = measured_peaks()
+    n_calls = (cfg.n_layers + 63) // 64
+    # The timed region holds nothing but launches of ssd_decode_layers_kernel (one per step for up to
+    # 64 layers, each preceded by a 4-byte memset of its unit counter), so its launch duration is the
+    # region time per launch.
+    achieved = bytes_step / (ms_per_step * 1e-3) / 1e9
+    traffic = decode_traffic(cfg)
     dec_mean_ms = float(np.mean(dec_ms)) if len(dec_ms) else float("nan")
-    # The timed region consists of nothing but launches of this one kernel (n_layers per step, each
-    # appending and attending), so its average launch duration over the region is region time /
-    # launches.  Consecutive launches overlap by design (programmatic dependent launch): timed one at
-    # a time, with an event between launches that forbids the overlap, a launch takes longer
-    # ("isolated" below).
-    launch_ms = ms_per_step / cfg.n_layers
-    achieved = bytes_launch / (launch_ms * 1e-3) / 1e9
+    # Per-layer form: its region also holds only one kernel (n_layers launches per step); launches
+    # overlap by design, so timed one at a time (an event between launches forbids the overlap) a
+    # launch takes longer ("isolated").
+    launch_ms = ms_layers / cfg.n_layers
+    ach_l = bytes_launch / (launch_ms * 1e-3) / 1e9
     iso = bytes_launch / (dec_mean_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "ssd_decode_kernel (fused append)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": decode_traffic(cfg),
-                "bytes_per_launch": bytes_launch, "launch_ms_mean": launch_ms, "launches_in_region": K * cfg.n_layers,
-                "isolated": {"launch_ms_mean": dec_mean_ms, "achieved": iso, "frac": iso / peak,
-                             "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
-                             "launches_timed": int(len(dec_ms)), "ms_per_step_while_timing_launches": ms_r / Kr},
-                "frac_of_8TBs_nominal": achieved / 8000.0}
+    per_layer = {"value": cfg.images_per_step * world / (ms_layers * 1e-3), "unit": UNIT, "ms_per_step": ms_layers,
+                 "launches_per_step": cfg.n_layers, "ms_per_step_two_launches_per_layer": ms_two,
+                 "roofline": {"bound": "hbm", "kernel": "ssd_decode_kernel (fused append)", "achieved": ach_l, "peak": peak,
+                              "unit": "GB/s", "frac": ach_l / peak, "peak_kind": f"of {peak_kind}",
+                              "traffic": traffic["per_layer"] if traffic else None,
+                              "bytes_per_launch": bytes_launch, "launch_ms_mean": launch_ms,
+                              "isolated": {"launch_ms_mean": dec_mean_ms, "achieved": iso, "frac": iso / peak,
+                                           "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
+                                           "launches_timed": int(len(dec_ms)),
+                                           "ms_per_step_while_timing_launches": ms_r / Kr},
+                              "frac_of_8TBs_nominal": ach_l / 8000.0}}
+    roofline = {"bound": "hbm", "kernel": "ssd_decode_layers_kernel (whole step, fused append)", "achieved": achieved,
+                "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": traffic["per_layer_of_step"] * cfg.n_layers / n_calls if traffic else None,
+                "bytes_per_launch": bytes_step / n_calls, "launch_ms_mean": ms_per_step / n_calls,
+                "launches_in_region": K * n_calls, "frac_of_8TBs_nominal": achieved / 8000.0}
 
     # ---- end to end: the same step through ssd_step_host_layers with pinned host buffers: one call
     # per step takes every layer's q, k_new, v_new from the host and returns every layer's output
@@ -470,7 +491,8 @@ def run_ours(args, cfg):
                        "l2": "inputs larger than L2 (each layer's slab is >126 MB and is touched once per step)",
                        "kv_bytes_per_seq": kv_bytes_per_seq},
             "sequence_tokens_per_s": value * 2 if S > 1 else value,
-            "ms_per_step_two_launches_per_layer": ms_two, "ms_per_step_one_launch": ms_one,
+            "step_form": "one launch per step (ssd_append_decode_layers); per_layer = one launch per layer",
+            "per_layer": per_layer,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf,
         }
