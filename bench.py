@@ -422,15 +422,19 @@ def run_ours(args, cfg):
     full = None
     if not args.no_full_cache:
         Kf = max(2, min(K, 8))
-        fcache, fsteps = build_cache(cfg, device, rank * S, rank, world, full_cache=True, t_steps=Kf + 3)
+        fcache, fsteps = build_cache(cfg, device, rank * S, rank, world, full_cache=True, t_steps=2 * Kf + 5)
         fst = Stepper(cfg, fcache, fsteps, out)
         for _ in range(3):
             fst.step()
-        ms_f = max_over_ranks(timed(fst.step, Kf, barrier))
-        t_mid = n0 + 3 + (Kf + 1) / 2
+        ms_fl = max_over_ranks(timed(fst.step, Kf, barrier))                       # one launch per layer
+        f_one = lambda: fst.step(one_launch=True)
+        f_one()
+        ms_f = max_over_ranks(timed(f_one, Kf, barrier))                           # one launch per step
+        t_mid = n0 + 3 + Kf + 1 + (Kf + 1) / 2
         fbytes = cfg.n_layers * S * H * ((cfg.prompt_len + t_mid) * 512 + 512)
         full = {"value": cfg.images_per_step * world / (ms_f / Kf * 1e-3), "unit": UNIT, "ms_per_step": ms_f / Kf,
                 "steps": Kf, "image_step": t_mid, "gbs": fbytes / (ms_f / Kf * 1e-3) / 1e9,
+                "ms_per_step_per_layer_launches": ms_fl / Kf,
                 "kv_bytes_per_seq": fcache.kv_bytes_per_seq()}
         fcache.close()
         del fcache, fsteps, fst
@@ -531,6 +535,9 @@ def run_sweep(args):
         for _ in range(3):
             st.step()
         ms = timed(st.step, K, lambda: None) / K
+        one = lambda: st.step(one_launch=True)
+        one()
+        ms_one = timed(one, K, lambda: None) / K
         slots = sum(int(cache.get_lengths(l).sum()) for l in range(n_layers)) / n_layers
         bytes_layer = S * (slots * 512 + H * 2 * 256 + H * 2 * 512)
         line = {"sweep": cfg.name, "batch": batch, "n_seqs": S, "ratio": ratio, "sink_frac": frac,
@@ -538,6 +545,7 @@ def run_sweep(args):
                 "layers_timed": n_layers, "us_per_layer": ms / n_layers * 1e3,
                 "ms_per_step_30_layers": ms / n_layers * 30, "image_tokens_per_s": batch / (ms / n_layers * 30 * 1e-3),
                 "gbs": bytes_layer / (ms / n_layers * 1e-3) / 1e9,
+                "one_launch": {"us_per_layer": ms_one / n_layers * 1e3, "gbs": bytes_layer / (ms_one / n_layers * 1e-3) / 1e9},
                 "kv_bytes_per_seq_30_layers": cache.kv_bytes_per_seq() // n_layers * 30,
                 "slots_per_head_mean": slots / H, "status": cache.device_status()}
         print(json.dumps(line), flush=True)
