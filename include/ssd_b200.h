@@ -143,8 +143,13 @@ int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const 
  * Results are those of the per-layer call up to the rounding order of the softmax sums (a head is
  * summed by one warp here, by up to several there).  The work is handed out head by head from a
  * counter in the cache buffer, so the layers need not have the same layout or occupancy.
- * SSD_ERR_LIMIT if n_layers > 64 (issue several calls), SSD_ERR_OVERFLOW (nothing launched) if any
- * of the layers is full, SSD_ERR_BAD_STATE in row-buffer mode.  Asynchronous. */
+ * In row-buffer mode (Algorithm 2) the kernel also adds the step's attention weights to the scores
+ * of semantic heads (a head is summed by one warp, which therefore holds all its weights), so
+ * nothing is left pending for the next append or ssd_recompress; the per-layer calls and this one
+ * can be mixed freely.
+ * SSD_ERR_LIMIT if n_layers > 64 (issue several calls) or, in row-buffer mode, if sink_budget +
+ * sink_recent exceeds what a warp can keep in shared memory (about 2800);  SSD_ERR_OVERFLOW (nothing
+ * launched) if any of the layers, or its row buffer, is full.  Asynchronous. */
 int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *k_new,
                              const void *v_new, const void *q, void *out, void *stream);
 

@@ -561,13 +561,28 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   const ssd_config& g = c->cfg;
   if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
   if (n_layers > kMaxLayersPerLaunch) return SSD_ERR_LIMIT;
-  if (!c->labels_set || c->row_buffer) return SSD_ERR_BAD_STATE;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (c->row_buffer && c->mr() > decode_layers_max_mr()) return SSD_ERR_LIMIT;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
-  for (int i = 0; i < n_layers; ++i)
-    if (c->t_img[first_layer + i] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  for (int i = 0; i < n_layers; ++i) {
+    const int layer = first_layer + i;
+    if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+    if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent)
+      return SSD_ERR_OVERFLOW;          // Algorithm 2: row buffer overflow; call ssd_recompress first
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Row-buffer mode: the kernel adds each step's attention weights to the scores itself.  A layer whose
+  // last decode came from the per-layer call still has that step's weights pending: add them first.
+  for (int i = 0; c->row_buffer && i < n_layers; ++i) {
+    const int layer = first_layer + i;
+    if (!c->pending[layer] || c->n_sink[layer] == 0) continue;
+    if (launch_fold_pending(c->d_acc(layer), c->d_logits(layer), c->d_ml(layer), c->d_desc(layer), g.n_seqs, g.n_heads,
+                            c->mr(), c->static_valid[layer], c->sem_tokens(layer), st) != cudaSuccess)
+      return SSD_ERR_CUDA;
+    c->pending[layer] = 0;
+  }
   DecodeLayersParams p;
   p.slab = reinterpret_cast<uint4*>(c->base + c->reg.slab);
   p.q = static_cast<const unsigned char*>(q);
@@ -577,6 +592,7 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   p.status = c->d_status();
   p.work = c->d_work();
   p.n_layers = n_layers; p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
+  p.mr = c->row_buffer ? c->mr() : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   for (int i = 0; i < n_layers; ++i) {
     const int layer = first_layer + i;
@@ -588,12 +604,18 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     ls.static_valid = c->static_valid[layer];
     ls.new_j = c->t_img[layer];
     ls.t_img = c->t_img[layer] + 1;
+    ls.acc = c->row_buffer ? c->d_acc(layer) : nullptr;
+    ls.sem_slot = c->sem_tokens(layer);
+    ls.t_sem = ls.sem_slot + 1;
   }
   if (cudaMemsetAsync(p.work, 0, 4, st) != cudaSuccess || launch_decode_layers(p, st) != cudaSuccess) {
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }
-  for (int i = 0; i < n_layers; ++i) c->t_img[first_layer + i] += 1;
+  for (int i = 0; i < n_layers; ++i) {
+    c->t_img[first_layer + i] += 1;
+    c->pending[first_layer + i] = 0;   // this step's weights are already in the scores
+  }
   c->last_writer = -2;                 // several layers' slabs were written
   return SSD_OK;
 }

@@ -701,6 +701,8 @@ struct Unit {
   int fresh;                    // valid-slot index of the token being appended
   int phys;                     // and its slot counted from the head's first slot
   int contig;                   // the valid slots are one physical run
+  int u;                        // the unit's number
+  int scored;                   // 1: a semantic head whose attention scores are accumulated (Algorithm 2)
 };
 
 __device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Unit& U) {
@@ -709,11 +711,14 @@ __device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Un
   const int seq = pair / p.H, head = pair - seq * p.H;
   const LayerState& ls = p.layer[layer];
   const HeadDesc d = __ldg(ls.desc + head);
-  const int r = ls.new_j % d.z;
+  U.u = u;
+  U.scored = (ls.acc != nullptr && d.w) ? 1 : 0;
+  const int held = U.scored ? ls.t_sem : ls.t_img;          // tokens the ring holds
+  const int r = U.scored ? ls.sem_slot : ls.new_j % d.z;    // ring slot of the token being appended
   U.pv = ls.prompt_valid;
   U.sv = d.w ? ls.static_valid : 0;
   U.y = d.y;
-  U.vh = U.pv + U.sv + (ls.t_img < d.z ? ls.t_img : d.z);
+  U.vh = U.pv + U.sv + (held < d.z ? held : d.z);
   U.fresh = U.pv + U.sv + r;
   U.phys = p.L + d.y + r;
   U.contig = (U.pv == p.L && U.sv == d.y) ? 1 : 0;
@@ -733,6 +738,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
   const uint32_t ring_s = smem_u32(ring);
   const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
   volatile int* fifo = reinterpret_cast<volatile int*>(smem + kRingBytes + kWarps * kStages * 8) + warp * 4;
+  // row-buffer mode: the logits of the head being streamed, entry e = static slot e or, from the
+  // static capacity on, buffer slot e - capacity (the layout of the score rows)
+  float* lgbuf = reinterpret_cast<float*>(smem + kLayersSmemBytes) + (size_t)warp * ((p.mr + 3) & ~3);
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -823,7 +831,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
   uint32_t parity = 0;
   float2 q[8];
   State st;
-  const LogitSink sink = {nullptr, 0, 0, 0, 0};
+  LogitSink sink = {nullptr, 0, 0, 0, 0};
   bool begin = true;
 
 #pragma unroll 1
@@ -854,7 +862,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
       q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
       state_init(st);
       begin = false;
+      sink.row = CU.scored ? lgbuf : nullptr;
+      sink.skip = CU.pv;
+      sink.ring_from = CU.pv + CU.sv;
+      sink.ring_shift = CU.y - CU.sv;
     }
+    sink.i0 = ci;
     Rows rows;
     load_stage(sb, n, grp, l8, rows);
     {
@@ -876,9 +889,45 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
       state_merge_lane(tot, 8);
       state_merge_lane(tot, 16);
       if (grp == 0) write_out(reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<unsigned char*>(p.out) + CU.row), tot, l8);
+      if (CU.scored) {
+        // Algorithm 2, "accumulate semantic attention scores": this warp saw the whole head, so the
+        // normalised weights go straight into the head's score row (which no other warp touches;
+        // additions without a return value, so nothing waits for them).  The token appended in this
+        // step starts its score here.
+        __syncwarp();                    // the logits written by the group leaders, for every lane
+        const int pairs = p.n_seqs * p.H, layer = CU.u / pairs;
+        float* acc = p.layer[layer].acc + (size_t)(CU.u - layer * pairs) * p.mr;
+        const float inv = 1.f / tot.l;
+        const int n_scored = CU.vh - CU.pv, e_new = CU.phys - p.L;     // entries that hold a token; the new one
+        for (int i = lane; i < n_scored; i += 32) {
+          const int e = i < CU.sv ? i : CU.y + (i - CU.sv);
+          const float w = ex2(lgbuf[e] - tot.m) * inv;
+          if (e == e_new) acc[e] = w;
+          else atomicAdd(acc + e, w);
+        }
+        __syncwarp();                    // before the next head's logits overwrite the buffer
+      }
       begin = true;
     }
     if (++stage == kStages) { stage = 0; parity ^= 1u; }
+  }
+}
+
+// acc += exp2(logit - max) / sum over the entries that held a token at the layer's last decode
+__global__ void __launch_bounds__(256) ssd_fold_pending_kernel(float* acc, const float* logits, const float2* ml,
+                                                               const HeadDesc* desc, int n_pairs, int H, int mr,
+                                                               int static_valid, int buffered) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= n_pairs) return;
+  const HeadDesc d = desc[warp % H];
+  if (!d.w) return;
+  float* a = acc + (size_t)warp * mr;
+  const float* lg = logits + (size_t)warp * mr;
+  const float2 s = ml[warp];
+  const float inv = 1.f / s.y;
+  for (int i = lane; i < static_valid + buffered; i += 32) {
+    const int c = i < static_valid ? i : d.y + (i - static_valid);
+    a[c] += ex2(lg[c] - s.x) * inv;
   }
 }
 
@@ -965,6 +1014,18 @@ cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
   return e;
 }
 
+// Longest score row (M + R) whose logits a warp of the one-launch kernel can keep in shared memory.
+int decode_layers_max_mr() { return ((227 * 1024 - kLayersSmemBytes) / (kWarps * 4)) & ~3; }
+
+cudaError_t launch_fold_pending(float* acc, const float* logits, const float2* ml, const HeadDesc* desc, int n_seqs,
+                                int H, int mr, int static_valid, int buffered, cudaStream_t st) {
+  const int pairs = n_seqs * H;
+  ssd_fold_pending_kernel<<<(pairs * 32 + 255) / 256, 256, 0, st>>>(acc, logits, ml, desc, pairs, H, mr, static_valid,
+                                                                    buffered);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   static bool smem_set[64] = {};
   static int n_sm[64] = {};
@@ -974,7 +1035,8 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   const bool cached = dev >= 0 && dev < 64;
   int sms = cached ? n_sm[dev] : 0;
   if (!cached || !smem_set[dev]) {
-    e = cudaFuncSetAttribute(ssd_decode_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kLayersSmemBytes);
+    e = cudaFuncSetAttribute(ssd_decode_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kLayersSmemBytes + kWarps * decode_layers_max_mr() * 4);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     if (cached) {
@@ -984,9 +1046,11 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   }
   const long units = (long)p.n_layers * p.n_seqs * p.H;
   if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  if (p.mr < 0 || p.mr > decode_layers_max_mr()) return cudaErrorInvalidValue;
   const long want = (units + kWarps - 1) / kWarps;            // no more CTAs than there are units for
   const int grid = (int)(want < sms ? want : sms);
-  ssd_decode_layers_kernel<<<grid, kWarps * 32, kLayersSmemBytes, st>>>(p);
+  const int smem = kLayersSmemBytes + kWarps * ((p.mr + 3) & ~3) * 4;
+  ssd_decode_layers_kernel<<<grid, kWarps * 32, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }

@@ -56,6 +56,10 @@ struct LayerState {
   int static_valid;         // valid static slots of semantic heads
   int t_img;                // image tokens held, the one being appended included
   int new_j;                // image index of the token being appended
+  // row-buffer mode (Algorithm 2): the rings of semantic heads are buffers filled from slot 0
+  float* acc;               // [n_seqs * H, M + R] accumulated attention scores; null outside that mode
+  int t_sem;                // tokens in those buffers, the one being appended included
+  int sem_slot;             // buffer slot of the token being appended
 };
 struct DecodeLayersParams {
   uint4* slab;              // slot 0 of the slab
@@ -66,6 +70,7 @@ struct DecodeLayersParams {
   uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
   uint32_t* work;           // next unit to hand out; zero at launch
   int n_layers, n_seqs, H, L;
+  int mr;                   // M + R: entries of a head's score row (row-buffer mode)
   float scale_log2;
   LayerState layer[kMaxLayersPerLaunch];
 };
@@ -130,6 +135,11 @@ struct ClassifyParams {
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st);
+// acc += the normalised weights of the layer's last decode (its logits and (max, exp-sum) are in
+// `logits` and `ml`): what the next append of the row-buffer mode would do first
+cudaError_t launch_fold_pending(float* acc, const float* logits, const float2* ml, const HeadDesc* desc, int n_seqs,
+                                int H, int mr, int static_valid, int buffered, cudaStream_t st);
+int decode_layers_max_mr();
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);

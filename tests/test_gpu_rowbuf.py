@@ -47,7 +47,9 @@ def _run(cfg, layer, seqs, t_end, fused=False):
     outs = []
     for t in range(n0 + 1, t_end + 1):
         kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
-        if fused and t % 3:              # mostly the single launch, now and then the two calls
+        if fused == "layers" and t % 3:  # the one-launch form (accumulates the scores itself), and after
+            o = cache.append_decode_layers(0, kt[None], vt[None], qt[None])[0]    # every two of them the two calls
+        elif fused and t % 3:            # mostly the single launch, now and then the two calls
             o = cache.append_decode(0, kt, vt, qt)
         else:
             cache.append(0, kt, vt)
@@ -84,13 +86,13 @@ def _run(cfg, layer, seqs, t_end, fused=False):
     return n_band[0]
 
 
-@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("fused", [False, True, "layers"])
 def test_rowbuf_tiny_every_step(fused):
     cfg = wl.CONFIGS["tiny"]
     _run(cfg, 0, [0], cfg.n_img, fused)
 
 
-@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("fused", [False, True, "layers"])
 def test_rowbuf_janus1b_slice(fused):
     cfg = wl.CONFIGS["janus1b"]
     _run(cfg, 3, [0, 1], cfg.n0 + 3 * cfg.sink_recent + 5, fused)
@@ -109,8 +111,10 @@ def test_rowbuf_scores_match_oracle_before_reselection():
     cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
     for t in range(n0 + 1, n0 + R + 1):
         kt, vt, qt = (x.contiguous() for x in (k[:, :, L + t - 1], v[:, :, L + t - 1], q[:, :, t - 1]))
-        if t % 2:
+        if t % 3 == 0:
             cache.append_decode(0, kt, vt, qt)
+        elif t % 3 == 1:
+            cache.append_decode_layers(0, kt[None], vt[None], qt[None])
         else:
             cache.append(0, kt, vt)
             cache.decode_attn(0, qt)
