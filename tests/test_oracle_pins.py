@@ -391,3 +391,44 @@ def test_rowbuf_promotes_a_heavily_attended_buffer_token():
     t, static, acc, buf, _ = hist[-1]
     assert n0 in static and 0 in static and buf == []
     assert abs(acc[static.index(n0)] - R) < 1e-9              # R steps of weight ~1 each
+
+
+# ------------------------------------------------------------------ stored closed-form values
+def test_golden_closed_forms():
+    """tests/golden/closed_forms.txt holds values fixed by the definitions (Sec. 3.3 metric, Algorithm 1
+    running sum) under uniform or one-token attention, evaluated in exact rational arithmetic by the
+    script beside it; the oracle must reproduce each of them."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "closed_forms.txt")
+    rng = np.random.default_rng(11)
+    D, n_checked = 8, 0
+    for ln in open(path):
+        f = ln.split()
+        if not f or f[0].startswith("#"):
+            continue
+        want = float(f[-1])
+        if f[0] in ("sparsity_uniform", "sparsity_token0"):
+            N, w = int(f[1]), int(f[2])
+            L = 3
+            if f[0] == "sparsity_uniform":
+                Q = bf16(np.zeros((1, 1, 1, N, D)))
+                K = rand_bf16(rng, 1, 1, 1, L + N, D)
+            else:
+                # every query points at image token 0's key, far more strongly than at any other key
+                K = np.zeros((L + N, D))
+                K[L, 0] = 64.0
+                K[L + 1:, 1] = 1.0
+                Q = np.zeros((N, D))
+                Q[:, 0] = 64.0
+                K, Q = bf16(K[None, None, None]), bf16(Q[None, None, None])
+            got = oracle.sparsity(Q, K, L, w)[0, 0]
+            assert abs(got - want) < (1e-12 if f[0] == "sparsity_uniform" else 1e-9), (ln, got)
+        elif f[0] == "score_uniform":
+            L, n0, n_obs, j = (int(x) for x in f[1:5])
+            K = rand_bf16(rng, L + n0, D)
+            sc = oracle.scores(bf16(np.zeros((n_obs, D))), K, L, n0)
+            assert abs(sc[j] - want) < 1e-12, (ln, sc[j])
+        else:
+            raise AssertionError(f"unknown golden line: {ln}")
+        n_checked += 1
+    assert n_checked >= 14
