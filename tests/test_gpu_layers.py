@@ -108,3 +108,55 @@ def test_layers_launch_argument_errors():
     assert lib.ssd_append_decode_layers(c._h, 0, 2, x.data_ptr() + 2, *args[1:]) == B.SSD_ERR_INVALID_ARG   # misaligned
     assert B.kernel_launch_count() == before
     c.close()
+
+
+def test_janus7b_whole_step_launch_size_sampled_pairs():
+    """The launch the benchmark times: all 30 layers x 64 sequences x 32 heads of janus7b in one
+    launch.  The oracle recomputes sampled (layer, sequence, head) pairs one by one: their selected
+    sets (exact outside the tie band) and their outputs at three steps."""
+    from parity_util import MAX_ABS, MEAN_ABS, bf16_to_f64, check_index_sets
+    cfg = wl.CONFIGS["janus7b"]
+    dev = torch.device("cuda:0")
+    L, N, n0, W, M, R, H, S, NL = (cfg.prompt_len, cfg.n_img, cfg.n0, cfg.window, cfg.sink_budget, cfg.sink_recent,
+                                   cfg.n_heads, cfg.n_seqs, cfg.n_layers)
+    n_steps = 3
+    labels = np.stack([wl.sink_mask(cfg, l) for l in range(NL)])
+    rng = np.random.default_rng(42)
+    sample = {}
+    for i, layer in enumerate((0, 0, 9, 9, 17, 17, 29, 29)):
+        heads = np.nonzero(labels[layer] == (i % 2))[0]         # alternately a spatial and a semantic head
+        sample.setdefault(layer, []).append((int(rng.integers(0, S)), int(rng.choice(heads))))
+    cache = B.SsdCache(B.config_from_workload(cfg), n_sink_heads_total=int(labels.sum()), device=dev)
+    cache.set_head_labels(labels)
+    step_in = [torch.empty((n_steps, NL, S, H, 128), dtype=torch.bfloat16, device=dev) for _ in range(3)]
+    picked = {}
+    n_cand = max(n0 - R, 0)
+    for layer in range(NL):
+        q, k, v, _ = wl.gen_layer(cfg, layer, list(range(S)), device=dev)
+        cache.compress(layer, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        step_in[0][:, layer] = q[:, :, n0:n0 + n_steps].permute(2, 0, 1, 3)
+        step_in[1][:, layer] = k[:, :, L + n0:L + n0 + n_steps].permute(2, 0, 1, 3)
+        step_in[2][:, layer] = v[:, :, L + n0:L + n0 + n_steps].permute(2, 0, 1, 3)
+        if layer in sample:
+            gi = cache.get_indices(layer)
+            for (s, h) in sample[layer]:
+                qu, ku, vu = wl.to_u16(q[s, h]), wl.to_u16(k[s, h]), wl.to_u16(v[s, h])
+                sem = np.array([[labels[layer][h]]], np.uint8)
+                gidx = np.full((1, 1, M), -1, np.int32)
+                if labels[layer][h]:
+                    st = gi[s, h, L:L + M]
+                    gidx[0, 0] = np.where(st >= 0, st - L, -1)
+                    sc, oidx, ocnt = oracle.select_batch(qu[None, None, :n0], ku[None, None, : L + n0], sem, L, n0, M, R)
+                    check_index_sets(gidx, sc, oidx, ocnt, sem, n_cand, M)
+                picked[(layer, s, h)] = (qu, ku, vu, sem, gidx, (gidx >= 0).sum(-1).astype(np.int32))
+        del q, k, v
+    assert len(picked) == 8
+    for i in range(n_steps):
+        t = n0 + 1 + i
+        out = bf16_to_f64(cache.append_decode_layers(0, step_in[1][i], step_in[2][i], step_in[0][i]))
+        for (layer, s, h), (qu, ku, vu, sem, gidx, gcnt) in picked.items():
+            want = oracle.decode_batch(qu[None, None, t - 1], ku[None, None], vu[None, None], sem, gidx, gcnt, L, t, W, M, R)
+            err = np.abs(out[layer, s, h] - want[0, 0])
+            assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (layer, s, h, t, err.max())
+    assert cache.device_status() == 0
+    cache.close()
