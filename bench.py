@@ -462,8 +462,12 @@ def run_ours(args, cfg):
                     rcache.append_decode(layer, kk[i], vv[i], qq[i], out)
             rstate["i"] += 1
             if rstate["i"] % R == 0:
-                for layer in range(cfg.n_layers):
-                    rcache.recompress(layer)
+                if one_launch:
+                    for l0 in range(0, cfg.n_layers, 64):
+                        rcache.recompress_layers(l0, min(64, cfg.n_layers - l0))
+                else:
+                    for layer in range(cfg.n_layers):
+                        rcache.recompress(layer)
 
         ms_rb = {}
         for form in (False, True):    # per-layer launches (append, decode), then the one-launch step
@@ -476,6 +480,33 @@ def run_ours(args, cfg):
                   "device_status": rcache.device_status()}
         rcache.close()
         del rcache, rsteps
+        torch.cuda.empty_cache()
+        # Algorithm 1 taken literally: a re-selection after every step = a row buffer of one token with the
+        # same number of slots per head (M + R - 1 static, 1 buffered); two launches per step
+        import dataclasses
+        ecfg = dataclasses.replace(cfg, sink_budget=cfg.sink_budget + R - 1, sink_recent=1, name=cfg.name + "_evict_every_step")
+        Kv = min(K, 48)
+        ecache, _ = build_cache(ecfg, device, rank * S, rank, world, t_steps=Kv + 3, row_buffer=True, classify=False)
+        estate = {"i": 0}
+        eout = torch.empty((cfg.n_layers, S, H, 128), dtype=torch.bfloat16, device=device)
+
+        def ev_step():
+            i = estate["i"]
+            qq, kk, vv = ecache.step_all
+            for l0 in range(0, cfg.n_layers, 64):
+                l1 = min(l0 + 64, cfg.n_layers)
+                ecache.append_decode_layers(l0, kk[i, l0:l1], vv[i, l0:l1], qq[i, l0:l1], eout[l0:l1])
+                ecache.recompress_layers(l0, l1 - l0)
+            estate["i"] += 1
+
+        for _ in range(3):
+            ev_step()
+        ms_ev = max_over_ranks(timed(ev_step, Kv, barrier))
+        rowbuf["evict_every_step"] = {"value": cfg.images_per_step * world / (ms_ev / Kv * 1e-3), "unit": UNIT,
+                                      "ms_per_step": ms_ev / Kv, "steps": Kv, "sink_budget": ecfg.sink_budget,
+                                      "sink_recent": 1, "device_status": ecache.device_status()}
+        ecache.close()
+        del ecache
         torch.cuda.empty_cache()
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)

@@ -172,6 +172,11 @@ int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_la
  * token or belong to spatial heads.  Synchronises the device. */
 int ssd_cache_set_row_buffer(ssd_cache *cache, int32_t enable);
 int ssd_recompress(ssd_cache *cache, int32_t layer, void *stream);
+/* ssd_recompress for n_layers consecutive layers in one launch (same results, layer by layer).  With
+ * ssd_append_decode_layers this makes a step of the row-buffer mode two launches, and Algorithm 1's
+ * re-selection at every step (sink_recent = 1, one call per step) affordable.  SSD_ERR_LIMIT if
+ * n_layers > 64. */
+int ssd_recompress_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, void *stream);
 int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
 
 /* ssd_decode_attn for callers that cannot allocate.  The paper has no counterpart; this is a

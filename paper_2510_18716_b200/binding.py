@@ -26,7 +26,7 @@ SSD_ERR_LIMIT = -6
 EXPORTS = [
     "ssd_status_string", "ssd_cache_required_bytes", "ssd_cache_create", "ssd_cache_free",
     "ssd_classify_heads", "ssd_classify_partial", "ssd_set_head_labels", "ssd_compress", "ssd_append",
-    "ssd_decode_attn", "ssd_append_decode_layers", "ssd_step_host", "ssd_step_host_layers", "ssd_cache_get_indices", "ssd_cache_max_slots",
+    "ssd_decode_attn", "ssd_append_decode_layers", "ssd_recompress_layers", "ssd_step_host", "ssd_step_host_layers", "ssd_cache_get_indices", "ssd_cache_max_slots",
     "ssd_cache_get_lengths", "ssd_cache_get_labels", "ssd_cache_tokens", "ssd_cache_rewind",
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
@@ -83,6 +83,7 @@ def load():
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_append_decode_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    L.ssd_recompress_layers.argtypes = [vp, i32, i32, vp]
     L.ssd_step_host_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_get_indices.argtypes = [vp, i32, vp]
     L.ssd_cache_max_slots.argtypes = [vp]
@@ -274,6 +275,9 @@ class SsdCache:
 
     def recompress(self, layer: int):
         self._check(self.lib.ssd_recompress(self._h, layer, _stream()), "ssd_recompress")
+
+    def recompress_layers(self, first_layer: int, n_layers: int):
+        self._check(self.lib.ssd_recompress_layers(self._h, first_layer, n_layers, _stream()), "ssd_recompress_layers")
 
     def get_scores(self, layer: int) -> np.ndarray:
         c = self.cfg

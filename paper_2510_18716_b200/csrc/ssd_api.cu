@@ -828,6 +828,47 @@ int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
   return SSD_OK;
 }
 
+int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, void* stream) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
+  if (n_layers > kMaxLayersPerLaunch) return SSD_ERR_LIMIT;
+  if (!c->labels_set || !c->row_buffer) return SSD_ERR_BAD_STATE;
+  RecompressLayersParams p;
+  p.slab = reinterpret_cast<uint4*>(c->base + c->reg.slab);
+  p.desc = c->d_desc(first_layer);
+  p.static_idx = c->d_idx(first_layer);
+  p.acc = c->d_acc(first_layer);
+  p.logits = c->d_logits(first_layer);
+  p.ml = c->d_ml(first_layer);
+  p.n_layers = n_layers; p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len; p.M = g.sink_budget; p.mr = c->mr();
+  bool any = false;
+  for (int i = 0; i < n_layers; ++i) {
+    const int layer = first_layer + i;
+    RecompressLayer& ly = p.layer[i];
+    ly.first_slot = c->layer_base[layer];
+    ly.seq_slots = c->seq_slots[layer];
+    ly.static_valid = c->static_valid[layer];
+    ly.buffered = c->sem_tokens(layer);
+    ly.t_base = c->t_base[layer];
+    ly.pending = c->pending[layer];
+    ly.todo = (c->n_sink[layer] > 0 && (ly.buffered > 0 || ly.pending)) ? 1 : 0;
+    any = any || ly.todo;
+  }
+  if (any && launch_recompress_layers(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  for (int i = 0; i < n_layers; ++i) {
+    const int layer = first_layer + i;
+    if (p.layer[i].todo) {
+      const int n = c->static_valid[layer] + p.layer[i].buffered;
+      c->static_valid[layer] = n < g.sink_budget ? n : g.sink_budget;
+    }
+    c->t_base[layer] = c->t_img[layer];
+    c->pending[layer] = 0;
+  }
+  c->last_writer = -2;
+  return SSD_OK;
+}
+
 int ssd_cache_get_scores(ssd_cache* c, int32_t layer, float* acc_host) {
   if (!c || !acc_host) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;

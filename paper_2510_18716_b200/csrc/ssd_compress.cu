@@ -141,12 +141,11 @@ __global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams
 // shared memory in ascending batches, so no source is overwritten before it is read.
 constexpr int kMoveBatch = 32;
 
-__global__ void __launch_bounds__(kThreads) ssd_recompress_kernel(const RecompressParams p) {
+__device__ __forceinline__ void recompress_pair(const RecompressParams& p, int pair) {
   extern __shared__ __align__(16) unsigned char rsm[];
   __shared__ uint32_t s_hist[256];
   __shared__ uint32_t s_prefix, s_need;
   __shared__ int s_count;
-  const int pair = blockIdx.x;
   const int seq = pair / p.H, head = pair - seq * p.H;
   const HeadDesc d = p.desc[head];
   if (!d.w) return;
@@ -232,13 +231,17 @@ __global__ void __launch_bounds__(kThreads) ssd_recompress_kernel(const Recompre
   uint4* hbase = p.slab + ((size_t)seq * p.seq_slots + d.x + p.L) * kSlotU4;
   for (int o0 = 0; o0 < kept; o0 += kMoveBatch) {
     const int nb = min(kMoveBatch, kept - o0);
+    // a kept static row that no dropped row precedes is already where it belongs (candidate c of the
+    // static set sits in slot c): neither read nor written
     for (int r = warp; r < nb; r += kThreads / 32) {
       const int c = s_keep[o0 + r];
+      if (c == o0 + r) continue;
       const int e = c < p.static_valid ? c : d.y + (c - p.static_valid);
       s_rows[r * 32 + lane] = hbase[(size_t)e * kSlotU4 + lane];
     }
     __syncthreads();
-    for (int r = warp; r < nb; r += kThreads / 32) hbase[(size_t)(o0 + r) * kSlotU4 + lane] = s_rows[r * 32 + lane];
+    for (int r = warp; r < nb; r += kThreads / 32)
+      if (s_keep[o0 + r] != o0 + r) hbase[(size_t)(o0 + r) * kSlotU4 + lane] = s_rows[r * 32 + lane];
     __syncthreads();
   }
   for (int r = 0; r < 2; ++r) {
@@ -246,6 +249,30 @@ __global__ void __launch_bounds__(kThreads) ssd_recompress_kernel(const Recompre
     if (o < kept) { acc[o] = my_sc[r]; idx[o] = my_pos[r]; }
   }
   for (int o = kept + tid; o < p.M; o += kThreads) idx[o] = -1;
+}
+
+__global__ void __launch_bounds__(kThreads) ssd_recompress_kernel(const RecompressParams p) { recompress_pair(p, blockIdx.x); }
+
+// One CTA per (pair, layer): blockIdx.y is the layer.
+__global__ void __launch_bounds__(kThreads) ssd_recompress_layers_kernel(const __grid_constant__ RecompressLayersParams q) {
+  const int layer = blockIdx.y;
+  const RecompressLayer& ly = q.layer[layer];
+  if (!ly.todo) return;
+  const size_t pairs = (size_t)q.n_seqs * q.H;
+  RecompressParams p;
+  p.slab = q.slab + (size_t)ly.first_slot * kSlotU4;
+  p.desc = q.desc + (size_t)layer * q.H;
+  p.static_idx = q.static_idx + (size_t)layer * pairs * (q.M > 0 ? q.M : 1);
+  p.acc = q.acc + (size_t)layer * pairs * q.mr;
+  p.logits = q.logits + (size_t)layer * pairs * q.mr;
+  p.ml = q.ml + (size_t)layer * pairs;
+  p.pending = ly.pending;
+  p.n_seqs = q.n_seqs; p.H = q.H; p.L = q.L; p.M = q.M; p.mr = q.mr;
+  p.static_valid = ly.static_valid;
+  p.buffered = ly.buffered;
+  p.t_base = ly.t_base;
+  p.seq_slots = ly.seq_slots;
+  recompress_pair(p, blockIdx.x);
 }
 
 }  // namespace
@@ -259,6 +286,16 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st) {
   dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
   ssd_gather_kernel<<<grid, kThreads, 0, st>>>(p, max_slots);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream_t st) {
+  if (p.M > 2 * kThreads || p.n_layers < 1 || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  const size_t smem = (size_t)(3 * p.mr + 4) * 4 + (size_t)kMoveBatch * 512;
+  cudaError_t e = cudaFuncSetAttribute(ssd_recompress_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  ssd_recompress_layers_kernel<<<dim3(p.n_seqs * p.H, p.n_layers), kThreads, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }

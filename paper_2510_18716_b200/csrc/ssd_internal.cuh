@@ -159,6 +159,24 @@ struct RecompressParams {
   int seq_slots;
 };
 cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st);
+// The same for several layers in one launch: what differs from layer to layer, and the first layer's
+// tables (a layer's tables follow the previous layer's at fixed strides).
+struct RecompressLayer {
+  long long first_slot;        // the layer's first slot in the slab
+  int seq_slots, static_valid, buffered, t_base, pending;
+  int todo;                    // 0: nothing buffered and nothing pending in this layer
+};
+struct RecompressLayersParams {
+  uint4* slab;                 // slot 0 of the slab
+  const HeadDesc* desc;        // first layer's [H] records; next layer H records further
+  int32_t* static_idx;         // first layer's [n_seqs, H, M]
+  float* acc;                  // first layer's [n_seqs * H, mr]
+  const float* logits;
+  const float2* ml;
+  int n_layers, n_seqs, H, L, M, mr;
+  RecompressLayer layer[kMaxLayersPerLaunch];
+};
+cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream_t st);
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st);
 int classify_rows_per_block();
 int decode_max_workers();

@@ -56,7 +56,10 @@ def _run(cfg, layer, seqs, t_end, fused=False):
             o = cache.decode_attn(0, qt)
         outs.append(o.float().cpu().numpy().astype(np.float64))
         if (t - n0) % R == 0:
-            cache.recompress(0)
+            if fused == "layers":
+                cache.recompress_layers(0, 1)
+            else:
+                cache.recompress(0)
             gi = cache.get_indices(0)
             for s in range(S):
                 for h in range(H):
@@ -146,3 +149,49 @@ def test_per_step_eviction_is_a_row_buffer_of_one():
     import dataclasses
     cfg = dataclasses.replace(wl.CONFIGS["tiny"], sink_recent=1, name="tiny_r1")
     _run(cfg, 0, [0], cfg.n0 + 20, fused=True)
+    _run(cfg, 0, [0], cfg.n0 + 20, fused="layers")     # one decode launch and one re-selection launch per step
+
+
+def test_recompress_layers_equals_per_layer_recompress():
+    """Three layers with different head layouts, two buffer cycles: the one-launch step with the
+    one-launch re-selection against per-layer calls; same static sets and (to rounding) same scores."""
+    cfg = wl.CONFIGS["tiny"]
+    dev = torch.device("cuda:0")
+    L, n0, M, R, H, NL, S = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.n_heads, 3, 2
+    rng = np.random.default_rng(9)
+    labels = np.stack([wl.sink_mask(cfg, 0), np.ones(H, np.uint8), rng.integers(0, 2, H).astype(np.uint8)])
+    data = [wl.gen_layer(cfg, l, [0, 1], device=dev) for l in range(NL)]
+    caches = []
+    for _ in range(2):
+        c = B.SsdCache(B.config_from_workload(cfg, n_layers=NL, n_seqs=S), device=dev)
+        c.set_row_buffer(True)
+        c.set_head_labels(labels)
+        for l, (q, k, v, _) in enumerate(data):
+            c.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(c)
+    a, b = caches
+    for t in range(n0 + 1, n0 + 2 * R + 1):
+        qs = torch.stack([data[l][0][:, :, t - 1] for l in range(NL)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + t - 1] for l in range(NL)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + t - 1] for l in range(NL)]).contiguous()
+        want = torch.stack([a.append_decode(l, ks[l], vs[l], qs[l]) for l in range(NL)])
+        got = b.append_decode_layers(0, ks, vs, qs)
+        d = (got.float() - want.float()).abs()
+        assert d.max().item() <= 2e-2 and d.mean().item() <= 5e-4
+        if (t - n0) % R == 0:
+            for l in range(NL):
+                a.recompress(l)
+            b.recompress_layers(0, NL)
+            for l in range(NL):
+                assert np.array_equal(a.get_indices(l), b.get_indices(l)), (t, l)
+                sa, sb = a.get_scores(l), b.get_scores(l)
+                assert np.array_equal(sa < 0, sb < 0)
+                assert np.allclose(sa, sb, rtol=1e-4, atol=1e-6)
+    lib = B.load()
+    st = torch.cuda.current_stream().cuda_stream
+    assert lib.ssd_recompress_layers(b._h, 2, 2, st) == B.SSD_ERR_INVALID_ARG
+    b.set_row_buffer(False)
+    assert lib.ssd_recompress_layers(b._h, 0, NL, st) == B.SSD_ERR_BAD_STATE
+    assert a.device_status() == 0 and b.device_status() == 0
+    for c in caches:
+        c.close()
