@@ -34,8 +34,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.83e6, "per_layer_of_step": 160.85e6,
-                  "sha256": "f230d96f3e2a86c5ed55eaf19eead62edea9e2450c4e68145cb27b99a82baf00"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.16e6, "per_layer_of_step": 160.75e6,
+                  "sha256": "f642104b48bfedb3baf6c1d8a883ee1807c03f9b22d78d7fc126426296b2dabe"}
 
 
 def decode_traffic(cfg):
