@@ -163,8 +163,10 @@ int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_la
  *                    of the static and buffered tokens of semantic heads; they are added to the tokens'
  *                    accumulated scores by the layer's next ssd_append or ssd_recompress;
  *   ssd_recompress   ("row buffer full"): per (sequence, semantic head) keeps the top-M of static set +
- *                    buffer by accumulated score (ties: lowest position) as the new static set, in
- *                    ascending position, and empties the buffer.  Asynchronous.
+ *                    buffer by accumulated score (ties: lowest position) as the new static set and
+ *                    empties the buffer.  Tokens that stay keep their slots; tokens that enter take
+ *                    the slots of those that leave, so static slots are in ascending position only
+ *                    until the first re-selection.  Asynchronous.
  * Spatial heads keep exactly their W newest tokens in both modes.  ssd_cache_set_row_buffer switches the
  * mode and resets every layer to the empty state (call it before ssd_compress).
  * ssd_cache_get_scores: acc_host [n_seqs, n_heads, M + R] accumulated scores, entry e < M for static
@@ -225,7 +227,8 @@ int ssd_step_host_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers
 
 /* Absolute positions held by each slot of a layer, for inspection and index-set parity:
  * idx_host [n_seqs, n_heads, max_slots] int32 with max_slots = ssd_cache_max_slots(); slots are
- * ordered prompt, static (ascending position), ring (physical ring order); -1 = empty or unused.
+ * ordered prompt, static (ascending position after ssd_compress; slot order after re-selections
+ * in row-buffer mode), ring (physical ring order); -1 = empty or unused.
  * Synchronises the device. */
 int ssd_cache_get_indices(ssd_cache *cache, int32_t layer, int32_t *idx_host);
 int32_t ssd_cache_max_slots(const ssd_cache *cache); /* prompt_len + max(window, M + R) */

@@ -17,6 +17,27 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Selection among few candidates without a radix pass: candidate c is kept iff fewer than k
+// candidates come before it in the order (score descending, then position ascending); its rank is
+// counted directly (n * n / kThreads comparisons per thread, all reading the same shared-memory
+// word at a time).  bits[]: the scores' bit patterns (non-negative floats order like unsigned
+// integers); pos == nullptr means a candidate's position is its index.
+constexpr int kRankMax = 1024;
+
+__device__ __forceinline__ void rank_select(const uint32_t* bits, const int* pos, int n, int k, int* flag) {
+  for (int c = threadIdx.x; c < n; c += kThreads) {
+    const uint32_t b = bits[c];
+    const int pc = pos ? pos[c] : c;
+    int rank = 0;
+    for (int j = 0; j < n; ++j) {
+      const uint32_t bj = bits[j];
+      const int pj = pos ? pos[j] : j;
+      rank += (bj > b || (bj == b && pj < pc)) ? 1 : 0;
+    }
+    flag[c] = rank < k ? 1 : 0;
+  }
+}
+
 // ----------------------------------------------------------------------------- select
 // One CTA per (sequence, semantic head): radix-select the k-th largest score (scores are
 // non-negative floats, so their bit patterns order like unsigned integers), then emit, in
@@ -36,6 +57,30 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
   for (int i = tid; i < p.M; i += kThreads) out[i] = -1;
   if (k <= 0) return;
   __syncthreads();
+  float* acc_row = p.acc ? p.acc + (size_t)pair * p.mr : nullptr;   // row-buffer mode: scores travel with the tokens
+  if (n <= kRankMax) {
+    __shared__ uint32_t s_bits[kRankMax];
+    __shared__ int s_flag[kRankMax];
+    for (int i = tid; i < n; i += kThreads) s_bits[i] = sc[i];
+    __syncthreads();
+    rank_select(s_bits, nullptr, n, k, s_flag);
+    __syncthreads();
+    if (tid < 32) {                    // ordered compaction by one warp
+      int cnt = 0;
+      for (int c0 = 0; c0 < n; c0 += 32) {
+        const int c = c0 + tid;
+        const bool take = c < n && s_flag[c];
+        const unsigned m = __ballot_sync(0xffffffffu, take);
+        if (take) {
+          const int o = cnt + __popc(m & ((1u << tid) - 1u));
+          out[o] = c;
+          if (acc_row) acc_row[o] = __uint_as_float(s_bits[c]);
+        }
+        cnt += __popc(m);
+      }
+    }
+    return;
+  }
 
   // find the bit pattern of the k-th largest candidate
   if (tid == 0) { s_prefix = 0u; s_need = (uint32_t)k; }
@@ -85,7 +130,7 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
   }
   __syncthreads();
   uint32_t g_before = s_gt[tid], e_before = s_eq[tid];
-  float* acc = p.acc ? p.acc + (size_t)pair * p.mr : nullptr;   // row-buffer mode: scores travel with the tokens
+  float* acc = acc_row;
   for (int i = a; i < b; ++i) {
     uint32_t v = sc[i];
     if (v > thr) {
@@ -134,47 +179,53 @@ __global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams
 
 // ----------------------------------------------------------------------------- recompress
 // Algorithm 2, "row buffer full": for every (sequence, semantic head) keep the top-M of the static
-// set plus the buffered tokens by accumulated attention score (ties: lowest position), in ascending
-// position, as the new static set; the buffer is then empty.  One CTA per pair.  Candidates are
-// already in ascending position (static slots, then buffer slots), so selection is an ordered
-// compaction, done in place: a kept row never moves to a higher slot, and rows are moved through
-// shared memory in ascending batches, so no source is overwritten before it is read.
-constexpr int kMoveBatch = 32;
-
+// set plus the buffered tokens by accumulated attention score (ties: lowest position) as the new
+// static set; the buffer is then empty.  One CTA per pair.  Static tokens that stay keep their
+// slots; the buffered tokens that make it take the slots of the static tokens that do not (and the
+// still unused static slots), in ascending slot order.  So only the tokens that enter move (at most
+// R rows per head, from the ring region into the static region: sources and destinations never
+// overlap), and after the first re-selection the static slots are no longer ordered by position,
+// which nothing depends on: ties are broken on the positions themselves.
 __device__ __forceinline__ void recompress_pair(const RecompressParams& p, int pair) {
   extern __shared__ __align__(16) unsigned char rsm[];
   __shared__ uint32_t s_hist[256];
   __shared__ uint32_t s_prefix, s_need;
-  __shared__ int s_count;
+  __shared__ int s_nt, s_nsrc;
   const int seq = pair / p.H, head = pair - seq * p.H;
   const HeadDesc d = p.desc[head];
   if (!d.w) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n = p.static_valid + p.buffered;          // candidates
+  const int sv = p.static_valid;
+  const int n = sv + p.buffered;                       // candidates: static slots, then buffer slots
   const int k = min(p.M, n);
-  float* s_sc = reinterpret_cast<float*>(rsm);         // [mr] candidate scores, candidate order
+  float* s_sc = reinterpret_cast<float*>(rsm);         // [mr] candidate scores
   int* s_pos = reinterpret_cast<int*>(s_sc + p.mr);    // [mr] candidate image indices
-  int* s_keep = s_pos + p.mr;                          // [mr] kept candidates, ascending
-  uint4* s_rows = reinterpret_cast<uint4*>(s_keep + p.mr + ((4 - (3 * p.mr) % 4) % 4));   // [kMoveBatch][32]
+  int* s_flag = s_pos + p.mr;                          // [mr] 1 = kept
+  int* s_tie = s_flag + p.mr;                          // [mr] candidates whose score equals the threshold
+  int* s_src = s_tie + p.mr;                           // [mr] kept buffered candidates, buffer order
+  int* s_dst = s_src + p.mr;                           // [mr] free static slots, ascending
   float* acc = p.acc + (size_t)pair * p.mr;
   int32_t* idx = p.static_idx + (size_t)pair * p.M;
 
   // candidate c lives in entry e(c) of the score row and of the head's static+ring slots
   for (int c = tid; c < n; c += kThreads) {
-    const int e = c < p.static_valid ? c : d.y + (c - p.static_valid);
+    const int e = c < sv ? c : d.y + (c - sv);
     float sc = acc[e];
     if (p.pending) {
       const float2 ml = p.ml[pair];
       sc += ex2(p.logits[(size_t)pair * p.mr + e] - ml.x) / ml.y;
     }
     s_sc[c] = sc;
-    s_pos[c] = c < p.static_valid ? idx[c] : p.t_base + (c - p.static_valid);
+    s_pos[c] = c < sv ? idx[c] : p.t_base + (c - sv);
   }
+  if (tid == 0) { s_prefix = 0u; s_need = (uint32_t)k; s_nt = 0; s_nsrc = 0; }
   __syncthreads();
 
-  // bit pattern of the k-th largest score (scores are non-negative)
   const uint32_t* bits = reinterpret_cast<const uint32_t*>(s_sc);
-  if (tid == 0) { s_prefix = 0u; s_need = (uint32_t)k; s_count = 0; }
+  if (n <= kRankMax) {
+    rank_select(bits, s_pos, n, k, s_flag);
+  } else {
+  // bit pattern of the k-th largest score (scores are non-negative)
   for (int shift = 24; shift >= 0; shift -= 8) {
     s_hist[tid] = 0u;
     __syncthreads();
@@ -197,58 +248,65 @@ __device__ __forceinline__ void recompress_pair(const RecompressParams& p, int p
     }
     __syncthreads();
   }
-  // ordered compaction by one warp: above the threshold, or equal to it among the first s_need such
-  if (warp == 0) {
-    const uint32_t thr = s_prefix;
-    uint32_t eq_left = s_need;
-    int kept = 0;
-    for (int c0 = 0; c0 < n; c0 += 32) {
-      const int c = c0 + lane;
-      const uint32_t b = c < n ? bits[c] : 0u;
-      const bool gt = c < n && b > thr, eq = c < n && b == thr;
-      const unsigned eq_mask = __ballot_sync(0xffffffffu, eq);
-      const uint32_t eq_before = __popc(eq_mask & ((1u << lane) - 1u));
-      const bool take = gt || (eq && eq_before < eq_left);
-      const unsigned take_mask = __ballot_sync(0xffffffffu, take);
-      if (take) s_keep[kept + __popc(take_mask & ((1u << lane) - 1u))] = c;
-      kept += __popc(take_mask);
-      const uint32_t eq_taken = min((uint32_t)__popc(eq_mask), eq_left);
-      eq_left -= eq_taken;
-    }
-    if (lane == 0) s_count = kept;
+  const uint32_t thr = s_prefix;
+  const int need_eq = (int)s_need;
+
+  // above the threshold: kept; equal to it: the need_eq lowest positions (positions are distinct)
+  for (int c = tid; c < n; c += kThreads) {
+    const uint32_t b = bits[c];
+    s_flag[c] = b > thr ? 1 : 0;
+    if (b == thr) s_tie[atomicAdd(&s_nt, 1)] = c;
   }
   __syncthreads();
-  const int kept = s_count;                            // == k
+  const int nt = s_nt;
+  for (int i = tid; i < nt; i += kThreads) {
+    const int c = s_tie[i], pc = s_pos[c];
+    int rank = 0;
+    for (int j = 0; j < nt; ++j) rank += s_pos[s_tie[j]] < pc ? 1 : 0;
+    if (rank < need_eq) s_flag[c] = 1;
+  }
+  }
+  __syncthreads();
+
+  // who moves where: the j-th kept buffered token (buffer order) into the j-th free static slot
+  // (slots of dropped static tokens and slots never used so far, ascending); one warp, by ballots
+  if (warp == 0) {
+    int cnt = 0;
+    for (int c0 = sv; c0 < n; c0 += 32) {
+      const int c = c0 + lane;
+      const bool take = c < n && s_flag[c];
+      const unsigned m = __ballot_sync(0xffffffffu, take);
+      if (take) s_src[cnt + __popc(m & ((1u << lane) - 1u))] = c;
+      cnt += __popc(m);
+    }
+    if (lane == 0) s_nsrc = cnt;
+    cnt = 0;
+    for (int o0 = 0; o0 < p.M; o0 += 32) {
+      const int o = o0 + lane;
+      const bool free_slot = o < p.M && (o >= sv || !s_flag[o]);
+      const unsigned m = __ballot_sync(0xffffffffu, free_slot);
+      if (free_slot) s_dst[cnt + __popc(m & ((1u << lane) - 1u))] = o;
+      cnt += __popc(m);
+    }
+  }
+  __syncthreads();
+  const int nmove = s_nsrc;                            // free slots never run out: there are at least as many
 
   // scores and positions of the new static set
-  float my_sc[2];
-  int my_pos[2];
-  for (int r = 0; r < 2; ++r) {
-    const int o = tid + r * kThreads;
-    if (o < kept) { my_sc[r] = s_sc[s_keep[o]]; my_pos[r] = s_pos[s_keep[o]]; }
+  for (int c = tid; c < sv; c += kThreads)
+    if (s_flag[c]) acc[c] = s_sc[c];                   // with the last decode's weights folded in
+  for (int j = tid; j < nmove; j += kThreads) {
+    const int c = s_src[j], o = s_dst[j];
+    acc[o] = s_sc[c];
+    idx[o] = s_pos[c];
   }
-  // rows: slot of candidate c is L + e(c); destination of the o-th kept row is static slot o
+  for (int o = k + tid; o < p.M; o += kThreads) idx[o] = -1;
+  // rows of the tokens that enter: ring slot of buffer entry (c - sv) -> static slot
   uint4* hbase = p.slab + ((size_t)seq * p.seq_slots + d.x + p.L) * kSlotU4;
-  for (int o0 = 0; o0 < kept; o0 += kMoveBatch) {
-    const int nb = min(kMoveBatch, kept - o0);
-    // a kept static row that no dropped row precedes is already where it belongs (candidate c of the
-    // static set sits in slot c): neither read nor written
-    for (int r = warp; r < nb; r += kThreads / 32) {
-      const int c = s_keep[o0 + r];
-      if (c == o0 + r) continue;
-      const int e = c < p.static_valid ? c : d.y + (c - p.static_valid);
-      s_rows[r * 32 + lane] = hbase[(size_t)e * kSlotU4 + lane];
-    }
-    __syncthreads();
-    for (int r = warp; r < nb; r += kThreads / 32)
-      if (s_keep[o0 + r] != o0 + r) hbase[(size_t)(o0 + r) * kSlotU4 + lane] = s_rows[r * 32 + lane];
-    __syncthreads();
+  for (int j = warp; j < nmove; j += kThreads / 32) {
+    const int e = d.y + (s_src[j] - sv), o = s_dst[j];
+    hbase[(size_t)o * kSlotU4 + lane] = hbase[(size_t)e * kSlotU4 + lane];
   }
-  for (int r = 0; r < 2; ++r) {
-    const int o = tid + r * kThreads;
-    if (o < kept) { acc[o] = my_sc[r]; idx[o] = my_pos[r]; }
-  }
-  for (int o = kept + tid; o < p.M; o += kThreads) idx[o] = -1;
 }
 
 __global__ void __launch_bounds__(kThreads) ssd_recompress_kernel(const RecompressParams p) { recompress_pair(p, blockIdx.x); }
@@ -291,8 +349,8 @@ cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st)
 }
 
 cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream_t st) {
-  if (p.M > 2 * kThreads || p.n_layers < 1 || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
-  const size_t smem = (size_t)(3 * p.mr + 4) * 4 + (size_t)kMoveBatch * 512;
+  if (p.n_layers < 1 || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  const size_t smem = (size_t)(6 * p.mr + 4) * 4;
   cudaError_t e = cudaFuncSetAttribute(ssd_recompress_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   ssd_recompress_layers_kernel<<<dim3(p.n_seqs * p.H, p.n_layers), kThreads, smem, st>>>(p);
@@ -301,8 +359,7 @@ cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream
 }
 
 cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st) {
-  if (p.M > 2 * kThreads) return cudaErrorInvalidValue;      // each thread carries two kept entries
-  const size_t smem = (size_t)(3 * p.mr + 4) * 4 + (size_t)kMoveBatch * 512;
+  const size_t smem = (size_t)(6 * p.mr + 4) * 4;
   cudaError_t e = cudaFuncSetAttribute(ssd_recompress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   ssd_recompress_kernel<<<p.n_seqs * p.H, kThreads, smem, st>>>(p);

@@ -65,7 +65,10 @@ def _run(cfg, layer, seqs, t_end, fused=False):
                 for h in range(H):
                     if labels[h]:
                         st = gi[s, h, L:L + M]
-                        gpu_sets[(s, h, t)] = (st[st >= 0] - L).tolist()
+                        # tokens that stay keep their slots and the ones that enter take the freed ones, so
+                        # the static slots are not ordered by position after a re-selection: compare as sets
+                        gpu_sets[(s, h, t)] = sorted((st[st >= 0] - L).tolist())
+                        assert len(set(gpu_sets[(s, h, t)])) == len(gpu_sets[(s, h, t)])
                         ring = gi[s, h, L + M:L + M + R]
                         assert (ring == -1).all(), "the buffer is empty after a re-selection"
             assert (cache.get_lengths(0)[labels == 1] == L + min(M, t)).all()
