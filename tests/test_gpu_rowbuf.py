@@ -198,3 +198,14 @@ def test_recompress_layers_equals_per_layer_recompress():
     assert a.device_status() == 0 and b.device_status() == 0
     for c in caches:
         c.close()
+
+
+def test_rowbuf_more_than_1024_candidates_takes_the_radix_path():
+    """Up to 1024 candidates a re-selection counts ranks directly; above, it radix-selects the
+    threshold score and breaks ties on positions.  A head with M + R = 1108 exercises the second
+    path (and the score row of that length in the one-launch kernel), against the oracle."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], grid=(35, 40), n0=1200, sink_budget=1100, sink_recent=8,
+                              window=24, name="tiny_wide")
+    n = _run(cfg, 0, [0], cfg.n0 + 2 * cfg.sink_recent + 3, fused="layers")
+    assert n >= 0
