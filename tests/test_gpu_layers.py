@@ -34,7 +34,7 @@ def test_layers_launch_matches_per_layer_calls_and_oracle(case):
     if case == "janus7b_slice":
         cfg, nl, seqs, n_steps, kind = wl.CONFIGS["janus7b"], 3, list(range(6)), 20, "generator"
     else:
-        cfg, nl, seqs, n_steps, kind = wl.CONFIGS["tiny"], 4, [0, 1], 32, "mixed"
+        cfg, nl, seqs, n_steps, kind = wl.CONFIGS["tiny"], 4, [0, 1], 28, "mixed"
     L, N, n0, W, M, R, H, S = (cfg.prompt_len, cfg.n_img, cfg.n0, cfg.window, cfg.sink_budget, cfg.sink_recent,
                                cfg.n_heads, len(seqs))
     labels = _labels(cfg, kind, nl)
@@ -88,6 +88,21 @@ def test_layers_launch_matches_per_layer_calls_and_oracle(case):
             kt, vt, qt = (x.contiguous() for x in (data[l][1][:, :, L + t - 1], data[l][2][:, :, L + t - 1],
                                                    data[l][0][:, :, t - 1]))
             assert torch.equal(fused.append_decode(l, kt, vt, qt), per_layer.append_decode(l, kt, vt, qt))
+    # layers need not be at the same step: layer 0 runs one step ahead, then one launch serves them all
+    if t + 2 <= N:
+        step_of = [t + 2] + [t + 1] * (nl - 1)
+        kt, vt, qt = (x.contiguous() for x in (data[0][1][:, :, L + t], data[0][2][:, :, L + t], data[0][0][:, :, t]))
+        assert torch.equal(fused.append_decode(0, kt, vt, qt), per_layer.append_decode(0, kt, vt, qt))
+        qs = torch.stack([data[l][0][:, :, step_of[l] - 1] for l in range(nl)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + step_of[l] - 1] for l in range(nl)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + step_of[l] - 1] for l in range(nl)]).contiguous()
+        want = torch.stack([per_layer.append_decode(l, ks[l], vs[l], qs[l]) for l in range(nl)])
+        got = fused.append_decode_layers(0, ks, vs, qs)
+        d = (got.float() - want.float()).abs()
+        assert d.max().item() <= 2e-2 and d.mean().item() <= 5e-4
+        assert [fused.tokens(l) for l in range(nl)] == step_of == [per_layer.tokens(l) for l in range(nl)]
+        for l in range(nl):
+            assert np.array_equal(fused.get_indices(l), per_layer.get_indices(l))
     assert fused.device_status() == 0 and per_layer.device_status() == 0
     for c in caches:
         c.close()
