@@ -148,7 +148,7 @@ int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const 
  * nothing is left pending for the next append or ssd_recompress; the per-layer calls and this one
  * can be mixed freely.
  * SSD_ERR_LIMIT if n_layers > 64 (issue several calls) or, in row-buffer mode, if sink_budget +
- * sink_recent exceeds what a warp can keep in shared memory (about 2800);  SSD_ERR_OVERFLOW (nothing
+ * sink_recent exceeds what a warp can keep in shared memory (about 3000);  SSD_ERR_OVERFLOW (nothing
  * launched) if any of the layers, or its row buffer, is full.  Asynchronous. */
 int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *k_new,
                              const void *v_new, const void *q, void *out, void *stream);
