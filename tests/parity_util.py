@@ -79,7 +79,7 @@ class RunResult:
 
 
 def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, full_every_step=False,
-                 n_obs=None, check_planted=False, device="cuda:0", labels_override=None) -> RunResult:
+                 n_obs=None, check_planted=False, device="cuda:0", labels_override=None, step_form="two") -> RunResult:
     """Drive the C-ABI path for `layers` x `seqs` of a workload and check every stage.
 
     The cache is created with len(layers) layers and len(seqs) sequences; layer i of the cache holds
@@ -135,10 +135,18 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
         # --- decode steps
         steps = list(range(n0 + 1, N + 1))
         for t in steps:
-            cache.append(li, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
+            kt, vt = k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous()
             if not (full_every_step or t in check_steps):
+                cache.append(li, kt, vt)
                 continue
-            out = cache.decode_attn(li, q[:, :, t - 1].contiguous())
+            qt = q[:, :, t - 1].contiguous()
+            if step_form == "fused":           # ssd_append_decode
+                out = cache.append_decode(li, kt, vt, qt)
+            elif step_form == "layers":        # ssd_append_decode_layers on this one layer
+                out = cache.append_decode_layers(li, kt[None], vt[None], qt[None])[0]
+            else:                              # ssd_append, ssd_decode_attn
+                cache.append(li, kt, vt)
+                out = cache.decode_attn(li, qt)
             # attention over the GPU's own (validated) index set, so band cases compare like with like
             want = oracle.decode_batch(qu[:, :, t - 1], ku, vu, sem, gidx, gcnt, L, t, W, M, R)
             errs.append(check_outputs(out, want, f"layer {layer} step {t}"))

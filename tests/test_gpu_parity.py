@@ -94,7 +94,8 @@ def test_random_small_shapes(seed):
     if cfg.prompt_len + cfg.n0 == 0:
         pytest.skip("nothing to load")
     run_workload(cfg, [0], list(range(cfg.n_seqs)), (), classify=False, full_every_step=True,
-                 n_obs=min(cfg.n0, seed % 5 + (cfg.n0 if seed % 2 else 0)))
+                 n_obs=min(cfg.n0, seed % 5 + (cfg.n0 if seed % 2 else 0)),
+                 step_form=("two", "fused", "layers")[seed % 3])      # every form of the step sees odd shapes
 
 
 def test_decode_before_any_compress_fills_ring_from_zero():
