@@ -261,8 +261,8 @@ def test_other_head_partitions(kind):
         elif kind == "all_semantic":
             lab = np.ones((len(layers), H), np.uint8)
         else:
-            rng = np.random.default_rng(123)
-            lab = np.stack([rng.permutation(wl.sink_mask(cfg, l)) for l in layers])
+            from paper_2510_18716_b200 import ablation
+            lab = ablation.random_partition(np.stack([wl.sink_mask(cfg, l) for l in layers]), seed=123)
         r = run_workload(cfg, layers, seqs, (cfg.n0 + 1, cfg.n0 + 9, cfg.n_img), classify=False, labels_override=lab)
         assert r.steps_checked == 3 * len(layers)
 
