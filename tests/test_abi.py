@@ -86,6 +86,14 @@ def test_null_and_bad_arguments_are_rejected_on_the_host():
     assert lib.ssd_append(None, 0, x.ctypes.data, x.ctypes.data, None) == B.SSD_ERR_INVALID_ARG
     assert lib.ssd_decode_attn(None, 0, x.ctypes.data, x.ctypes.data, None) == B.SSD_ERR_INVALID_ARG
     assert lib.ssd_compress(None, 0, None, x.ctypes.data, x.ctypes.data, 0, 0, None) == B.SSD_ERR_INVALID_ARG
+    p = x.ctypes.data
+    assert lib.ssd_append_decode(None, 0, p, p, p, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_append_decode_layers(None, 0, 1, p, p, p, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_step_host(None, 0, p, p, p, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_step_host_layers(None, 0, 1, p, p, p, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_recompress(None, 0, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_recompress_layers(None, 0, 1, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_decode_attn_static(None, 0, p, p, None) == B.SSD_ERR_INVALID_ARG
     assert lib.ssd_cache_max_slots(None) == -1
     assert lib.ssd_cache_tokens(None, 0) == -1
     assert isinstance(B.kernel_launch_count(), int)
