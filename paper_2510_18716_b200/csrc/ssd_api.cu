@@ -652,8 +652,11 @@ int ssd_step_host_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, co
   const ssd_config& g = c->cfg;
   if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
-  for (int i = 0; i < n_layers; ++i)
-    if (c->t_img[first_layer + i] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;   // before anything is enqueued
+  for (int i = 0; i < n_layers; ++i) {             // before anything is enqueued
+    const int layer = first_layer + i;
+    if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+    if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;
+  }
   if (!make_host_pipe(c)) return SSD_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t nb = (size_t)g.n_seqs * g.n_heads * kHeadDim * 2;

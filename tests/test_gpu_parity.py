@@ -50,7 +50,7 @@ def test_sweep_points():
         run_workload(cfg, [3], seqs, (cfg.n0 + 1, cfg.n0 + 30, cfg.n_img), classify=False)
 
 
-def _full_cache_case(cfg: wl.Workload, seqs, steps):
+def _full_cache_case(cfg: wl.Workload, seqs, steps, one_launch=False):
     """Uncompressed baseline: every head spatial with W = N, prompt loaded with n0 = 0."""
     dev = torch.device("cuda:0")
     L, N, H, S = cfg.prompt_len, cfg.n_img, cfg.n_heads, len(seqs)
@@ -62,18 +62,26 @@ def _full_cache_case(cfg: wl.Workload, seqs, steps):
     cache.compress(0, None, k[:, :, :L].contiguous(), v[:, :, :L].contiguous(), 0, 0)
     sem = np.zeros((S, H), np.uint8)
     for t in range(1, N + 1):
-        cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
-        if t in steps:
+        kt, vt = k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous()
+        if t not in steps:
+            cache.append(0, kt, vt)
+            continue
+        if one_launch:
+            out = cache.append_decode_layers(0, kt[None], vt[None], q[:, :, t - 1].contiguous()[None])[0]
+        else:
+            cache.append(0, kt, vt)
             out = cache.decode_attn(0, q[:, :, t - 1].contiguous())
-            want = oracle.decode_batch(qu[:, :, t - 1], ku, vu, sem, None, None, L, t, N, 0, 1, full=True)
-            check_outputs(out, want, f"full cache step {t}")
-            assert (cache.get_lengths(0) == L + t).all()
+        want = oracle.decode_batch(qu[:, :, t - 1], ku, vu, sem, None, None, L, t, N, 0, 1, full=True)
+        check_outputs(out, want, f"full cache step {t}")
+        assert (cache.get_lengths(0) == L + t).all()
     cache.close()
 
 
 def test_full_cache_baseline_matches_full_attention():
     _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65))
     _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576))
+    _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65), one_launch=True)
+    _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576), one_launch=True)
 
 
 def _small_cfg(seed):
