@@ -497,7 +497,7 @@ def run_ours(args, cfg):
         del rcache, rsteps
         torch.cuda.empty_cache()
         # Algorithm 1 taken literally: a re-selection after every step = a row buffer of one token with the
-        # same number of slots per head (M + R - 1 static, 1 buffered); two launches per step
+        # same number of slots per head (M + R - 1 static, 1 buffered)
         import dataclasses
         ecfg = dataclasses.replace(cfg, sink_budget=cfg.sink_budget + R - 1, sink_recent=1, name=cfg.name + "_evict_every_step")
         Kv = min(K, 48)
@@ -510,8 +510,8 @@ def run_ours(args, cfg):
             qq, kk, vv = ecache.step_all
             for l0 in range(0, cfg.n_layers, 64):
                 l1 = min(l0 + 64, cfg.n_layers)
+                # with a buffer of one token the launch re-selects as well: one launch per step
                 ecache.append_decode_layers(l0, kk[i, l0:l1], vv[i, l0:l1], qq[i, l0:l1], eout[l0:l1])
-                ecache.recompress_layers(l0, l1 - l0)
             estate["i"] += 1
 
         for _ in range(3):

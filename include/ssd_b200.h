@@ -147,8 +147,13 @@ int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const 
  * of semantic heads (a head is summed by one warp, which therefore holds all its weights), so
  * nothing is left pending for the next append or ssd_recompress; the per-layer calls and this one
  * can be mixed freely.
+ * With a row buffer of one token (sink_recent = 1) the launch re-selects too, which is Algorithm 1
+ * taken literally: after the step's attention the token just appended takes the place of the
+ * lowest-scoring static token (or a still unused static slot), or is dropped itself if its own
+ * score is the lowest (ties: the highest position leaves); the buffer is empty again when the call
+ * returns and ssd_recompress has nothing left to do.
  * SSD_ERR_LIMIT if n_layers > 64 (issue several calls) or, in row-buffer mode, if sink_budget +
- * sink_recent exceeds what a warp can keep in shared memory (about 3000);  SSD_ERR_OVERFLOW (nothing
+ * sink_recent exceeds what a warp can keep in shared memory (about 3000; 1000 with sink_recent = 1);  SSD_ERR_OVERFLOW (nothing
  * launched) if any of the layers, or its row buffer, is full.  Asynchronous. */
 int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *k_new,
                              const void *v_new, const void *q, void *out, void *stream);

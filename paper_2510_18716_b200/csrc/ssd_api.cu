@@ -562,7 +562,9 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
   if (n_layers > kMaxLayersPerLaunch) return SSD_ERR_LIMIT;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
-  if (c->row_buffer && c->mr() > decode_layers_max_mr()) return SSD_ERR_LIMIT;
+  // Row buffer of one token: the launch re-selects as well (Algorithm 1 taken literally)
+  const bool evict = c->row_buffer && g.sink_recent == 1;
+  if (c->row_buffer && c->mr() * (evict ? 3 : 1) > decode_layers_max_mr()) return SSD_ERR_LIMIT;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
@@ -592,7 +594,11 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   p.status = c->d_status();
   p.work = c->d_work();
   p.n_layers = n_layers; p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len;
+  p.acc = c->row_buffer ? c->d_acc(first_layer) : nullptr;
+  p.static_idx = c->d_idx(first_layer);
+  p.M = g.sink_budget;
   p.mr = c->row_buffer ? c->mr() : 0;
+  p.evict = evict ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   for (int i = 0; i < n_layers; ++i) {
     const int layer = first_layer + i;
@@ -604,7 +610,6 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     ls.static_valid = c->static_valid[layer];
     ls.new_j = c->t_img[layer];
     ls.t_img = c->t_img[layer] + 1;
-    ls.acc = c->row_buffer ? c->d_acc(layer) : nullptr;
     ls.sem_slot = c->sem_tokens(layer);
     ls.t_sem = ls.sem_slot + 1;
   }
@@ -613,8 +618,13 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     return SSD_ERR_CUDA;
   }
   for (int i = 0; i < n_layers; ++i) {
-    c->t_img[first_layer + i] += 1;
-    c->pending[first_layer + i] = 0;   // this step's weights are already in the scores
+    const int layer = first_layer + i;
+    c->t_img[layer] += 1;
+    c->pending[layer] = 0;             // this step's weights are already in the scores
+    if (evict) {                       // and the buffer is empty again: the token entered the static set or left
+      if (c->n_sink[layer] > 0 && c->static_valid[layer] < g.sink_budget) c->static_valid[layer] += 1;
+      c->t_base[layer] = c->t_img[layer];
+    }
   }
   c->last_writer = -2;                 // several layers' slabs were written
   return SSD_OK;

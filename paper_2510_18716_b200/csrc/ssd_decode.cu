@@ -712,7 +712,7 @@ __device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Un
   const LayerState& ls = p.layer[layer];
   const HeadDesc d = __ldg(ls.desc + head);
   U.u = u;
-  U.scored = (ls.acc != nullptr && d.w) ? 1 : 0;
+  U.scored = (p.acc != nullptr && d.w) ? 1 : 0;
   const int held = U.scored ? ls.t_sem : ls.t_img;          // tokens the ring holds
   const int r = U.scored ? ls.sem_slot : ls.new_j % d.z;    // ring slot of the token being appended
   U.pv = ls.prompt_valid;
@@ -729,6 +729,8 @@ __device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Un
 
 constexpr int kLayersSmemBytes = kRingBytes + kWarps * kStages * 8 + kWarps * 4 * 4;
 
+// kEvict: Algorithm 1 taken literally (a row buffer of one token, re-selected in the same launch).
+template <bool kEvict>
 __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const __grid_constant__ DecodeLayersParams p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -740,7 +742,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
   volatile int* fifo = reinterpret_cast<volatile int*>(smem + kRingBytes + kWarps * kStages * 8) + warp * 4;
   // row-buffer mode: the logits of the head being streamed, entry e = static slot e or, from the
   // static capacity on, buffer slot e - capacity (the layout of the score rows)
-  float* lgbuf = reinterpret_cast<float*>(smem + kLayersSmemBytes) + (size_t)warp * ((p.mr + 3) & ~3);
+  const int mrp = (p.mr + 3) & ~3;
+  float* lgbuf = reinterpret_cast<float*>(smem + kLayersSmemBytes) + (size_t)warp * mrp * (kEvict ? 3 : 1);
+  float* accbuf = lgbuf + mrp;                         // kEvict: the head's score row ...
+  int* idxbuf = reinterpret_cast<int*>(accbuf + mrp);  // ... and the image indices of its static slots
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -866,6 +871,18 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
       sink.skip = CU.pv;
       sink.ring_from = CU.pv + CU.sv;
       sink.ring_shift = CU.y - CU.sv;
+      if (kEvict && CU.scored) {
+        // the head's scores and static positions are wanted when its last chunk is done: start them
+        // towards shared memory now (4-byte asynchronous copies; nothing waits for them here)
+        const int pairs = p.n_seqs * p.H, layer = CU.u / pairs;
+        const size_t pr = (size_t)layer * pairs + (CU.u - layer * pairs);
+        const float* acc = p.acc + pr * p.mr;
+        const int32_t* idx = p.static_idx + pr * (p.M > 0 ? p.M : 1);
+        for (int i = lane; i < CU.sv; i += 32) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(accbuf + i)), "l"(acc + i) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(idxbuf + i)), "l"(idx + i) : "memory");
+        }
+      }
     }
     sink.i0 = ci;
     Rows rows;
@@ -889,14 +906,58 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
       state_merge_lane(tot, 8);
       state_merge_lane(tot, 16);
       if (grp == 0) write_out(reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<unsigned char*>(p.out) + CU.row), tot, l8);
-      if (CU.scored) {
+      if (kEvict && CU.scored) {
+        // Algorithm 1, one step: add the step's attention weights to the scores, then keep the M best
+        // of the static tokens and the token just appended (lowest score leaves; among equal scores
+        // the highest position, so the new token loses ties).  The new token's rows were stored in the
+        // head's one-slot buffer above by these very lanes; if it stays, they copy it into the static
+        // slot that is free or freed.  Nothing of this head is in flight any more: all its chunks are
+        // consumed.
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        __syncwarp();                    // scores, positions and logits in shared memory, for every lane
+        const int pairs = p.n_seqs * p.H, layer = CU.u / pairs;
+        const size_t pr = (size_t)layer * pairs + (CU.u - layer * pairs);
+        float* acc = p.acc + pr * p.mr;
+        int32_t* idx = p.static_idx + pr * (p.M > 0 ? p.M : 1);
+        const float inv = 1.f / tot.l;
+        const int sv = CU.sv;
+        float worst = 3.0e38f;
+        int worst_pos = -1, worst_e = -1;
+        for (int i = lane; i < sv; i += 32) {
+          const float sc = accbuf[i] + ex2(lgbuf[i] - tot.m) * inv;
+          accbuf[i] = sc;
+          const int pos = idxbuf[i];
+          if (sc < worst || (sc == worst && pos > worst_pos)) { worst = sc; worst_pos = pos; worst_e = i; }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const float w2 = __shfl_xor_sync(FULL, worst, off);
+          const int p2 = __shfl_xor_sync(FULL, worst_pos, off), e2 = __shfl_xor_sync(FULL, worst_e, off);
+          if (w2 < worst || (w2 == worst && p2 > worst_pos)) { worst = w2; worst_pos = p2; worst_e = e2; }
+        }
+        const float w_new = ex2(lgbuf[CU.phys - p.L] - tot.m) * inv;   // the new token's score starts here
+        int dest = -1;                                                 // static slot the new token takes
+        if (sv < p.M) dest = sv;
+        else if (sv > 0 && !(w_new <= worst)) dest = worst_e;
+        for (int i = lane; i < sv; i += 32)
+          if (i != dest) acc[i] = accbuf[i];
+        if (dest >= 0) {
+          if (lane == 0) {
+            acc[dest] = w_new;
+            idx[dest] = p.layer[layer].new_j;
+          }
+          uint4* hb = reinterpret_cast<uint4*>(const_cast<unsigned char*>(CU.hbase));
+          hb[(size_t)(p.L + dest) * kSlotU4 + lane] = hb[(size_t)CU.phys * kSlotU4 + lane];
+        }
+        __syncwarp();                    // before the next head's copies and logits reuse the buffers
+      } else if (CU.scored) {
         // Algorithm 2, "accumulate semantic attention scores": this warp saw the whole head, so the
         // normalised weights go straight into the head's score row (which no other warp touches;
         // additions without a return value, so nothing waits for them).  The token appended in this
         // step starts its score here.
         __syncwarp();                    // the logits written by the group leaders, for every lane
         const int pairs = p.n_seqs * p.H, layer = CU.u / pairs;
-        float* acc = p.layer[layer].acc + (size_t)(CU.u - layer * pairs) * p.mr;
+        float* acc = p.acc + ((size_t)layer * pairs + (CU.u - layer * pairs)) * p.mr;
         const float inv = 1.f / tot.l;
         const int n_scored = CU.vh - CU.pv, e_new = CU.phys - p.L;     // entries that hold a token; the new one
         for (int i = lane; i < n_scored; i += 32) {
@@ -1035,8 +1096,11 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   const bool cached = dev >= 0 && dev < 64;
   int sms = cached ? n_sm[dev] : 0;
   if (!cached || !smem_set[dev]) {
-    e = cudaFuncSetAttribute(ssd_decode_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(ssd_decode_layers_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kLayersSmemBytes + kWarps * decode_layers_max_mr() * 4);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ssd_decode_layers_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kLayersSmemBytes + kWarps * decode_layers_max_mr() * 4);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     if (cached) {
@@ -1046,11 +1110,12 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   }
   const long units = (long)p.n_layers * p.n_seqs * p.H;
   if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
-  if (p.mr < 0 || p.mr > decode_layers_max_mr()) return cudaErrorInvalidValue;
+  if (p.mr < 0 || p.mr * (p.evict ? 3 : 1) > decode_layers_max_mr()) return cudaErrorInvalidValue;
   const long want = (units + kWarps - 1) / kWarps;            // no more CTAs than there are units for
   const int grid = (int)(want < sms ? want : sms);
-  const int smem = kLayersSmemBytes + kWarps * ((p.mr + 3) & ~3) * 4;
-  ssd_decode_layers_kernel<<<grid, kWarps * 32, smem, st>>>(p);
+  const int smem = kLayersSmemBytes + kWarps * ((p.mr + 3) & ~3) * 4 * (p.evict ? 3 : 1);
+  if (p.evict) ssd_decode_layers_kernel<true><<<grid, kWarps * 32, smem, st>>>(p);
+  else ssd_decode_layers_kernel<false><<<grid, kWarps * 32, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }

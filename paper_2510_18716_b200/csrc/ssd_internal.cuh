@@ -57,7 +57,6 @@ struct LayerState {
   int t_img;                // image tokens held, the one being appended included
   int new_j;                // image index of the token being appended
   // row-buffer mode (Algorithm 2): the rings of semantic heads are buffers filled from slot 0
-  float* acc;               // [n_seqs * H, M + R] accumulated attention scores; null outside that mode
   int t_sem;                // tokens in those buffers, the one being appended included
   int sem_slot;             // buffer slot of the token being appended
 };
@@ -70,7 +69,14 @@ struct DecodeLayersParams {
   uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
   uint32_t* work;           // next unit to hand out; zero at launch
   int n_layers, n_seqs, H, L;
-  int mr;                   // M + R: entries of a head's score row (row-buffer mode)
+  // row-buffer mode (Algorithm 2); acc == nullptr outside it.  A layer's tables follow the previous
+  // layer's at fixed strides, so the first layer's pointers serve all.
+  float* acc;               // first layer's [n_seqs * H, M + R] accumulated attention scores
+  int32_t* static_idx;      // first layer's [n_seqs, H, M] image indices of the static slots
+  int M;                    // static capacity of semantic heads
+  int mr;                   // M + R: entries of a head's score row
+  int evict;                // 1 (R == 1 only): the launch also re-selects, i.e. the token just appended
+                            // takes the place of the lowest-scoring static token, or is dropped itself
   float scale_log2;
   LayerState layer[kMaxLayersPerLaunch];
 };

@@ -209,3 +209,56 @@ def test_rowbuf_more_than_1024_candidates_takes_the_radix_path():
                               window=24, name="tiny_wide")
     n = _run(cfg, 0, [0], cfg.n0 + 2 * cfg.sink_recent + 3, fused="layers")
     assert n >= 0
+
+
+def test_eviction_in_the_launch_equals_reselection_after_the_step():
+    """With a buffer of one token ssd_append_decode_layers re-selects inside the launch.  Against the
+    general path (append, attend, ssd_recompress) on a slice of janus1b: same retained sets after every
+    step, same scores to rounding, outputs within the usual bar; and ssd_recompress has nothing to do."""
+    import dataclasses
+    base = wl.CONFIGS["janus1b"]
+    cfg = dataclasses.replace(base, sink_budget=base.sink_budget + base.sink_recent - 1, sink_recent=1, name="janus1b_r1")
+    dev = torch.device("cuda:0")
+    L, n0, M, H, S, NL = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.n_heads, 3, 2
+    labels = np.stack([wl.sink_mask(cfg, l) for l in range(NL)])
+    data = [wl.gen_layer(cfg, l, list(range(S)), device=dev) for l in range(NL)]
+    caches = []
+    for _ in range(2):
+        c = B.SsdCache(B.config_from_workload(cfg, n_layers=NL, n_seqs=S), device=dev)
+        c.set_row_buffer(True)
+        c.set_head_labels(labels)
+        for l, (q, k, v, _) in enumerate(data):
+            c.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(c)
+    general, fused = caches
+    launches_before = None
+    for t in range(n0 + 1, n0 + 41):
+        qs = torch.stack([data[l][0][:, :, t - 1] for l in range(NL)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + t - 1] for l in range(NL)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + t - 1] for l in range(NL)]).contiguous()
+        want = []
+        for l in range(NL):
+            general.append(l, ks[l], vs[l])
+            want.append(general.decode_attn(l, qs[l]))
+            general.recompress(l)
+        got = fused.append_decode_layers(0, ks, vs, qs)
+        launches_before = B.kernel_launch_count()
+        fused.recompress_layers(0, NL)                      # the buffer is already empty
+        assert B.kernel_launch_count() == launches_before
+        d = (got.float() - torch.stack(want).float()).abs()
+        assert d.max().item() <= 2e-2 and d.mean().item() <= 5e-4, (t, d.max().item())
+        for l in range(NL):
+            ga, gb = general.get_indices(l), fused.get_indices(l)
+            assert np.array_equal(np.sort(ga[:, :, L:L + M], axis=-1), np.sort(gb[:, :, L:L + M], axis=-1)), (t, l)
+            assert (gb[:, :, L + M:] == -1)[:, labels[l] == 1].all()          # semantic heads: buffer empty
+            # scores travel with the tokens: compare them by position
+            sa, sb = general.get_scores(l), fused.get_scores(l)
+            for s in range(S):
+                for h in np.nonzero(labels[l])[0]:
+                    a = dict(zip(ga[s, h, L:L + M].tolist(), sa[s, h, :M].tolist()))
+                    b = dict(zip(gb[s, h, L:L + M].tolist(), sb[s, h, :M].tolist()))
+                    assert a.keys() == b.keys()
+                    assert all(abs(a[k] - b[k]) <= 1e-4 * max(abs(a[k]), 1e-3) for k in a), (t, l, s, h)
+    assert general.device_status() == 0 and fused.device_status() == 0
+    for c in caches:
+        c.close()
