@@ -34,8 +34,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.16e6, "per_layer_of_step": 160.75e6,
-                  "sha256": "f642104b48bfedb3baf6c1d8a883ee1807c03f9b22d78d7fc126426296b2dabe"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.39e6, "per_layer_of_step": 160.84e6,
+                  "sha256": "897dd95c647319ed9b92ff857ce2835f7195184c50e275e7842b45dbdb885b7a"}
 
 
 def decode_traffic(cfg):
