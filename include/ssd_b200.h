@@ -153,8 +153,9 @@ int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const 
  * score is the lowest (ties: the highest position leaves); the buffer is empty again when the call
  * returns and ssd_recompress has nothing left to do.
  * SSD_ERR_LIMIT if n_layers > 64 (issue several calls) or, in row-buffer mode, if sink_budget +
- * sink_recent exceeds what a warp can keep in shared memory (about 3000; 1000 with sink_recent = 1);  SSD_ERR_OVERFLOW (nothing
- * launched) if any of the layers, or its row buffer, is full.  Asynchronous. */
+ * sink_recent exceeds what a warp can keep in shared memory (about 3000; 1000 with
+ * sink_recent = 1); SSD_ERR_OVERFLOW (nothing launched) if any of the layers, or its row buffer,
+ * is full.  Asynchronous. */
 int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *k_new,
                              const void *v_new, const void *q, void *out, void *stream);
 
@@ -179,10 +180,10 @@ int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_la
  * token or belong to spatial heads.  Synchronises the device. */
 int ssd_cache_set_row_buffer(ssd_cache *cache, int32_t enable);
 int ssd_recompress(ssd_cache *cache, int32_t layer, void *stream);
-/* ssd_recompress for n_layers consecutive layers in one launch (same results, layer by layer).  With
- * ssd_append_decode_layers this makes a step of the row-buffer mode two launches, and Algorithm 1's
- * re-selection at every step (sink_recent = 1, one call per step) affordable.  SSD_ERR_LIMIT if
- * n_layers > 64. */
+/* ssd_recompress for n_layers consecutive layers in one launch (same results, layer by layer): with
+ * ssd_append_decode_layers, a buffer cycle of Algorithm 2 is R + 1 launches for all layers.  Layers
+ * with an empty buffer and nothing pending are skipped (no launch at all if that is all of them).
+ * SSD_ERR_LIMIT if n_layers > 64. */
 int ssd_recompress_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, void *stream);
 int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
 
