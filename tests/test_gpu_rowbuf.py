@@ -211,15 +211,19 @@ def test_rowbuf_more_than_1024_candidates_takes_the_radix_path():
     assert n >= 0
 
 
-def test_eviction_in_the_launch_equals_reselection_after_the_step():
+@pytest.mark.parametrize("case", ["janus1b_after_prefill", "tiny_from_empty"])
+def test_eviction_in_the_launch_equals_reselection_after_the_step(case):
     """With a buffer of one token ssd_append_decode_layers re-selects inside the launch.  Against the
-    general path (append, attend, ssd_recompress) on a slice of janus1b: same retained sets after every
-    step, same scores to rounding, outputs within the usual bar; and ssd_recompress has nothing to do."""
+    general path (append, attend, ssd_recompress): same retained sets after every step, same scores to
+    rounding, outputs within the usual bar; and ssd_recompress has nothing to do.  Once on a slice of
+    janus1b after a prefill (static set full: every step evicts or drops), once on the tiny shape
+    from an empty cache (the static set first grows slot by slot, then starts evicting)."""
     import dataclasses
-    base = wl.CONFIGS["janus1b"]
-    cfg = dataclasses.replace(base, sink_budget=base.sink_budget + base.sink_recent - 1, sink_recent=1, name="janus1b_r1")
+    base = wl.CONFIGS["janus1b" if case == "janus1b_after_prefill" else "tiny"]
+    cfg = dataclasses.replace(base, sink_budget=base.sink_budget + base.sink_recent - 1, sink_recent=1, name=base.name + "_r1")
     dev = torch.device("cuda:0")
-    L, n0, M, H, S, NL = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.n_heads, 3, 2
+    prefill = case == "janus1b_after_prefill"
+    L, n0, M, H, S, NL = cfg.prompt_len, (cfg.n0 if prefill else 0), cfg.sink_budget, cfg.n_heads, 3, 2
     labels = np.stack([wl.sink_mask(cfg, l) for l in range(NL)])
     data = [wl.gen_layer(cfg, l, list(range(S)), device=dev) for l in range(NL)]
     caches = []
@@ -228,7 +232,8 @@ def test_eviction_in_the_launch_equals_reselection_after_the_step():
         c.set_row_buffer(True)
         c.set_head_labels(labels)
         for l, (q, k, v, _) in enumerate(data):
-            c.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+            if prefill:
+                c.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
         caches.append(c)
     general, fused = caches
     launches_before = None
