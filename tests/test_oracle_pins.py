@@ -432,3 +432,37 @@ def test_golden_closed_forms():
             raise AssertionError(f"unknown golden line: {ln}")
         n_checked += 1
     assert n_checked >= 14
+
+
+def test_rowbuf_of_one_is_the_drop_one_rule_of_algorithm_1():
+    """Algorithm 1 taken literally evicts one token per step: after the step's attention the token
+    with the lowest accumulated score leaves (among equal scores the newest).  The row-buffer
+    function with R = 1 states it as "top-M of M + 1"; the two must retain the same sets, with the
+    same scores and outputs, step by step."""
+    rng = np.random.default_rng(21)
+    L, N, n0, M, D = 3, 40, 12, 6, 8
+    Q, K, V = rand_bf16(rng, N, D), rand_bf16(rng, L + N, D), rand_bf16(rng, L + N, D)
+    outs, hist = oracle.rowbuf_semantic(Q, K, V, L, n0, M, 1, N)
+
+    qf, kf, vf = widen(Q), widen(K), widen(V)
+    scale = 1.0 / math.sqrt(D)
+    sc0 = oracle.scores(Q[:n0], K[: L + n0], L, n0)
+    kept = sorted(sorted(range(n0), key=lambda j: (-sc0[j], j))[:M])
+    score = {j: float(sc0[j]) for j in kept}
+    for i, t in enumerate(range(n0 + 1, N + 1)):
+        held = kept + [t - 1]
+        score[t - 1] = 0.0
+        pos = list(range(L)) + [L + j for j in held]
+        logit = np.array([scale * float(qf[t - 1] @ kf[p]) for p in pos])
+        w = np.exp(logit - logit.max())
+        w /= w.sum()
+        assert np.allclose(outs[i], w @ vf[pos], rtol=1e-12, atol=1e-13)
+        for k, j in enumerate(held):
+            score[j] += w[L + k]
+        if len(held) > M:
+            worst = min(held, key=lambda j: (score[j], -j))      # lowest score; among equals the newest
+            held.remove(worst)
+            del score[worst]
+        kept = sorted(held)
+        assert hist[i][0] == t and hist[i][1] == kept and hist[i][3] == []
+        assert np.allclose(hist[i][2], [score[j] for j in kept], rtol=1e-12, atol=0)
