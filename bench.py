@@ -261,6 +261,14 @@ class Stepper:
         self.i = 0
         self.T = steps_in[0][0].shape[0]
         self.out_all = torch.empty((cfg.n_layers,) + tuple(out.shape), dtype=out.dtype, device=out.device)
+        # device addresses of every step's inputs: the per-layer loop below makes 30 calls per 0.85 ms,
+        # so the host must not spend its time slicing tensors and re-checking shapes at every call
+        qa, ka, va = cache.step_all
+        per = qa[0, 0].numel() * qa.element_size()
+        base = (qa.data_ptr(), ka.data_ptr(), va.data_ptr())
+        self.addr = lambda j, i, layer: base[j] + (i * cfg.n_layers + layer) * per
+        self.call = cache.lib.ssd_append_decode
+        self.h = cache._h
 
     def step(self, fused=True, one_launch=False):
         """One decoded token per sequence: for every layer append the new K/V and attend
@@ -278,13 +286,19 @@ class Stepper:
                 self.cache.append_decode_layers(l0, k[i, l0:l1], v[i, l0:l1], q[i, l0:l1], self.out_all[l0:l1])
             self.i += 1
             return
+        if fused:
+            stream, outp = torch.cuda.current_stream().cuda_stream, self.out.data_ptr()
+            for layer in range(self.cfg.n_layers):
+                rc = self.call(self.h, layer, self.addr(1, i, layer), self.addr(2, i, layer), self.addr(0, i, layer),
+                               outp, stream)
+                if rc != 0:
+                    raise RuntimeError(f"ssd_append_decode: status {rc}")
+            self.i += 1
+            return
         for layer in range(self.cfg.n_layers):
             q, k, v = self.steps_in[layer]
-            if fused:
-                self.cache.append_decode(layer, k[i], v[i], q[i], self.out)
-            else:
-                self.cache.append(layer, k[i], v[i])
-                self.cache.decode_attn(layer, q[i], self.out)
+            self.cache.append(layer, k[i], v[i])
+            self.cache.decode_attn(layer, q[i], self.out)
         self.i += 1
 
 
