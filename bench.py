@@ -358,6 +358,9 @@ def run_ours(args, cfg):
     ms = max_over_ranks(ms)
     ms_per_step = ms / K
     value = cfg.images_per_step * world / (ms_per_step * 1e-3)
+    # stability: five more passes of the same region, shorter
+    Ks = min(K, 50)
+    repeats = [max_over_ranks(timed(one_step, Ks, barrier)) / Ks for _ in range(5)]
 
     # ---- the same step as one launch per layer (ssd_append_decode; what a model calls, since layer
     # l+1's inputs depend on layer l's output); consecutive launches overlap by programmatic dependent launch
@@ -567,6 +570,7 @@ def run_ours(args, cfg):
                        "kv_bytes_per_seq": kv_bytes_per_seq},
             "sequence_tokens_per_s": value * 2 if S > 1 else value,
             "step_form": "one launch per step (ssd_append_decode_layers); per_layer = one launch per layer",
+            "ms_per_step_repeats": repeats,
             "per_layer": per_layer,
             "one_time": setup_times,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
