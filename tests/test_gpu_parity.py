@@ -135,6 +135,22 @@ def test_decode_before_any_compress_fills_ring_from_zero():
     cache.close()
 
 
+def test_hires7b_classifier_one_layer():
+    """Head classification at the 4096-token grid (32 blocks of query rows per unit): sparsity values and
+    labels of one layer's 32 heads over the configuration's calibration sequences, against the oracle."""
+    from parity_util import check_labels
+    cfg = wl.CONFIGS["hires7b"]
+    dev = torch.device("cuda:0")
+    qc, kc = wl.gen_calibration(cfg, [7], device=dev)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=1))
+    s_gpu, lab_gpu = cache.classify_heads(qc, kc)
+    s_ora = oracle.sparsity(wl.to_u16(qc), wl.to_u16(kc), cfg.prompt_len, cfg.cls_window)
+    labels = check_labels(s_gpu, lab_gpu, s_ora, cfg.tau)
+    assert np.array_equal(labels[0], wl.sink_mask(cfg, 7)), "classifier must recover the generator's split"
+    assert cache.device_status() == 0
+    cache.close()
+
+
 def test_classifier_scores_match_oracle_on_mixed_heads():
     # sparsity values themselves (not only labels), on data with no planted structure
     cfg = wl.Workload("cls", 2, 2, 5, 7, (6, 9), 8, 8, 4, 11, 0, 20, 3, 1.2, seed=7)
