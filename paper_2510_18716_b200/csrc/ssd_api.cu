@@ -585,7 +585,7 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
       return SSD_ERR_CUDA;
     c->pending[layer] = 0;
   }
-  DecodeLayersParams p;
+  DecodeLayersParams p = {};          // entries past n_layers stay zero
   p.slab = reinterpret_cast<uint4*>(c->base + c->reg.slab);
   p.q = static_cast<const unsigned char*>(q);
   p.k_new = static_cast<const unsigned char*>(k_new);
@@ -847,7 +847,7 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
   if (first_layer < 0 || n_layers < 1 || first_layer > g.n_layers - n_layers) return SSD_ERR_INVALID_ARG;
   if (n_layers > kMaxLayersPerLaunch) return SSD_ERR_LIMIT;
   if (!c->labels_set || !c->row_buffer) return SSD_ERR_BAD_STATE;
-  RecompressLayersParams p;
+  RecompressLayersParams p = {};      // entries past n_layers stay zero
   p.slab = reinterpret_cast<uint4*>(c->base + c->reg.slab);
   p.desc = c->d_desc(first_layer);
   p.static_idx = c->d_idx(first_layer);
