@@ -135,6 +135,16 @@ int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, v
 int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new,
                       const void *q, void *out, void *stream);
 
+/* Hand-over between consecutive per-layer launches (no paper counterpart; a scheduling hint).  A caller
+ * that goes round the layers (layer 0, 1, .., n_layers-1, 0, ..) issues launches whose first copies find
+ * HBM idle while the previous launch drains.  To close that gap each decode worker, once its own last
+ * copy is issued, asks the L2 cache to fetch the first `slots` slots (512 B each) of the same share of
+ * the NEXT layer's slab.  It applies only when both layers are full (prompt, static sets and rings hold
+ * tokens in every slot) and of equal size; it never changes results.  slots = 0 switches it off (useful
+ * when other kernels that sweep the L2 cache run between the layers' calls); the default is 48.
+ * SSD_ERR_INVALID_ARG if slots < 0 or > 4096. */
+int ssd_cache_set_prefetch(ssd_cache *cache, int32_t slots);
+
 /* ssd_append_decode for n_layers consecutive layers in ONE launch (a whole decode step when the
  * inputs of all layers exist up front, as in a benchmark of this path or a host-driven replay; in a
  * model, layer l+1's query depends on layer l's output and the per-layer call is the one to use).
@@ -164,11 +174,11 @@ int ssd_append_decode_layers(ssd_cache *cache, int32_t first_layer, int32_t n_la
  *   ssd_compress     selects the top-M over all n0 tokens (the buffer starts empty) and records the
  *                    selected tokens' scores;
  *   ssd_append       puts the token into the buffer; SSD_ERR_OVERFLOW when the buffer already holds R
- *                    tokens ("row buffer overflow"): call ssd_recompress first;
+ *                    tokens (Algorithm 2, overflow branch): call ssd_recompress first;
  *   ssd_decode_attn  attends over prompt + static set + buffer and keeps the step's attention weights
  *                    of the static and buffered tokens of semantic heads; they are added to the tokens'
  *                    accumulated scores by the layer's next ssd_append or ssd_recompress;
- *   ssd_recompress   ("row buffer full"): per (sequence, semantic head) keeps the top-M of static set +
+ *   ssd_recompress   (Algorithm 2, buffer-full branch): per (sequence, semantic head) keeps the top-M of static set +
  *                    buffer by accumulated score (ties: lowest position) as the new static set and
  *                    empties the buffer.  Tokens that stay keep their slots; tokens that enter take
  *                    the slots of those that leave, so static slots are in ascending position only

@@ -228,17 +228,18 @@ class RowBufferOverflow(RuntimeError):
 
 
 def rowbuf_semantic(Q, K, V, L, n0, M, R, t_end, compress_when_full=True, scale=None, choose=None):
-    """Algorithm 2 (compression with a row buffer) for ONE semantic (sequence, head), step by step.
+    """Algorithm 2 (compression with a row buffer) for ONE semantic (sequence, head).
 
-    Q [N,D] image queries, K, V [L+N,D] (uint16 bf16).  State: a static set of at most M image
-    tokens with their accumulated attention scores, and a row buffer of at most R tokens.
-      prefill (image step n0):  scores = running sum of attention over steps 1..n0 (Algorithm 1);
-                                static = top-M of them over all n0 tokens; buffer empty.
-      decode step t = n0+1..t_end, in the algorithm's order:
-        append token t-1 to the buffer (overflow is an error); attend over prompt + static + buffer;
-        add the step's attention weights to the scores of the static and buffered tokens;
-        if the buffer holds R tokens: keep the top-M of static + buffer by score (ties: lowest
-        position), in ascending position; empty the buffer.
+    Q [N,D] image queries, K, V [L+N,D] (uint16 bf16).  State carried from step to step: `static`, at
+    most M image tokens; `buf`, the row buffer, at most R tokens newer than every static token; `acc`,
+    the accumulated attention score of every held token.  Invariants: static and buf are disjoint and
+    each in ascending position; acc[j] = (prefill running sum of Algorithm 1, if j was selected at
+    prefill, else 0) + the attention weight j received at every decode step since it was appended.
+      prefill (image step n0): static = top-M of the running sums over all n0 tokens; buf empty.
+      decode step t: token t-1 joins buf (a full buffer is the overflow error); the step attends over
+        prompt + static + buf and every held token's weight is added to its acc; a buffer that now
+        holds R tokens triggers the re-selection: static = top-M of static + buf by acc (ties: lowest
+        position), buf = empty, acc of dropped tokens forgotten.
     Returns (outs [t_end-n0, D] fp64, history): history[k] = (t, static positions after step t,
     their scores, buffered positions, their scores) for every step.
     `choose(t, candidates, scores, keep)` may replace the kept candidate indices at a compression (a

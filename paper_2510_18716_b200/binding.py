@@ -31,6 +31,7 @@ EXPORTS = [
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
+    "ssd_cache_set_prefetch",
 ]
 
 
@@ -79,6 +80,7 @@ def load():
     L.ssd_decode_attn_static.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_append_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_set_row_buffer.argtypes = [vp, i32]
+    L.ssd_cache_set_prefetch.argtypes = [vp, i32]
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
@@ -272,6 +274,10 @@ class SsdCache:
     # -- Algorithm 2 (row buffer)
     def set_row_buffer(self, enable: bool = True):
         self._check(self.lib.ssd_cache_set_row_buffer(self._h, 1 if enable else 0), "ssd_cache_set_row_buffer")
+
+    def set_prefetch(self, slots: int):
+        """Slots of the next layer each decode worker asks L2 to fetch at its end (0 = off)."""
+        self._check(self.lib.ssd_cache_set_prefetch(self._h, int(slots)), "ssd_cache_set_prefetch")
 
     def recompress(self, layer: int):
         self._check(self.lib.ssd_recompress(self._h, layer, _stream()), "ssd_recompress")

@@ -20,6 +20,8 @@ static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 // staging slots; a slot holds q, k_new, v_new and out of a whole group.
 constexpr int kHostGroup = 4;
 constexpr int kHostSlots = 3;
+// Slots of the next layer each decode worker asks the L2 cache to fetch when its own copies are issued.
+constexpr int kDefaultPrefetchSlots = 48;
 
 struct Regions {
   size_t desc, idx, counters, status, partial, score, staging, acc, logits, ml, slab;  // byte offsets
@@ -96,6 +98,7 @@ struct ssd_cache {
   cudaEvent_t h_fork = nullptr, h_loaded[kHostSlots] = {}, h_done[kHostSlots] = {}, h_stored[kHostSlots] = {};
   long h_groups = 0;                  // groups sent through the staging ring so far
   bool h_foreign = false;             // ssd_step_host has used the staging area since
+  int pf_slots = kDefaultPrefetchSlots;   // L2 hand-over depth per worker (ssd_cache_set_prefetch)
   std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
   int prof_n = 0;                     // launches recorded since the last collect
 
@@ -123,6 +126,25 @@ struct ssd_cache {
   int max_slots() const {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
     return cfg.prompt_len + (a > b ? a : b);
+  }
+  // True if every slot of the layer will hold a token once the layer holds t image tokens (t_sem of them
+  // in the rings of semantic heads): the layer's valid slots are then its whole slab, in slab order.
+  bool layer_full(int layer, int t, int t_sem) const {
+    if (prompt_valid[layer] != cfg.prompt_len) return false;
+    if (n_sink[layer] > 0 && (static_valid[layer] != cfg.sink_budget || t_sem < cfg.sink_recent)) return false;
+    if (n_sink[layer] < cfg.n_heads && t < cfg.window) return false;
+    return true;
+  }
+  // Where a launch on `layer` (which will hold t / t_sem tokens when it runs) hands over to: the slab of
+  // the layer a caller going round the layers attends to next, if both layers are full and of the same
+  // size, so that a worker's share covers the same byte range in both; else null.
+  const unsigned char* hand_over_to(int layer, int t, int t_sem) const {
+    if (pf_slots <= 0 || cfg.n_layers < 2) return nullptr;
+    const int nl = layer + 1 < cfg.n_layers ? layer + 1 : 0;
+    const int tn = t_img[nl] + 1 < cfg.max_image_tokens ? t_img[nl] + 1 : cfg.max_image_tokens;
+    const int tn_sem = row_buffer ? sem_tokens(nl) + 1 : tn;
+    if (seq_slots[nl] != seq_slots[layer] || !layer_full(layer, t, t_sem) || !layer_full(nl, tn, tn_sem)) return nullptr;
+    return reinterpret_cast<const unsigned char*>(d_slab(nl));
   }
   // layout and occupancy of a layer, as the decode kernel sees it
   void fill_view(int layer, LayerView& v) const {
@@ -447,12 +469,13 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
 
 int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new, void* stream) {
   if (!c || !k_new || !v_new) return SSD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
   if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent)
-    return SSD_ERR_OVERFLOW;            // Algorithm 2: row buffer overflow; call ssd_recompress first
+    return SSD_ERR_OVERFLOW;            // Algorithm 2, overflow branch: call ssd_recompress first
   AppendParams p;
   p.slab = c->d_slab(layer);
   p.desc = c->d_desc(layer);
@@ -496,6 +519,8 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
+  p.next_slab = c->hand_over_to(layer, c->t_img[layer], c->sem_tokens(layer));
+  p.pf_slots = c->pf_slots;
   c->fill_view(layer, p.view);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
@@ -539,6 +564,8 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->t_img[layer] += 1;                // the view describes the layer with the token in place
+  p.next_slab = c->hand_over_to(layer, c->t_img[layer], c->sem_tokens(layer));
+  p.pf_slots = c->pf_slots;
   c->fill_view(layer, p.view);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
@@ -572,7 +599,7 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     const int layer = first_layer + i;
     if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
     if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent)
-      return SSD_ERR_OVERFLOW;          // Algorithm 2: row buffer overflow; call ssd_recompress first
+      return SSD_ERR_OVERFLOW;          // Algorithm 2, overflow branch: call ssd_recompress first
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Row-buffer mode: the kernel adds each step's attention weights to the scores itself.  A layer whose
@@ -798,6 +825,12 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
   size_t slots = 0;
   for (int l = 0; l < c->cfg.n_layers; ++l) slots += (size_t)c->seq_slots[l];
   *bytes_per_seq = slots * kSlotBytes;
+  return SSD_OK;
+}
+
+int ssd_cache_set_prefetch(ssd_cache* c, int32_t slots) {
+  if (!c || slots < 0 || slots > 4096) return SSD_ERR_INVALID_ARG;
+  c->pf_slots = slots;
   return SSD_OK;
 }
 
@@ -1048,6 +1081,8 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
+  p.next_slab = nullptr;
+  p.pf_slots = 0;
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;

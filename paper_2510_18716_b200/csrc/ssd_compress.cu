@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams
 }
 
 // ----------------------------------------------------------------------------- recompress
-// Algorithm 2, "row buffer full": for every (sequence, semantic head) keep the top-M of the static
+// Algorithm 2, the branch taken when the buffer is full: for every (sequence, semantic head) keep the top-M of the static
 // set plus the buffered tokens by accumulated attention score (ties: lowest position) as the new
 // static set; the buffer is then empty.  One CTA per pair.  Static tokens that stay keep their
 // slots; the buffered tokens that make it take the slots of the static tokens that do not (and the

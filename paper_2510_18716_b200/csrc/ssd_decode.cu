@@ -139,6 +139,12 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 // transitively; and when a kernel starts, everything before its predecessor has completed (the
 // predecessor passed its own wait before allowing it), which is what makes the slab prefetch of the
 // decode kernel's prologue safe.
+// Ask the L2 cache to fetch [src, src + bytes) (16-byte aligned, a multiple of 16): no destination, no
+// completion to wait for.
+__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ void pdl_allow_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -557,6 +563,23 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     }
   }
 
+  // Once the last copy of the share has been issued this worker's demand on HBM ends: fill the gap
+  // with the start of the same share of the next layer, in the order the next launch will read it.
+  bool handed_over = p.next_slab == nullptr || p.pf_slots <= 0;
+  auto hand_over = [&]() {
+    handed_over = true;
+    if (lane != 0) return;
+    int left = p.pf_slots;
+    const int a0 = two_parts ? g_tail : g_begin;
+    const int n0 = left < g_end - a0 ? left : g_end - a0;
+    l2_prefetch(p.next_slab + (size_t)a0 * kSlotBytes, (uint32_t)n0 * kSlotBytes);
+    left -= n0;
+    if (two_parts && left > 0) {
+      const int n1 = left < g_tail - g_begin ? left : g_tail - g_begin;
+      l2_prefetch(p.next_slab + (size_t)g_begin * kSlotBytes, (uint32_t)n1 * kSlotBytes);
+    }
+  };
+
   int stage = 0;
   uint32_t parity = 0;
   bool begin = true, leading = true;
@@ -612,6 +635,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
     if (prod.g < prod.g_end) issue(stage);
+    else if (!handed_over) hand_over();
     fold_stage(rows, n, grp, l8, q, st, sink);
 
     const int i1 = cons.i + n;
@@ -951,7 +975,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
         }
         __syncwarp();                    // before the next head's copies and logits reuse the buffers
       } else if (CU.scored) {
-        // Algorithm 2, "accumulate semantic attention scores": this warp saw the whole head, so the
+        // Algorithm 2, post-processing (score accumulation): this warp saw the whole head, so the
         // normalised weights go straight into the head's score row (which no other warp touches;
         // additions without a return value, so nothing waits for them).  The token appended in this
         // step starts its score here.
@@ -1002,8 +1026,8 @@ __global__ void __launch_bounds__(256) ssd_append_kernel(const AppendParams p) {
   int ring_slot = p.j % d.z;
   if (p.acc != nullptr && d.w) {
     // Algorithm 2: the ring of a semantic head is a row buffer filled from slot 0.  First bring the
-    // scores up to date with the attention of the layer's last decode ("accumulate semantic
-    // attention scores"), then start the new token's score at zero.
+    // scores up to date with the attention of the layer's last decode (Algorithm 2, score
+    // accumulation), then start the new token's score at zero.
     float* acc = p.acc + (size_t)warp * p.mr;
     if (p.pending) {
       const float* lg = p.logits + (size_t)warp * p.mr;

@@ -41,6 +41,11 @@ struct DecodeParams {
   const unsigned char* v_new;
   int new_j;                // image index of that token; the view already counts it
   int early;                // 1: the launch before this one on the stream does not write this layer's slab
+  // Hand-over to the next launch: a worker that has issued its last copy asks the L2 cache to fetch the
+  // first pf_slots slots of the same share of the layer that will be attended to next (null: none), so
+  // that HBM stays busy while this launch drains and the next one starts.  A hint only.
+  const unsigned char* next_slab;
+  int pf_slots;
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
   LayerView view;           // layout and occupancy of the layer
