@@ -68,7 +68,8 @@ const char *ssd_status_string(int status);
 size_t ssd_cache_required_bytes(const ssd_config *cfg, int32_t n_sink_heads_total);
 
 /* Create a cache over caller-owned device memory [dev_mem, dev_mem + dev_bytes) (256-byte
- * aligned).  Validates the config, lays out tables and scratch at the front of the buffer and
+ * aligned).  The config carries what Algorithm 1 lists as its parameters (window size, token budget) and
+ * what Sec. 3.3 adds (reserved recent window, threshold).  Validates the config, lays out tables and scratch at the front of the buffer and
  * clears them (synchronously, on the default stream).  Head labels do not exist yet: call
  * ssd_classify_heads or ssd_set_head_labels next.  The buffer must outlive the cache. */
 int ssd_cache_create(const ssd_config *cfg, void *dev_mem, size_t dev_bytes, ssd_cache **out);
@@ -96,8 +97,21 @@ int ssd_classify_heads(ssd_cache *cache, const void *q_cal, const void *k_cal, i
 int ssd_classify_partial(ssd_cache *cache, const void *q_cal, const void *k_cal, int32_t n_cal_seqs,
                          int32_t n_img, double *ratio_sums_host, void *stream);
 
-/* Install head labels directly ([n_layers * n_heads] uint8, 1 = semantic): by-construction or
- * random partitions (Sec. 4.4 ablation).  Resets every layer to the empty state. */
+/* The threshold rule of Sec. 3.3 on its own, for callers that hold ratio sums (ssd_classify_partial,
+ * added over ranks) or sparsity values (a sweep of tau, Sec. 4.3/4.4).  Host arithmetic only; no GPU and
+ * no cache is needed.
+ *   ssd_labels_from_ratio_sums: s[i] = (float)(ratio_sums[i] / (n_cal_total * n_img)), label[i] = s[i] > tau
+ *     (equality is spatial), exactly what ssd_classify_heads computes; s_out_host and labels_out_host
+ *     [n] may each be NULL.
+ *   ssd_labels_from_sparsity:   label[i] = s[i] > tau for float32 sparsity values.
+ * SSD_ERR_INVALID_ARG on null inputs, n < 0, non-finite tau, n_cal_total < 1 or n_img < 1. */
+int ssd_labels_from_ratio_sums(const double *ratio_sums_host, int64_t n, int32_t n_cal_total, int32_t n_img,
+                               float tau, float *s_out_host, uint8_t *labels_out_host);
+int ssd_labels_from_sparsity(const float *s_host, int64_t n, float tau, uint8_t *labels_out_host);
+
+/* Install head labels directly ([n_layers * n_heads] uint8, 1 = semantic): what a caller that shards
+ * the calibration batch does after ssd_labels_from_ratio_sums (Sec. 3.3), and how by-construction or
+ * random partitions are set (Sec. 4.4 ablation).  Resets every layer to the empty state. */
 int ssd_set_head_labels(ssd_cache *cache, const uint8_t *labels_host);
 
 /* Bulk-load one layer from an uncompressed cache holding the prompt and n0 image tokens, and
@@ -120,7 +134,9 @@ int ssd_compress(ssd_cache *cache, int32_t layer, const void *q_obs, const void 
  * SSD_ERR_OVERFLOW once max_image_tokens tokens are held.  Asynchronous. */
 int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new, void *stream);
 
-/* Single-token decode attention over the layer's retained slots, both head types in one launch:
+/* Single-token decode attention (Sec. 3.1, the attention of one generated token over the cached keys and
+ * values; the caches are Algorithm 1's output, its Ensure line) over the layer's retained slots, both
+ * head types in one launch:
  * out[s,h] = sum_i softmax_i(scale * <q[s,h], K_i>) V_i over the prompt, static and ring slots
  * that hold a token (the token just appended included).  fp32 accumulation, bf16 output.
  *   q, out [n_seqs, n_heads, head_dim], 16-byte aligned
@@ -144,6 +160,18 @@ int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const 
  * when other kernels that sweep the L2 cache run between the layers' calls); the default is 48.
  * SSD_ERR_INVALID_ARG if slots < 0 or > 4096. */
 int ssd_cache_set_prefetch(ssd_cache *cache, int32_t slots);
+
+/* Which kernel ssd_decode_attn and ssd_append_decode launch (no paper counterpart; both compute the same
+ * attention, results differ only in the rounding order of the softmax sums):
+ *   1  equal shares: the layer's slots are cut into equal byte ranges, one per warp; a head cut by a
+ *      range boundary is merged through scratch memory.  Best when a layer has few, long heads.
+ *   2  heads to thread blocks: a thread block claims whole heads from a counter and its warps share each
+ *      head's chunks, so a slower SM takes fewer heads.  Best when every SM gets many heads.  In row-buffer
+ *      mode ssd_append_decode is then ONE launch that also maintains the scores (and, with sink_recent = 1,
+ *      re-selects, which is Algorithm 1 taken literally).
+ *   0  (default) form 2 when the layer has at least 8 heads per SM (n_seqs * n_heads >= 8 * SMs), else 1.
+ * SSD_ERR_INVALID_ARG for other values. */
+int ssd_cache_set_decode_form(ssd_cache *cache, int32_t form);
 
 /* ssd_append_decode for n_layers consecutive layers in ONE launch (a whole decode step when the
  * inputs of all layers exist up front, as in a benchmark of this path or a host-driven replay; in a
@@ -206,7 +234,9 @@ int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
  * allocation's implicit synchronisation is not acceptable.  For them the same scratch is a fixed
  * array inside the library image (about 0.4 MB, held by every GPU that loads the library until the
  * process ends), and this call allocates nothing, on the device or through any library.
- *   Same arguments, results and errors as ssd_decode_attn (outputs are bit-identical), plus
+ *   Same arguments, results and errors as ssd_decode_attn (it runs the equal-shares kernel: outputs are
+ *   bit-identical to ssd_decode_attn's when that call runs the same kernel, see
+ *   ssd_cache_set_decode_form, and equal up to the rounding order of the softmax sums otherwise), plus
  *   SSD_ERR_LIMIT if n_seqs * n_heads > 32768 or the GPU has more than 256 SMs: the array is sized
  *   for those maxima.
  * The first call on each device looks up the array's device address (a synchronous runtime query);
@@ -241,7 +271,8 @@ int ssd_step_host(ssd_cache *cache, int32_t layer, const void *q_host, const voi
 int ssd_step_host_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, const void *q_host,
                          const void *k_new_host, const void *v_new_host, void *out_host, void *stream);
 
-/* Absolute positions held by each slot of a layer, for inspection and index-set parity:
+/* Absolute positions held by each slot of a layer (the index sets Algorithm 1 keeps: IndicesOfTopM for
+ * semantic heads, the last W for spatial heads), for inspection and index-set parity:
  * idx_host [n_seqs, n_heads, max_slots] int32 with max_slots = ssd_cache_max_slots(); slots are
  * ordered prompt, static (ascending position after ssd_compress; slot order after re-selections
  * in row-buffer mode), ring (physical ring order); -1 = empty or unused.

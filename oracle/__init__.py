@@ -223,6 +223,24 @@ def decode_batch(q, K_hist, V_hist, is_semantic, idx, cnt, L, t, W, M, R, scale=
     return out
 
 
+def _widen(a):
+    """bf16 bit patterns (uint16) -> float64, exactly."""
+    return (_u16(a).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def kv_token_mse(K_a, V_a, K_b, V_b):
+    """Per-token divergence of two KV caches (Sec. 3.2, the MSE_token equation):
+    out[..., j] = ||K_a[..., j, :] - K_b[..., j, :]||^2 + ||V_a[..., j, :] - V_b[..., j, :]||^2.
+
+    Inputs [..., T, D] uint16 bf16 bit patterns, all of one shape (the paper's two caches are the
+    CFG branch and the native branch of one prompt); output [..., T] float64.  The equation has no
+    1/D in it although it is called a mean; it is written out as printed."""
+    Ka, Va, Kb, Vb = _widen(K_a), _widen(V_a), _widen(K_b), _widen(V_b)
+    assert Ka.shape == Va.shape == Kb.shape == Vb.shape
+    dk, dv = Ka - Kb, Va - Vb
+    return (dk * dk).sum(-1) + (dv * dv).sum(-1)
+
+
 class RowBufferOverflow(RuntimeError):
     """Algorithm 2: a token was appended to a row buffer that already holds R tokens."""
 

@@ -10,8 +10,9 @@ import numpy as np
 
 
 def labels_for_tau(s: np.ndarray, tau: float) -> np.ndarray:
-    """label = s > tau, decided in float32 like the library's classifier (equality is spatial)."""
-    return (np.asarray(s, np.float32) > np.float32(tau)).astype(np.uint8)
+    """Labels the library's threshold rule (ssd_labels_from_sparsity) gives for sparsity values s."""
+    from . import binding
+    return binding.labels_from_sparsity(s, tau)
 
 
 def tau_sweep(s: np.ndarray, taus: Iterable[float]) -> Dict[float, np.ndarray]:

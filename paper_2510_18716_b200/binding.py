@@ -31,7 +31,7 @@ EXPORTS = [
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
-    "ssd_cache_set_prefetch",
+    "ssd_cache_set_prefetch", "ssd_cache_set_decode_form", "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity",
 ]
 
 
@@ -81,6 +81,9 @@ def load():
     L.ssd_append_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_set_row_buffer.argtypes = [vp, i32]
     L.ssd_cache_set_prefetch.argtypes = [vp, i32]
+    L.ssd_cache_set_decode_form.argtypes = [vp, i32]
+    L.ssd_labels_from_ratio_sums.argtypes = [vp, C.c_int64, i32, i32, C.c_float, vp, vp]
+    L.ssd_labels_from_sparsity.argtypes = [vp, C.c_int64, C.c_float, vp]
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
@@ -128,6 +131,28 @@ def make_config(n_layers, n_seqs, n_heads, prompt_len, max_image_tokens, window,
 def config_from_workload(w, n_layers: Optional[int] = None, n_seqs: Optional[int] = None) -> SsdConfig:
     return make_config(n_layers or w.n_layers, n_seqs or w.n_seqs, w.n_heads, w.prompt_len, w.n_img,
                        w.window, w.sink_budget, w.sink_recent, w.cls_window, w.tau)
+
+
+def labels_from_ratio_sums(total_sums, n_cal_total: int, n_img: int, tau: float):
+    """(s float32, labels uint8), both shaped like total_sums: the library's threshold rule (Sec. 3.3)."""
+    sums = np.ascontiguousarray(total_sums, np.float64)
+    s = np.empty(sums.shape, np.float32)
+    lab = np.empty(sums.shape, np.uint8)
+    rc = load().ssd_labels_from_ratio_sums(sums.ctypes.data, sums.size, int(n_cal_total), int(n_img), float(tau),
+                                           s.ctypes.data, lab.ctypes.data)
+    if rc != SSD_OK:
+        raise SsdError(rc, "ssd_labels_from_ratio_sums")
+    return s, lab
+
+
+def labels_from_sparsity(s, tau: float):
+    """labels uint8 shaped like s: semantic iff s > tau, decided by the library in float32."""
+    s32 = np.ascontiguousarray(s, np.float32)
+    lab = np.empty(s32.shape, np.uint8)
+    rc = load().ssd_labels_from_sparsity(s32.ctypes.data, s32.size, float(tau), lab.ctypes.data)
+    if rc != SSD_OK:
+        raise SsdError(rc, "ssd_labels_from_sparsity")
+    return lab
 
 
 def required_bytes(cfg: SsdConfig, n_sink_heads_total: int = -1) -> int:
@@ -278,6 +303,10 @@ class SsdCache:
     def set_prefetch(self, slots: int):
         """Slots of the next layer each decode worker asks L2 to fetch at its end (0 = off)."""
         self._check(self.lib.ssd_cache_set_prefetch(self._h, int(slots)), "ssd_cache_set_prefetch")
+
+    def set_decode_form(self, form: int):
+        """Per-layer decode kernel: 0 chosen by size, 1 equal shares, 2 heads handed out to thread blocks."""
+        self._check(self.lib.ssd_cache_set_decode_form(self._h, int(form)), "ssd_cache_set_decode_form")
 
     def recompress(self, layer: int):
         self._check(self.lib.ssd_recompress(self._h, layer, _stream()), "ssd_recompress")

@@ -21,7 +21,7 @@ static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 constexpr int kHostGroup = 4;
 constexpr int kHostSlots = 3;
 // Slots of the next layer each decode worker asks the L2 cache to fetch when its own copies are issued.
-constexpr int kDefaultPrefetchSlots = 48;
+constexpr int kDefaultPrefetchSlots = 0;
 
 struct Regions {
   size_t desc, idx, counters, status, partial, score, staging, acc, logits, ml, slab;  // byte offsets
@@ -52,7 +52,8 @@ static Regions plan_regions(const ssd_config& c) {
   r.desc = off;      off = align_up(off + (size_t)c.n_layers * c.n_heads * sizeof(HeadDesc));
   r.idx = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * (c.sink_budget > 0 ? c.sink_budget : 1) * 4);
   r.counters = off;  off = align_up(off + pairs_layer * 4);
-  r.status = off;    off = align_up(off + 132);   // status word, and at +128 the unit counter of the all-layers launch
+  r.status = off;    off = align_up(off + 200);   // status word; at +128 the unit counter of the all-layers launch;
+                                                  // at +192 the two claim counters of the heads-to-blocks launch
   r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
   r.partial = off;   off = align_up(off + r.partial_bytes);
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
@@ -99,6 +100,8 @@ struct ssd_cache {
   long h_groups = 0;                  // groups sent through the staging ring so far
   bool h_foreign = false;             // ssd_step_host has used the staging area since
   int pf_slots = kDefaultPrefetchSlots;   // L2 hand-over depth per worker (ssd_cache_set_prefetch)
+  int decode_form = 0;                // per-layer decode kernel: 0 chosen by size, 1 equal shares, 2 heads to blocks
+  int claim_parity = 0;               // which claim counter the next heads-to-blocks launch uses
   std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
   int prof_n = 0;                     // launches recorded since the last collect
 
@@ -109,6 +112,29 @@ struct ssd_cache {
   }
   uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(base + reg.status); }
+  uint32_t* d_claim() const { return reinterpret_cast<uint32_t*>(base + reg.status + 192); }
+  // Per-layer decode with heads handed out to thread blocks: worth it when every SM gets many heads
+  // (else equal shares balance better), and possible while a head's score row fits its table entry.
+  bool heads_form() const {
+    if (decode_form == 1) return false;
+    if (row_buffer && mr() > decode_heads_max_mr(0)) return false;
+    return decode_form == 2 || (long)cfg.n_seqs * cfg.n_heads >= decode_heads_min_pairs();
+  }
+  void fill_heads(int layer, DecodeHeadsParams& p) {
+    p.slab = d_slab(layer);
+    p.desc = d_desc(layer);
+    p.status = d_status();
+    p.claim = d_claim();
+    p.parity = claim_parity;
+    p.n_seqs = cfg.n_seqs; p.H = cfg.n_heads; p.L = cfg.prompt_len; p.seq_slots = seq_slots[layer];
+    p.prompt_valid = prompt_valid[layer];
+    p.static_valid = static_valid[layer];
+    p.t_img = t_img[layer];
+    p.t_sem = sem_tokens(layer);
+    p.early = (last_writer >= -1 && last_writer != layer) ? 1 : 0;
+    p.acc = nullptr; p.static_idx = d_idx(layer); p.M = cfg.sink_budget; p.mr = 0; p.evict = 0;
+    p.scale_log2 = scale * 1.4426950408889634f;
+  }
   uint32_t* d_work() const { return reinterpret_cast<uint32_t*>(base + reg.status + 128); }   // unit counter of the all-layers launch
   int mr() const { return cfg.sink_budget + cfg.sink_recent; }
   size_t layer_scores(int layer) const { return (size_t)layer * cfg.n_seqs * cfg.n_heads * mr(); }
@@ -386,6 +412,25 @@ int ssd_classify_partial(ssd_cache* c, const void* q_cal, const void* k_cal, int
   return SSD_OK;
 }
 
+// The threshold rule (Sec. 3.3): s = mean ratio, taken in float32; a head is semantic iff s > tau, so
+// equality is spatial.  Host arithmetic only.
+int ssd_labels_from_sparsity(const float* s_host, int64_t n, float tau, uint8_t* labels_out_host) {
+  if (!s_host || !labels_out_host || n < 0 || !std::isfinite(tau)) return SSD_ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) labels_out_host[i] = s_host[i] > tau ? 1 : 0;
+  return SSD_OK;
+}
+
+int ssd_labels_from_ratio_sums(const double* ratio_sums_host, int64_t n, int32_t n_cal_total, int32_t n_img, float tau,
+                               float* s_out_host, uint8_t* labels_out_host) {
+  if (!ratio_sums_host || n < 0 || n_cal_total < 1 || n_img < 1 || !std::isfinite(tau)) return SSD_ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i) {
+    const float s = (float)(ratio_sums_host[i] / ((double)n_cal_total * (double)n_img));
+    if (s_out_host) s_out_host[i] = s;
+    if (labels_out_host) ssd_labels_from_sparsity(&s, 1, tau, labels_out_host + i);
+  }
+  return SSD_OK;
+}
+
 int ssd_classify_heads(ssd_cache* c, const void* q_cal, const void* k_cal, int32_t n_cal_seqs, int32_t n_img,
                        float* s_out_host, uint8_t* labels_out_host, void* stream) {
   if (!c) return SSD_ERR_INVALID_ARG;
@@ -394,11 +439,8 @@ int ssd_classify_heads(ssd_cache* c, const void* q_cal, const void* k_cal, int32
   int rc = ssd_classify_partial(c, q_cal, k_cal, n_cal_seqs, n_img, sums.data(), stream);
   if (rc != SSD_OK) return rc;
   std::vector<uint8_t> lab(nh);
-  for (size_t i = 0; i < nh; ++i) {
-    const float s = (float)(sums[i] / ((double)n_cal_seqs * (double)n_img));
-    if (s_out_host) s_out_host[i] = s;
-    lab[i] = s > c->cfg.tau ? 1 : 0;   // equality is spatial
-  }
+  rc = ssd_labels_from_ratio_sums(sums.data(), (int64_t)nh, n_cal_seqs, n_img, c->cfg.tau, s_out_host, lab.data());
+  if (rc != SSD_OK) return rc;
   rc = ssd_set_head_labels(c, lab.data());
   if (rc != SSD_OK) return rc;
   if (labels_out_host) std::memcpy(labels_out_host, lab.data(), nh);
@@ -505,6 +547,24 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
+  if (!c->row_buffer && c->heads_form()) {
+    DecodeHeadsParams hp;
+    c->fill_heads(layer, hp);
+    hp.q = static_cast<const unsigned char*>(q);
+    hp.k_new = nullptr; hp.v_new = nullptr; hp.new_j = -1; hp.sem_slot = 0;
+    hp.out = static_cast<__nv_bfloat16*>(out);
+    cudaStream_t hst = static_cast<cudaStream_t>(stream);
+    const bool htimed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
+    if (htimed) cudaEventRecord(c->prof_ev[2 * c->prof_n], hst);
+    if (launch_decode_heads(hp, hst) != cudaSuccess) return SSD_ERR_CUDA;
+    c->claim_parity ^= 1;
+    c->last_writer = -1;
+    if (htimed) {
+      cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], hst);
+      c->prof_n += 1;
+    }
+    return SSD_OK;
+  }
   DecodeParams p;
   p.slab = c->d_slab(layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -541,14 +601,60 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
+       reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
+    return SSD_ERR_INVALID_ARG;
+  if (c->heads_form()) {
+    // one launch in every mode: heads are handed out whole to thread blocks, so the block that finishes a
+    // semantic head also maintains its scores (Algorithm 2) and, with a buffer of one token, re-selects
+    if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+    const bool scored = c->row_buffer && c->n_sink[layer] > 0;
+    if (scored && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;   // Algorithm 2, overflow branch
+    cudaStream_t hst = static_cast<cudaStream_t>(stream);
+    if (scored && c->pending[layer]) {   // a decode by the equal-shares kernel left its weights pending: add them first
+      if (launch_fold_pending(c->d_acc(layer), c->d_logits(layer), c->d_ml(layer), c->d_desc(layer), g.n_seqs, g.n_heads,
+                              c->mr(), c->static_valid[layer], c->sem_tokens(layer), hst) != cudaSuccess)
+        return SSD_ERR_CUDA;
+    }
+    c->pending[layer] = 0;
+    const bool evict = c->row_buffer && g.sink_recent == 1;
+    DecodeHeadsParams hp;
+    c->fill_heads(layer, hp);
+    hp.q = static_cast<const unsigned char*>(q);
+    hp.k_new = static_cast<const unsigned char*>(k_new);
+    hp.v_new = static_cast<const unsigned char*>(v_new);
+    hp.out = static_cast<__nv_bfloat16*>(out);
+    hp.new_j = c->t_img[layer];
+    hp.sem_slot = c->sem_tokens(layer);
+    hp.t_img = c->t_img[layer] + 1;
+    hp.t_sem = hp.sem_slot + 1;
+    if (!c->row_buffer) { hp.sem_slot = 0; hp.t_sem = hp.t_img; }
+    if (c->row_buffer) {
+      hp.acc = c->d_acc(layer);
+      hp.mr = c->mr();
+      hp.evict = evict ? 1 : 0;
+    }
+    const bool htimed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
+    if (htimed) cudaEventRecord(c->prof_ev[2 * c->prof_n], hst);
+    if (launch_decode_heads(hp, hst) != cudaSuccess) return SSD_ERR_CUDA;
+    c->claim_parity ^= 1;
+    c->t_img[layer] += 1;
+    if (evict) {                         // the buffer is empty again: the token entered the static set or left
+      if (c->n_sink[layer] > 0 && c->static_valid[layer] < g.sink_budget) c->static_valid[layer] += 1;
+      c->t_base[layer] = c->t_img[layer];
+    }
+    c->last_writer = layer;
+    if (htimed) {
+      cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], hst);
+      c->prof_n += 1;
+    }
+    return SSD_OK;
+  }
   if (c->row_buffer) {                 // the row buffer's append also maintains the scores: two launches
     const int rc = ssd_append(c, layer, k_new, v_new, stream);
     return rc != SSD_OK ? rc : ssd_decode_attn(c, layer, q, out, stream);
   }
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
-  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
-       reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
-    return SSD_ERR_INVALID_ARG;
   DecodeParams p;
   p.slab = c->d_slab(layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -831,6 +937,12 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
 int ssd_cache_set_prefetch(ssd_cache* c, int32_t slots) {
   if (!c || slots < 0 || slots > 4096) return SSD_ERR_INVALID_ARG;
   c->pf_slots = slots;
+  return SSD_OK;
+}
+
+int ssd_cache_set_decode_form(ssd_cache* c, int32_t form) {
+  if (!c || form < 0 || form > 2) return SSD_ERR_INVALID_ARG;
+  c->decode_form = form;
   return SSD_OK;
 }
 

@@ -46,9 +46,10 @@ def reduce_ratio_sums(local_sums: np.ndarray, group=None) -> np.ndarray:
 
 
 def labels_from_sums(total_sums: np.ndarray, n_cal_total: int, n_img: int, tau: float) -> np.ndarray:
-    """label = s > tau with s = sums / (P * N), decided in float32 like the single-GPU entry point."""
-    s = (np.asarray(total_sums, np.float64) / (float(n_cal_total) * float(n_img))).astype(np.float32)
-    return (s > np.float32(tau)).astype(np.uint8)
+    """Labels from ratio sums added over ranks: the library's own threshold rule
+    (ssd_labels_from_ratio_sums, the arithmetic ssd_classify_heads uses), not a restatement of it."""
+    from . import binding
+    return binding.labels_from_ratio_sums(total_sums, n_cal_total, n_img, tau)[1]
 
 
 def classify_sharded(cache, q_cal_local, k_cal_local, n_cal_total: int, n_img: int, tau: float, group=None):

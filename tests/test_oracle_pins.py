@@ -466,3 +466,43 @@ def test_rowbuf_of_one_is_the_drop_one_rule_of_algorithm_1():
         kept = sorted(held)
         assert hist[i][0] == t and hist[i][1] == kept and hist[i][3] == []
         assert np.allclose(hist[i][2], [score[j] for j in kept], rtol=1e-12, atol=0)
+
+
+def test_kv_token_mse_pins():
+    """Sec. 3.2, MSE_token: identical caches give 0; one perturbed element gives its squared change at
+    that token only; the sum over tokens is the squared Frobenius distance of K plus that of V (library
+    norm); a Python-loop restatement on a small case; symmetry in the two caches; K and V both count."""
+    g = torch.Generator().manual_seed(11)
+    shape = (2, 3, 7, 16)
+    Ka, Va, Kb, Vb = (torch.randn(shape, generator=g).to(torch.bfloat16) for _ in range(4))
+    ua, uva, ub, uvb = (wl.to_u16(x) for x in (Ka, Va, Kb, Vb))
+    assert np.array_equal(oracle.kv_token_mse(ua, uva, ua, uva), np.zeros(shape[:-1]))
+    # one element of V changed by a known amount, at (1, 2, 5, 3)
+    Vp = Va.clone()
+    Vp[1, 2, 5, 3] = Va[1, 2, 5, 3] + 0.5
+    delta = float(Vp[1, 2, 5, 3].double() - Va[1, 2, 5, 3].double())      # after bf16 rounding
+    got = oracle.kv_token_mse(ua, wl.to_u16(Vp), ua, uva)
+    want = np.zeros(shape[:-1])
+    want[1, 2, 5] = delta * delta
+    assert np.array_equal(got, want) and delta != 0.0
+    # the same through K: both tensors count, and separately
+    Kp = Ka.clone()
+    Kp[0, 0, 0, 15] = Ka[0, 0, 0, 15] * 2
+    d2 = float(Kp[0, 0, 0, 15].double() - Ka[0, 0, 0, 15].double())
+    got = oracle.kv_token_mse(wl.to_u16(Kp), wl.to_u16(Vp), ua, uva)
+    assert got[0, 0, 0] == d2 * d2 and got[1, 2, 5] == delta * delta and got.sum() == d2 * d2 + delta * delta
+    # sum over tokens = squared Frobenius distances (numpy's norm), per (i, h)
+    m = oracle.kv_token_mse(ua, uva, ub, uvb)
+    for i in range(shape[0]):
+        for h in range(shape[1]):
+            fro = (np.linalg.norm((Ka[i, h].double() - Kb[i, h].double()).numpy()) ** 2 +
+                   np.linalg.norm((Va[i, h].double() - Vb[i, h].double()).numpy()) ** 2)
+            assert math.isclose(m[i, h].sum(), fro, rel_tol=1e-12)
+    # plain loops on one (i, h)
+    for j in range(shape[2]):
+        acc = 0.0
+        for d in range(shape[3]):
+            acc += (float(Ka[1, 0, j, d]) - float(Kb[1, 0, j, d])) ** 2 + (float(Va[1, 0, j, d]) - float(Vb[1, 0, j, d])) ** 2
+        assert math.isclose(m[1, 0, j], acc, rel_tol=1e-12)
+    assert np.array_equal(m, oracle.kv_token_mse(ub, uvb, ua, uva))
+    assert (m > 0).all()
