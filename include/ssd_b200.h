@@ -151,28 +151,6 @@ int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, v
 int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new,
                       const void *q, void *out, void *stream);
 
-/* Hand-over between consecutive per-layer launches (no paper counterpart; a scheduling hint).  A caller
- * that goes round the layers (layer 0, 1, .., n_layers-1, 0, ..) issues launches whose first copies find
- * HBM idle while the previous launch drains.  To close that gap each decode worker, once its own last
- * copy is issued, asks the L2 cache to fetch the first `slots` slots (512 B each) of the same share of
- * the NEXT layer's slab.  It applies only when both layers are full (prompt, static sets and rings hold
- * tokens in every slot) and of equal size; it never changes results.  slots = 0 switches it off (useful
- * when other kernels that sweep the L2 cache run between the layers' calls); the default is 48.
- * SSD_ERR_INVALID_ARG if slots < 0 or > 4096. */
-int ssd_cache_set_prefetch(ssd_cache *cache, int32_t slots);
-
-/* Which kernel ssd_decode_attn and ssd_append_decode launch (no paper counterpart; both compute the same
- * attention, results differ only in the rounding order of the softmax sums):
- *   1  equal shares: the layer's slots are cut into equal byte ranges, one per warp; a head cut by a
- *      range boundary is merged through scratch memory.  Best when a layer has few, long heads.
- *   2  heads to thread blocks: a thread block claims whole heads from a counter and its warps share each
- *      head's chunks, so a slower SM takes fewer heads.  Best when every SM gets many heads.  In row-buffer
- *      mode ssd_append_decode is then ONE launch that also maintains the scores (and, with sink_recent = 1,
- *      re-selects, which is Algorithm 1 taken literally).
- *   0  (default) form 2 when the layer has at least 8 heads per SM (n_seqs * n_heads >= 8 * SMs), else 1.
- * SSD_ERR_INVALID_ARG for other values. */
-int ssd_cache_set_decode_form(ssd_cache *cache, int32_t form);
-
 /* ssd_append_decode for n_layers consecutive layers in ONE launch (a whole decode step when the
  * inputs of all layers exist up front, as in a benchmark of this path or a host-driven replay; in a
  * model, layer l+1's query depends on layer l's output and the per-layer call is the one to use).
@@ -234,9 +212,7 @@ int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
  * allocation's implicit synchronisation is not acceptable.  For them the same scratch is a fixed
  * array inside the library image (about 0.4 MB, held by every GPU that loads the library until the
  * process ends), and this call allocates nothing, on the device or through any library.
- *   Same arguments, results and errors as ssd_decode_attn (it runs the equal-shares kernel: outputs are
- *   bit-identical to ssd_decode_attn's when that call runs the same kernel, see
- *   ssd_cache_set_decode_form, and equal up to the rounding order of the softmax sums otherwise), plus
+ *   Same arguments, results and errors as ssd_decode_attn (outputs are bit-identical), plus
  *   SSD_ERR_LIMIT if n_seqs * n_heads > 32768 or the GPU has more than 256 SMs: the array is sized
  *   for those maxima.
  * The first call on each device looks up the array's device address (a synchronous runtime query);

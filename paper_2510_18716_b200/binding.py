@@ -31,7 +31,7 @@ EXPORTS = [
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
-    "ssd_cache_set_prefetch", "ssd_cache_set_decode_form", "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity",
+    "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity",
 ]
 
 
@@ -80,8 +80,6 @@ def load():
     L.ssd_decode_attn_static.argtypes = [vp, i32, vp, vp, vp]
     L.ssd_append_decode.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_cache_set_row_buffer.argtypes = [vp, i32]
-    L.ssd_cache_set_prefetch.argtypes = [vp, i32]
-    L.ssd_cache_set_decode_form.argtypes = [vp, i32]
     L.ssd_labels_from_ratio_sums.argtypes = [vp, C.c_int64, i32, i32, C.c_float, vp, vp]
     L.ssd_labels_from_sparsity.argtypes = [vp, C.c_int64, C.c_float, vp]
     L.ssd_recompress.argtypes = [vp, i32, vp]
@@ -299,14 +297,6 @@ class SsdCache:
     # -- Algorithm 2 (row buffer)
     def set_row_buffer(self, enable: bool = True):
         self._check(self.lib.ssd_cache_set_row_buffer(self._h, 1 if enable else 0), "ssd_cache_set_row_buffer")
-
-    def set_prefetch(self, slots: int):
-        """Slots of the next layer each decode worker asks L2 to fetch at its end (0 = off)."""
-        self._check(self.lib.ssd_cache_set_prefetch(self._h, int(slots)), "ssd_cache_set_prefetch")
-
-    def set_decode_form(self, form: int):
-        """Per-layer decode kernel: 0 chosen by size, 1 equal shares, 2 heads handed out to thread blocks."""
-        self._check(self.lib.ssd_cache_set_decode_form(self._h, int(form)), "ssd_cache_set_decode_form")
 
     def recompress(self, layer: int):
         self._check(self.lib.ssd_recompress(self._h, layer, _stream()), "ssd_recompress")

@@ -20,8 +20,6 @@ static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 // staging slots; a slot holds q, k_new, v_new and out of a whole group.
 constexpr int kHostGroup = 4;
 constexpr int kHostSlots = 3;
-// Slots of the next layer each decode worker asks the L2 cache to fetch when its own copies are issued.
-constexpr int kDefaultPrefetchSlots = 0;
 
 struct Regions {
   size_t desc, idx, counters, status, partial, score, staging, acc, logits, ml, slab;  // byte offsets
@@ -52,8 +50,7 @@ static Regions plan_regions(const ssd_config& c) {
   r.desc = off;      off = align_up(off + (size_t)c.n_layers * c.n_heads * sizeof(HeadDesc));
   r.idx = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * (c.sink_budget > 0 ? c.sink_budget : 1) * 4);
   r.counters = off;  off = align_up(off + pairs_layer * 4);
-  r.status = off;    off = align_up(off + 200);   // status word; at +128 the unit counter of the all-layers launch;
-                                                  // at +192 the two claim counters of the heads-to-blocks launch
+  r.status = off;    off = align_up(off + 132);   // status word, and at +128 the unit counter of the all-layers launch
   r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
   r.partial = off;   off = align_up(off + r.partial_bytes);
   r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4;
@@ -99,9 +96,6 @@ struct ssd_cache {
   cudaEvent_t h_fork = nullptr, h_loaded[kHostSlots] = {}, h_done[kHostSlots] = {}, h_stored[kHostSlots] = {};
   long h_groups = 0;                  // groups sent through the staging ring so far
   bool h_foreign = false;             // ssd_step_host has used the staging area since
-  int pf_slots = kDefaultPrefetchSlots;   // L2 hand-over depth per worker (ssd_cache_set_prefetch)
-  int decode_form = 0;                // per-layer decode kernel: 0 chosen by size, 1 equal shares, 2 heads to blocks
-  int claim_parity = 0;               // which claim counter the next heads-to-blocks launch uses
   std::vector<cudaEvent_t> prof_ev;   // 2 events per timed decode launch (empty = timing off)
   int prof_n = 0;                     // launches recorded since the last collect
 
@@ -112,29 +106,6 @@ struct ssd_cache {
   }
   uint32_t* d_counters() const { return reinterpret_cast<uint32_t*>(base + reg.counters); }
   uint32_t* d_status() const { return reinterpret_cast<uint32_t*>(base + reg.status); }
-  uint32_t* d_claim() const { return reinterpret_cast<uint32_t*>(base + reg.status + 192); }
-  // Per-layer decode with heads handed out to thread blocks: worth it when every SM gets many heads
-  // (else equal shares balance better), and possible while a head's score row fits its table entry.
-  bool heads_form() const {
-    if (decode_form == 1) return false;
-    if (row_buffer && mr() > decode_heads_max_mr(0)) return false;
-    return decode_form == 2 || (long)cfg.n_seqs * cfg.n_heads >= decode_heads_min_pairs();
-  }
-  void fill_heads(int layer, DecodeHeadsParams& p) {
-    p.slab = d_slab(layer);
-    p.desc = d_desc(layer);
-    p.status = d_status();
-    p.claim = d_claim();
-    p.parity = claim_parity;
-    p.n_seqs = cfg.n_seqs; p.H = cfg.n_heads; p.L = cfg.prompt_len; p.seq_slots = seq_slots[layer];
-    p.prompt_valid = prompt_valid[layer];
-    p.static_valid = static_valid[layer];
-    p.t_img = t_img[layer];
-    p.t_sem = sem_tokens(layer);
-    p.early = (last_writer >= -1 && last_writer != layer) ? 1 : 0;
-    p.acc = nullptr; p.static_idx = d_idx(layer); p.M = cfg.sink_budget; p.mr = 0; p.evict = 0;
-    p.scale_log2 = scale * 1.4426950408889634f;
-  }
   uint32_t* d_work() const { return reinterpret_cast<uint32_t*>(base + reg.status + 128); }   // unit counter of the all-layers launch
   int mr() const { return cfg.sink_budget + cfg.sink_recent; }
   size_t layer_scores(int layer) const { return (size_t)layer * cfg.n_seqs * cfg.n_heads * mr(); }
@@ -152,25 +123,6 @@ struct ssd_cache {
   int max_slots() const {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
     return cfg.prompt_len + (a > b ? a : b);
-  }
-  // True if every slot of the layer will hold a token once the layer holds t image tokens (t_sem of them
-  // in the rings of semantic heads): the layer's valid slots are then its whole slab, in slab order.
-  bool layer_full(int layer, int t, int t_sem) const {
-    if (prompt_valid[layer] != cfg.prompt_len) return false;
-    if (n_sink[layer] > 0 && (static_valid[layer] != cfg.sink_budget || t_sem < cfg.sink_recent)) return false;
-    if (n_sink[layer] < cfg.n_heads && t < cfg.window) return false;
-    return true;
-  }
-  // Where a launch on `layer` (which will hold t / t_sem tokens when it runs) hands over to: the slab of
-  // the layer a caller going round the layers attends to next, if both layers are full and of the same
-  // size, so that a worker's share covers the same byte range in both; else null.
-  const unsigned char* hand_over_to(int layer, int t, int t_sem) const {
-    if (pf_slots <= 0 || cfg.n_layers < 2) return nullptr;
-    const int nl = layer + 1 < cfg.n_layers ? layer + 1 : 0;
-    const int tn = t_img[nl] + 1 < cfg.max_image_tokens ? t_img[nl] + 1 : cfg.max_image_tokens;
-    const int tn_sem = row_buffer ? sem_tokens(nl) + 1 : tn;
-    if (seq_slots[nl] != seq_slots[layer] || !layer_full(layer, t, t_sem) || !layer_full(nl, tn, tn_sem)) return nullptr;
-    return reinterpret_cast<const unsigned char*>(d_slab(nl));
   }
   // layout and occupancy of a layer, as the decode kernel sees it
   void fill_view(int layer, LayerView& v) const {
@@ -547,24 +499,6 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
-  if (!c->row_buffer && c->heads_form()) {
-    DecodeHeadsParams hp;
-    c->fill_heads(layer, hp);
-    hp.q = static_cast<const unsigned char*>(q);
-    hp.k_new = nullptr; hp.v_new = nullptr; hp.new_j = -1; hp.sem_slot = 0;
-    hp.out = static_cast<__nv_bfloat16*>(out);
-    cudaStream_t hst = static_cast<cudaStream_t>(stream);
-    const bool htimed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
-    if (htimed) cudaEventRecord(c->prof_ev[2 * c->prof_n], hst);
-    if (launch_decode_heads(hp, hst) != cudaSuccess) return SSD_ERR_CUDA;
-    c->claim_parity ^= 1;
-    c->last_writer = -1;
-    if (htimed) {
-      cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], hst);
-      c->prof_n += 1;
-    }
-    return SSD_OK;
-  }
   DecodeParams p;
   p.slab = c->d_slab(layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -579,8 +513,6 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
-  p.next_slab = c->hand_over_to(layer, c->t_img[layer], c->sem_tokens(layer));
-  p.pf_slots = c->pf_slots;
   c->fill_view(layer, p.view);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
@@ -604,52 +536,6 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
-  if (c->heads_form()) {
-    // one launch in every mode: heads are handed out whole to thread blocks, so the block that finishes a
-    // semantic head also maintains its scores (Algorithm 2) and, with a buffer of one token, re-selects
-    if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
-    const bool scored = c->row_buffer && c->n_sink[layer] > 0;
-    if (scored && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;   // Algorithm 2, overflow branch
-    cudaStream_t hst = static_cast<cudaStream_t>(stream);
-    if (scored && c->pending[layer]) {   // a decode by the equal-shares kernel left its weights pending: add them first
-      if (launch_fold_pending(c->d_acc(layer), c->d_logits(layer), c->d_ml(layer), c->d_desc(layer), g.n_seqs, g.n_heads,
-                              c->mr(), c->static_valid[layer], c->sem_tokens(layer), hst) != cudaSuccess)
-        return SSD_ERR_CUDA;
-    }
-    c->pending[layer] = 0;
-    const bool evict = c->row_buffer && g.sink_recent == 1;
-    DecodeHeadsParams hp;
-    c->fill_heads(layer, hp);
-    hp.q = static_cast<const unsigned char*>(q);
-    hp.k_new = static_cast<const unsigned char*>(k_new);
-    hp.v_new = static_cast<const unsigned char*>(v_new);
-    hp.out = static_cast<__nv_bfloat16*>(out);
-    hp.new_j = c->t_img[layer];
-    hp.sem_slot = c->sem_tokens(layer);
-    hp.t_img = c->t_img[layer] + 1;
-    hp.t_sem = hp.sem_slot + 1;
-    if (!c->row_buffer) { hp.sem_slot = 0; hp.t_sem = hp.t_img; }
-    if (c->row_buffer) {
-      hp.acc = c->d_acc(layer);
-      hp.mr = c->mr();
-      hp.evict = evict ? 1 : 0;
-    }
-    const bool htimed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
-    if (htimed) cudaEventRecord(c->prof_ev[2 * c->prof_n], hst);
-    if (launch_decode_heads(hp, hst) != cudaSuccess) return SSD_ERR_CUDA;
-    c->claim_parity ^= 1;
-    c->t_img[layer] += 1;
-    if (evict) {                         // the buffer is empty again: the token entered the static set or left
-      if (c->n_sink[layer] > 0 && c->static_valid[layer] < g.sink_budget) c->static_valid[layer] += 1;
-      c->t_base[layer] = c->t_img[layer];
-    }
-    c->last_writer = layer;
-    if (htimed) {
-      cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], hst);
-      c->prof_n += 1;
-    }
-    return SSD_OK;
-  }
   if (c->row_buffer) {                 // the row buffer's append also maintains the scores: two launches
     const int rc = ssd_append(c, layer, k_new, v_new, stream);
     return rc != SSD_OK ? rc : ssd_decode_attn(c, layer, q, out, stream);
@@ -670,8 +556,6 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->t_img[layer] += 1;                // the view describes the layer with the token in place
-  p.next_slab = c->hand_over_to(layer, c->t_img[layer], c->sem_tokens(layer));
-  p.pf_slots = c->pf_slots;
   c->fill_view(layer, p.view);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
@@ -934,18 +818,6 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
   return SSD_OK;
 }
 
-int ssd_cache_set_prefetch(ssd_cache* c, int32_t slots) {
-  if (!c || slots < 0 || slots > 4096) return SSD_ERR_INVALID_ARG;
-  c->pf_slots = slots;
-  return SSD_OK;
-}
-
-int ssd_cache_set_decode_form(ssd_cache* c, int32_t form) {
-  if (!c || form < 0 || form > 2) return SSD_ERR_INVALID_ARG;
-  c->decode_form = form;
-  return SSD_OK;
-}
-
 int ssd_cache_set_row_buffer(ssd_cache* c, int32_t enable) {
   if (!c) return SSD_ERR_INVALID_ARG;
   c->row_buffer = enable != 0;
@@ -1193,8 +1065,6 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
-  p.next_slab = nullptr;
-  p.pf_slots = 0;
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;

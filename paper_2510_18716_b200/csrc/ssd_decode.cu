@@ -35,8 +35,6 @@
 // during the launch, so no ordering is needed, and the per-layer append launch disappears.
 // Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
 // waits (bounded again) for its other copies in flight and leaves.
-#include <atomic>
-
 #include "ssd_internal.cuh"
 
 #ifndef SSD_DECODE_WARPS
@@ -141,12 +139,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 // transitively; and when a kernel starts, everything before its predecessor has completed (the
 // predecessor passed its own wait before allowing it), which is what makes the slab prefetch of the
 // decode kernel's prologue safe.
-// Ask the L2 cache to fetch [src, src + bytes) (16-byte aligned, a multiple of 16): no destination, no
-// completion to wait for.
-__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-
 __device__ __forceinline__ void pdl_allow_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -565,23 +557,6 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     }
   }
 
-  // Once the last copy of the share has been issued this worker's demand on HBM ends: fill the gap
-  // with the start of the same share of the next layer, in the order the next launch will read it.
-  bool handed_over = p.next_slab == nullptr || p.pf_slots <= 0;
-  auto hand_over = [&]() {
-    handed_over = true;
-    if (lane != 0) return;
-    int left = p.pf_slots;
-    const int a0 = two_parts ? g_tail : g_begin;
-    const int n0 = left < g_end - a0 ? left : g_end - a0;
-    l2_prefetch(p.next_slab + (size_t)a0 * kSlotBytes, (uint32_t)n0 * kSlotBytes);
-    left -= n0;
-    if (two_parts && left > 0) {
-      const int n1 = left < g_tail - g_begin ? left : g_tail - g_begin;
-      l2_prefetch(p.next_slab + (size_t)g_begin * kSlotBytes, (uint32_t)n1 * kSlotBytes);
-    }
-  };
-
   int stage = 0;
   uint32_t parity = 0;
   bool begin = true, leading = true;
@@ -637,7 +612,6 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
     if (prod.g < prod.g_end) issue(stage);
-    else if (!handed_over) hand_over();
     fold_stage(rows, n, grp, l8, q, st, sink);
 
     const int i1 = cons.i + n;
@@ -729,8 +703,6 @@ struct Unit {
   int contig;                   // the valid slots are one physical run
   int u;                        // the unit's number
   int scored;                   // 1: a semantic head whose attention scores are accumulated (Algorithm 2)
-  int nch;                      // per-layer kernel with heads handed out to blocks: chunks of the head, 0 = none left
-  int pad;
 };
 
 __device__ __forceinline__ void unit_load(const DecodeLayersParams& p, int u, Unit& U) {
@@ -1002,464 +974,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_kernel(const
   }
 }
 
-// ------------------------------------------------------------------ one layer, heads handed out to thread blocks
-// The per-layer launch for layers with many heads per SM.  Equal static shares (ssd_decode_kernel) make
-// every warp move the same bytes, but warps and SMs do not run at the same speed, and a launch lasts as
-// long as its slowest warp.  Here a thread block claims whole heads, one at a time, from a counter, so a
-// slower SM simply takes fewer; inside the block the chunks of the claimed heads form one stream that
-// the block's warps share round-robin (chunk g of the stream belongs to warp g mod kWarps).  A head is
-// therefore never cut between blocks, and its pieces meet in shared memory: partial r of a head holds its
-// chunks r, r + kWarps, ..; the warp that posts the last one merges them in the order of r and writes
-// the output row, so results do not depend on who claimed what.  An extra warp (the feeder) claims heads
-// and publishes their descriptions in a table of kTable open heads in shared memory, as far ahead of the
-// slowest consumer as the table allows (an entry is reused once every worker has moved past its head);
-// the first kLook heads of a block are fixed (block b takes heads b, b + grid, ..) so that their copies can
-// start before the preceding launch has ended.  The claim counters alternate between launches: a launch
-// uses one and clears the other for its successor, so no memset stands between two launches.
-// In row-buffer mode (Algorithm 2) the logits of a semantic head are kept in shared memory beside its
-// table entry and the merging warp, which knows the head's final (max, sum), adds the step's weights to
-// the head's score row; with a row buffer of one token (Algorithm 1 taken literally) it also re-selects.
-constexpr int kTable = 8;     // heads a block can have open (table entries, partial sets, logit rows)
-constexpr int kLook = 4;      // heads of a block that are fixed by its number rather than claimed
-constexpr int kHeadsThreads = (kWarps + 1) * 32;
-// table: entries, then per entry its published number and its count of posted partials, then per worker
-// the oldest entry it still needs, then the block's abort flag, then the layer's head records
-constexpr int kHeadsFlags = 2 * kTable + kWarps + 1;
-constexpr int kHeadsTableBytes = (kTable * (int)sizeof(Unit) + kHeadsFlags * 4 + 15) & ~15;
-constexpr int kHeadsPartialBytes = kTable * kWarps * kPartialFloats * 4;
-constexpr int kHeadsDescBytes = kMaxHeads * (int)sizeof(HeadDesc);
-constexpr int kHeadsSmemBytes = kRingBytes + kWarps * kStages * 8 + kHeadsTableBytes + kHeadsPartialBytes + kHeadsDescBytes;
-static_assert(kHeadsTableBytes % 16 == 0 && sizeof(Unit) % 16 == 0, "partials are read as float4");
-static_assert(kLook <= kTable, "the fixed heads are published without waiting for a free entry");
-constexpr int kAtEnd = 0x7fffffff;
-
-__device__ __forceinline__ void head_load(const DecodeHeadsParams& p, const HeadDesc* desc, int pair, Unit& U) {
-  const int seq = pair / p.H, head = pair - seq * p.H;
-  const HeadDesc d = desc[head];
-  U.u = pair;
-  U.scored = (p.acc != nullptr && d.w) ? 1 : 0;
-  const int held = U.scored ? p.t_sem : p.t_img;                 // tokens the ring holds
-  U.pv = p.prompt_valid;
-  U.sv = d.w ? p.static_valid : 0;
-  U.y = d.y;
-  U.vh = U.pv + U.sv + (held < d.z ? held : d.z);
-  if (p.new_j >= 0) {
-    const int r = U.scored ? p.sem_slot : p.new_j % d.z;         // ring slot of the token being appended
-    U.fresh = U.pv + U.sv + r;
-    U.phys = p.L + d.y + r;
-  } else {
-    U.fresh = -1;
-    U.phys = 0;
-  }
-  U.contig = (U.pv == p.L && U.sv == d.y) ? 1 : 0;
-  U.hbase = reinterpret_cast<const unsigned char*>(p.slab) + ((size_t)seq * p.seq_slots + d.x) * kSlotBytes;
-  U.row = (size_t)pair * kQBytes;
-  U.nch = (U.vh + kChunk - 1) / kChunk;
-  U.pad = 0;
-}
-
-// Wait (bounded) until cond() holds for some lane; false if the wait ran out or the block has given up.
-template <class Cond>
-__device__ __forceinline__ bool wait_until(Cond cond, const volatile int* abort) {
-  const uint32_t FULL = 0xffffffffu;
-  if (__any_sync(FULL, cond())) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i) {
-      if (__any_sync(FULL, cond())) return true;
-      __nanosleep(20);
-    }
-    if (__any_sync(FULL, *abort != 0) || global_ns() - t0 >= kWaitLimitNs) return false;
-  }
-}
-
-template <bool kEvict>
-__global__ void __launch_bounds__(kHeadsThreads, 1) ssd_decode_heads_kernel(const __grid_constant__ DecodeHeadsParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int grp = lane >> 3, l8 = lane & 7;
-  const uint32_t FULL = 0xffffffffu;
-  unsigned char* tbl = smem + kRingBytes + kWarps * kStages * 8;
-  Unit* ent = reinterpret_cast<Unit*>(tbl);
-  int* flags = reinterpret_cast<int*>(tbl + kTable * sizeof(Unit));
-  volatile int* pub = flags;                       // [kTable] entry k is published: k + 1
-  int* arrive = flags + kTable;                    // [kTable] partials posted for the entry
-  volatile int* at = flags + 2 * kTable;           // [kWarps] oldest entry the worker still needs
-  volatile int* abort = flags + 2 * kTable + kWarps;
-  float* partials = reinterpret_cast<float*>(tbl + kHeadsTableBytes);
-  HeadDesc* desc = reinterpret_cast<HeadDesc*>(tbl + kHeadsTableBytes + kHeadsPartialBytes);
-  const int mrp = (p.mr + 3) & ~3;
-  float* logit_rows = reinterpret_cast<float*>(smem + kHeadsSmemBytes);   // [kTable][mrp], row-buffer mode
-  const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
-  if (threadIdx.x < kHeadsFlags) flags[threadIdx.x] = 0;
-  if (threadIdx.x < p.H) desc[threadIdx.x] = __ldg(p.desc + threadIdx.x);   // fixed since the labels were set
-  if (lane == 0 && warp < kWarps) {
-#pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
-    mbar_init_fence();
-  }
-  __syncthreads();   // the only block-wide barrier
-  const int n_pairs = p.n_seqs * p.H;
-  auto give_up = [&]() {
-    if (lane == 0) {
-      atomicOr(p.status, 1u);
-      *abort = 1;
-    }
-  };
-
-  if (warp == kWarps) {
-    // ---- the feeder: publishes the heads this block works on
-    auto publish = [&](int k, int pair) -> bool {
-      const int slot = k % kTable;
-      // the slot's previous head is finished once every worker has moved past it
-      if (k >= kTable && !wait_until([&]() {
-            int lo = kAtEnd;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) lo = at[w] < lo ? at[w] : lo;
-            return lo > k - kTable;
-          }, abort)) {
-        give_up();
-        return false;
-      }
-      if (lane == 0) {
-        Unit U;
-        if (pair < n_pairs) {
-          head_load(p, desc, pair, U);
-        } else {
-          U = Unit{};                    // nch = 0: no more heads
-        }
-        ent[slot] = U;
-        arrive[slot] = 0;
-        __threadfence_block();
-        pub[slot] = k + 1;
-      }
-      __syncwarp();
-      return true;
-    };
-    bool more = true;
-#pragma unroll 1
-    for (int k = 0; k < kLook && more; ++k) {
-      const int pair = (int)blockIdx.x + k * (int)gridDim.x;
-      publish(k, pair);
-      more = pair < n_pairs;
-    }
-    pdl_wait_predecessor();              // the claim counters belong to the preceding launch until it has ended
-    pdl_allow_successor();
-    if (blockIdx.x == 0 && lane == 0) p.claim[p.parity ^ 1] = 0u;
-    // one claim is always in flight while the one before it is being published
-    auto claim = [&]() { return kLook * (int)gridDim.x + (int)atomicAdd(p.claim + p.parity, 1u); };
-    int next = 0;
-    if (more && lane == 0) next = claim();
-#pragma unroll 1
-    for (int k = kLook; more; ++k) {
-      const int pair = __shfl_sync(FULL, next, 0);
-      more = pair < n_pairs;
-      if (more && lane == 0) next = claim();
-      if (!publish(k, pair)) break;
-    }
-    return;
-  }
-
-  // ---- a worker: chunks warp, warp + kWarps, .. of the block's chunk stream
-  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
-  const uint32_t ring_s = smem_u32(ring);
-  // A position in the stream is an entry k of the table and the number c0 of that entry's first chunk.
-  // Move (k, c0) to the entry that holds chunk g and return its chunk count; 0: the stream ends before g;
-  // -1: the entry that would decide is not published yet (only when `block` is false); -2: gave up.
-  auto locate = [&](int& k, int& c0, int g, bool block) -> int {
-    for (;;) {
-      const int slot = k % kTable;
-      if (!__any_sync(FULL, pub[slot] >= k + 1)) {
-        if (!block) return -1;
-        if (!wait_until([&]() { return pub[slot] >= k + 1; }, abort)) return -2;
-      }
-      __threadfence_block();
-      const int nch = ent[slot].nch;
-      if (nch == 0) return 0;
-      if (g < c0 + nch) return nch;
-      c0 += nch;
-      ++k;
-    }
-  };
-
-  int pk = 0, pc0 = 0, pg = warp;       // producer side
-  int ck = 0, cc0 = 0, cg = warp;       // consumer side
-  int ahead = 0;                        // chunks issued and not yet consumed
-  bool feeding = true;
-
-  // Lane 0 starts the copies of chunk j of head U into `stage`.  what & 1: the slab part (and the barrier's
-  // byte count for the whole chunk); what & 2: the caller's inputs (query row, the newest token's rows).
-  auto copy_chunk = [&](const Unit& U, int j, int stage, int what) {
-    const int i0 = j * kChunk;
-    const int n = U.vh - i0 < kChunk ? U.vh - i0 : kChunk;
-    const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
-    const bool has_fresh = U.fresh >= i0 && U.fresh < i0 + n;
-    if (what & 1) {
-      // order the warp's reads of this stage (made visible to this lane by __syncwarp) before the
-      // asynchronous writes that follow
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + kQBytes));
-      auto copy_range = [&](int a, int len, int to) {
-        if (len <= 0) return;
-        if (U.contig) {
-          bulk_g2s(dst + (uint32_t)to * kSlotBytes, U.hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
-          return;
-        }
-        const int l0[3] = {0, U.pv, U.pv + U.sv};          // logical start of each run
-        const int l1[3] = {U.pv, U.pv + U.sv, U.vh};       // and end
-        const int p0[3] = {0, p.L, p.L + U.y};             // physical start
-#pragma unroll
-        for (int r = 0; r < 3; ++r) {
-          const int lo = a > l0[r] ? a : l0[r], hi = a + len < l1[r] ? a + len : l1[r];
-          if (hi > lo)
-            bulk_g2s(dst + (uint32_t)(to + lo - a) * kSlotBytes, U.hbase + (size_t)(p0[r] + lo - l0[r]) * kSlotBytes,
-                     (uint32_t)(hi - lo) * kSlotBytes, bar);
-        }
-      };
-      if (has_fresh) {                   // the slab is copied around the newest token's slot
-        copy_range(i0, U.fresh - i0, 0);
-        copy_range(U.fresh + 1, i0 + n - U.fresh - 1, U.fresh + 1 - i0);
-      } else {
-        copy_range(i0, n, 0);
-      }
-    }
-    if (what & 2) {
-      if (has_fresh) {
-        bulk_g2s(dst + (uint32_t)(U.fresh - i0) * kSlotBytes, p.k_new + U.row, kQBytes, bar);
-        bulk_g2s(dst + (uint32_t)(U.fresh - i0) * kSlotBytes + kQBytes, p.v_new + U.row, kQBytes, bar);
-      }
-      bulk_g2s(dst + kChunk * kSlotBytes, p.q + U.row, kQBytes, bar);
-    }
-  };
-  // The producer's next chunk into `stage`; every lane advances.  A producer never waits for the feeder
-  // while the warp still has chunks to fold (the feeder may be waiting for just those).
-  auto issue = [&](int stage, int what, bool block) {
-    const int nch = locate(pk, pc0, pg, block);
-    if (nch == -1) return;               // not published yet: try again after the next chunk
-    if (nch <= 0) {
-      feeding = false;
-      if (nch == -2) give_up();
-      return;
-    }
-    if (lane == 0) copy_chunk(ent[pk % kTable], pg - pc0, stage, what);
-    pg += kWarps;
-    ++ahead;
-  };
-  // let the copies in flight land (bounded) before the block's shared memory is given back
-  auto drain = [&](int stage, uint32_t parity) {
-    for (int k = 0; k < ahead; ++k) {
-      mbar_wait(bar0 + 8 * stage, parity);
-      if (++stage == kStages) { stage = 0; parity ^= 1u; }
-    }
-  };
-
-  // Prologue: the slab holds nothing that the preceding launch writes when that launch worked on another
-  // layer (p.early), so the first chunks' slab copies may start while it is still running; the caller's
-  // inputs and every write wait until it has completed.
-  if (!p.early) {
-    pdl_wait_predecessor();
-    pdl_allow_successor();
-  }
-  int n_pro = 0;
-#pragma unroll 1
-  for (; n_pro < kStages && feeding; ++n_pro) {
-    const int before = ahead;
-    issue(n_pro, p.early ? 1 : 3, ahead == 0);
-    if (ahead == before) break;
-  }
-  if (p.early) {
-    pdl_wait_predecessor();
-    pdl_allow_successor();
-    int rk = 0, rc0 = 0, rg = warp;
-#pragma unroll 1
-    for (int s = 0; s < n_pro; ++s) {
-      if (locate(rk, rc0, rg, false) <= 0) break;      // cannot happen: the producer has been here
-      if (lane == 0) copy_chunk(ent[rk % kTable], rg - rc0, s, 2);
-      rg += kWarps;
-    }
-  }
-
-  int stage = 0, fill = n_pro % kStages;   // stage to fold next, stage to fill next
-  uint32_t parity = 0;
-  float2 q[8];
-  State st;
-  LogitSink sink = {nullptr, 0, 0, 0, 0};
-
-#pragma unroll 1
-  while (ahead > 0 || feeding) {
-    if (ahead == 0) {                    // nothing in flight or in registers: wait for the feeder (or the end)
-      issue(fill, 3, true);
-      if (ahead == 0) break;
-      if (++fill == kStages) fill = 0;
-    }
-    const int nch = locate(ck, cc0, cg, false);   // published: the producer has been here
-    if (nch <= 0) {
-      give_up();
-      drain(stage, parity);
-      return;
-    }
-    if (lane == 0) at[warp] = ck;         // entries before this one are no longer needed by this warp
-    const int slot = ck % kTable;
-    const Unit& U = ent[slot];
-    const int j = cg - cc0, i0 = j * kChunk;
-    const int vh = U.vh;
-    const int n = vh - i0 < kChunk ? vh - i0 : kChunk;
-    if (!mbar_wait(bar0 + 8 * stage, parity)) {
-      give_up();
-      drain(stage, parity);
-      return;
-    }
-    const uint4* sb = reinterpret_cast<const uint4*>(ring + (size_t)stage * kStageBytes);
-    {
-      const uint4 qa = sb[kChunk * kSlotU4 + l8], qb = sb[kChunk * kSlotU4 + 8 + l8];
-      const float2 sc = make_float2(p.scale_log2, p.scale_log2);
-      q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
-      q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
-      q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
-      q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
-    }
-    if (j < kWarps) state_init(st);               // this warp's first chunk of the head
-    const int scored = U.scored, pv = U.pv, sv = U.sv, y = U.y;
-    sink.row = scored ? logit_rows + (size_t)slot * mrp : nullptr;
-    sink.skip = pv;
-    sink.ring_from = pv + sv;
-    sink.ring_shift = y - sv;
-    sink.i0 = i0;
-    Rows rows;
-    load_stage(sb, n, grp, l8, rows);
-    {
-      // the chunk that carries the newest token also stores it in the slab
-      const int s_new = U.fresh - i0;
-      if (s_new >= 0 && s_new < n) {
-        uint4* dstrow = reinterpret_cast<uint4*>(const_cast<unsigned char*>(U.hbase)) + (size_t)U.phys * kSlotU4;
-        dstrow[lane] = sb[s_new * kSlotU4 + lane];
-      }
-    }
-    __syncwarp();          // every lane has its rows in registers: the stage may be refilled
-    --ahead;
-    if (feeding) {
-      const int before = ahead;
-      issue(fill, 3, false);             // never wait with a chunk in registers: the feeder may need it folded
-      if (ahead != before && ++fill == kStages) fill = 0;
-    }
-    fold_stage(rows, n, grp, l8, q, st, sink);
-
-    if (j + kWarps >= nch) {
-      // this warp's last chunk of the head: merge the four groups, post the partial, and, if it was the
-      // head's last, merge the head's partials in the order of r and finish the head
-      State tot = st;
-      state_merge_lane(tot, 8);
-      state_merge_lane(tot, 16);
-      const int parts = nch < kWarps ? nch : kWarps;
-      float m = tot.m, l = tot.l;
-      bool finish = parts == 1;
-      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<unsigned char*>(p.out) + U.row);
-      if (parts == 1) {
-        if (grp == 0) write_out(orow, tot, l8);
-      } else {
-        float* P = partials + (size_t)(slot * kWarps + j % kWarps) * kPartialFloats;
-        if (lane == 0) {
-          P[0] = tot.m;
-          P[1] = tot.l;
-        }
-        if (grp == 0) {
-          float4* lo = reinterpret_cast<float4*>(P + 4 + 8 * l8);
-          float4* hi = reinterpret_cast<float4*>(P + 4 + 64 + 8 * l8);
-          lo[0] = make_float4(tot.acc[0].x, tot.acc[0].y, tot.acc[1].x, tot.acc[1].y);
-          lo[1] = make_float4(tot.acc[2].x, tot.acc[2].y, tot.acc[3].x, tot.acc[3].y);
-          hi[0] = make_float4(tot.acc[4].x, tot.acc[4].y, tot.acc[5].x, tot.acc[5].y);
-          hi[1] = make_float4(tot.acc[6].x, tot.acc[6].y, tot.acc[7].x, tot.acc[7].y);
-        }
-        __syncwarp();
-        int old = 0;
-        if (lane == 0) {
-          __threadfence_block();
-          old = atomicAdd(arrive + slot, 1);
-        }
-        old = __shfl_sync(FULL, old, 0);
-        if (old == parts - 1) {
-          __threadfence_block();
-          finish = true;
-          m = kNegBig;
-          l = 0.f;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int r = 0; r < parts; ++r) {
-            const float* Pr = partials + (size_t)(slot * kWarps + r) * kPartialFloats;
-            merge4(m, l, acc, Pr[0], Pr[1], reinterpret_cast<const float4*>(Pr + 4)[lane]);
-          }
-          write_out4(orow, l, acc, lane);
-        }
-      }
-      if (finish && scored) {
-        // Algorithm 2, post-processing (score accumulation): this warp knows the head's final (max, sum);
-        // the head's logits are in shared memory, written by the warps that folded them before they
-        // posted their partials.  No other warp touches the head's score row during the launch.
-        __syncwarp();
-        const float* lg = logit_rows + (size_t)slot * mrp;
-        float* acc = p.acc + (size_t)U.u * p.mr;
-        const float inv = 1.f / l;
-        if (kEvict) {
-          // Algorithm 1, one step: add the step's weights, then keep the M best of the static tokens and
-          // the token just appended (lowest score leaves; among equal scores the highest position, so the
-          // new token loses ties).  If it stays, its rows go into the static slot that is free or freed.
-          int32_t* idx = p.static_idx + (size_t)U.u * (p.M > 0 ? p.M : 1);
-          float worst = 3.0e38f;
-          int worst_pos = -1, worst_e = -1;
-          for (int i = lane; i < sv; i += 32) {
-            const float sc = acc[i] + ex2(lg[i] - m) * inv;
-            acc[i] = sc;
-            const int pos = idx[i];
-            if (sc < worst || (sc == worst && pos > worst_pos)) { worst = sc; worst_pos = pos; worst_e = i; }
-          }
-#pragma unroll
-          for (int off = 16; off >= 1; off >>= 1) {
-            const float w2 = __shfl_xor_sync(FULL, worst, off);
-            const int p2 = __shfl_xor_sync(FULL, worst_pos, off), e2 = __shfl_xor_sync(FULL, worst_e, off);
-            if (w2 < worst || (w2 == worst && p2 > worst_pos)) { worst = w2; worst_pos = p2; worst_e = e2; }
-          }
-          const float w_new = ex2(lg[U.phys - p.L] - m) * inv;     // the new token's score starts here
-          int dest = -1;                                           // static slot the new token takes
-          if (sv < p.M) dest = sv;
-          else if (sv > 0 && !(w_new <= worst)) dest = worst_e;
-          __syncwarp();                  // the scores written above, before the one written below
-          if (dest >= 0) {
-            if (lane == 0) {
-              acc[dest] = w_new;
-              idx[dest] = p.new_j;
-            }
-            uint4* hb = reinterpret_cast<uint4*>(const_cast<unsigned char*>(U.hbase)) + (size_t)(p.L + dest) * kSlotU4;
-            hb[lane] = *(reinterpret_cast<const uint4*>((lane < 16 ? p.k_new : p.v_new) + U.row) + (lane & 15));
-          }
-        } else {
-          const int n_scored = vh - pv, e_new = U.fresh >= 0 ? U.phys - p.L : -1;
-          for (int i = lane; i < n_scored; i += 32) {
-            const int e = i < sv ? i : y + (i - sv);
-            const float w = ex2(lg[e] - m) * inv;
-            acc[e] = e == e_new ? w : acc[e] + w;
-          }
-        }
-        __syncwarp();
-      }
-      // This warp is done with the head (and, if it finished it, so is everybody): step both sides past
-      // its entry, which may be reused from now on.
-      if (pk == ck) {
-        pc0 += nch;
-        ++pk;
-      }
-      cc0 += nch;
-      ++ck;
-      if (lane == 0) {
-        __threadfence_block();
-        at[warp] = ck;
-      }
-    }
-    cg += kWarps;
-    if (++stage == kStages) { stage = 0; parity ^= 1u; }
-  }
-  if (lane == 0) at[warp] = kAtEnd;
-}
-
 // acc += exp2(logit - max) / sum over the entries that held a token at the layer's last decode
 __global__ void __launch_bounds__(256) ssd_fold_pending_kernel(float* acc, const float* logits, const float2* ml,
                                                                const HeadDesc* desc, int n_pairs, int H, int mr,
@@ -1604,61 +1118,6 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
   else ssd_decode_layers_kernel<false><<<grid, kWarps * 32, smem, st>>>(p);
   count_launch();
   return cudaGetLastError();
-}
-
-// Heads per SM below which equal static shares (ssd_decode_kernel) balance better than whole heads.
-int decode_heads_min_pairs() {
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-    cudaGetLastError();
-    sms = 148;
-  }
-  return 8 * sms;
-}
-
-// Longest score row (M + R) whose logits the table of open heads can keep in shared memory.
-int decode_heads_max_mr(int) { return ((227 * 1024 - kHeadsSmemBytes) / (kTable * 4)) & ~3; }
-
-cudaError_t launch_decode_heads(const DecodeHeadsParams& p, cudaStream_t st) {
-  static std::atomic<int> ready[64] = {};
-  static int n_sm[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  const bool cached = dev >= 0 && dev < 64;
-  int sms = 0;
-  if (!cached || !ready[dev].load(std::memory_order_acquire)) {
-    const int most = kHeadsSmemBytes + kTable * decode_heads_max_mr(0) * 4;
-    e = cudaFuncSetAttribute(ssd_decode_heads_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ssd_decode_heads_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    if (cached) {
-      n_sm[dev] = sms;
-      ready[dev].store(1, std::memory_order_release);
-    }
-  } else {
-    sms = n_sm[dev];
-  }
-  const long pairs = (long)p.n_seqs * p.H;
-  if (pairs < 1 || pairs > 0x3fffffffL) return cudaErrorInvalidValue;
-  if (p.mr < 0 || p.mr > decode_heads_max_mr(p.evict)) return cudaErrorInvalidValue;
-  const int grid = (int)(pairs < sms ? pairs : sms);
-  const int smem = kHeadsSmemBytes + (p.acc != nullptr ? kTable * ((p.mr + 3) & ~3) * 4 : 0);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kHeadsThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  e = p.evict ? cudaLaunchKernelEx(&cfg, ssd_decode_heads_kernel<true>, p)
-              : cudaLaunchKernelEx(&cfg, ssd_decode_heads_kernel<false>, p);
-  count_launch();
-  return e;
 }
 
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st) {

@@ -41,11 +41,6 @@ struct DecodeParams {
   const unsigned char* v_new;
   int new_j;                // image index of that token; the view already counts it
   int early;                // 1: the launch before this one on the stream does not write this layer's slab
-  // Hand-over to the next launch: a worker that has issued its last copy asks the L2 cache to fetch the
-  // first pf_slots slots of the same share of the layer that will be attended to next (null: none), so
-  // that HBM stays busy while this launch drains and the next one starts.  A hint only.
-  const unsigned char* next_slab;
-  int pf_slots;
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
   LayerView view;           // layout and occupancy of the layer
@@ -84,34 +79,6 @@ struct DecodeLayersParams {
                             // takes the place of the lowest-scoring static token, or is dropped itself
   float scale_log2;
   LayerState layer[kMaxLayersPerLaunch];
-};
-
-// One layer, heads handed out to thread blocks (ssd_decode_heads_kernel): a thread block claims whole
-// heads from a counter and its warps share each head's chunks, so no head is ever cut between blocks.
-struct DecodeHeadsParams {
-  uint4* slab;              // first slot of the layer
-  const HeadDesc* desc;     // [H] layout records of the layer (device)
-  const unsigned char* q;   // [n_seqs, H, 128] bf16
-  const unsigned char* k_new;  // fused append: rows of the token being appended (null: it is in the slab)
-  const unsigned char* v_new;
-  __nv_bfloat16* out;       // [n_seqs, H, 128]
-  uint32_t* status;         // device status word (bit 0: a bounded wait ran out)
-  uint32_t* claim;          // two claim counters; this launch uses [parity] and clears the other
-  int parity;
-  int n_seqs, H, L, seq_slots;
-  int prompt_valid;         // 0 or L
-  int static_valid;         // valid static slots of semantic heads
-  int t_img;                // image tokens held (the one being appended included)
-  int t_sem;                // tokens in the rings of semantic heads (differs from t_img with a row buffer)
-  int new_j;                // image index of the token being appended, -1 if none
-  int sem_slot;             // row-buffer mode: buffer slot of that token in semantic heads
-  int early;                // 1: the launch before this one on the stream does not write this layer's slab
-  // row-buffer mode (Algorithm 2); acc == nullptr outside it
-  float* acc;               // [n_seqs * H, M + R] accumulated attention scores of the layer
-  int32_t* static_idx;      // [n_seqs, H, M] image indices of the static slots
-  int M, mr;
-  int evict;                // 1 (R == 1 only): the launch also re-selects (Algorithm 1 taken literally)
-  float scale_log2;
 };
 
 struct AppendParams {
@@ -174,9 +141,6 @@ struct ClassifyParams {
 
 cudaError_t launch_decode(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st);
-cudaError_t launch_decode_heads(const DecodeHeadsParams& p, cudaStream_t st);
-int decode_heads_min_pairs();   // fewest (sequence, head) pairs per layer for which that kernel is used
-int decode_heads_max_mr(int evict);
 // acc += the normalised weights of the layer's last decode (its logits and (max, exp-sum) are in
 // `logits` and `ml`): what the next append of the row-buffer mode would do first
 cudaError_t launch_fold_pending(float* acc, const float* logits, const float2* ml, const HeadDesc* desc, int n_seqs,

@@ -79,8 +79,7 @@ class RunResult:
 
 
 def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, full_every_step=False,
-                 n_obs=None, check_planted=False, device="cuda:0", labels_override=None, step_form="two",
-                 decode_form=0) -> RunResult:
+                 n_obs=None, check_planted=False, device="cuda:0", labels_override=None, step_form="two") -> RunResult:
     """Drive the C-ABI path for `layers` x `seqs` of a workload and check every stage.
 
     The cache is created with len(layers) layers and len(seqs) sequences; layer i of the cache holds
@@ -92,7 +91,6 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
     n_obs = n0 if n_obs is None else n_obs
     ccfg = B.config_from_workload(cfg, n_layers=len(layers), n_seqs=S)
     cache = B.SsdCache(ccfg, device=device)
-    cache.set_decode_form(decode_form)     # 0: chosen by size, 1: equal shares, 2: heads handed out to blocks
     res = RunResult()
 
     gen_masks = np.stack([wl.sink_mask(cfg, l) for l in layers])
@@ -172,7 +170,7 @@ def run_workload(cfg: wl.Workload, layers, seqs, check_steps, classify=True, ful
     return res
 
 
-def run_sampled(cfg: wl.Workload, layer: int, sample, steps, device="cuda:0", decode_form=0):
+def run_sampled(cfg: wl.Workload, layer: int, sample, steps, device="cuda:0"):
     """Full launch size on the GPU (all cfg.n_seqs sequences of one layer, the launch configuration the
     benchmark times); the oracle recomputes only the sampled (sequence, head) pairs one by one: their
     selected index sets (exact outside the tie band) and their outputs at the given image steps."""
@@ -181,7 +179,6 @@ def run_sampled(cfg: wl.Workload, layer: int, sample, steps, device="cuda:0", de
                                cfg.n_heads, cfg.n_seqs)
     labels = wl.sink_mask(cfg, layer)
     cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1), device=device)
-    cache.set_decode_form(decode_form)
     cache.set_head_labels(labels)
     q, k, v, _ = wl.gen_layer(cfg, layer, list(range(S)), device=dev)
     cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)

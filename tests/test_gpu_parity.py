@@ -12,11 +12,9 @@ from parity_util import check_outputs, run_workload
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("decode_form,step_form", [(1, "two"), (2, "two"), (2, "fused")])
-def test_tiny_every_step(decode_form, step_form):
+def test_tiny_every_step():
     cfg = wl.CONFIGS["tiny"]
-    r = run_workload(cfg, [0], [0], check_steps=(), full_every_step=True, check_planted=True,
-                     decode_form=decode_form, step_form=step_form)
+    r = run_workload(cfg, [0], [0], check_steps=(), full_every_step=True, check_planted=True)
     assert r.steps_checked == cfg.n_img - cfg.n0 and r.n_pairs == 8
 
 
@@ -26,31 +24,24 @@ def test_tiny_fewer_observation_queries():
         run_workload(cfg, [0], [0], check_steps=(cfg.n0 + 1, cfg.n_img), classify=False, n_obs=n_obs)
 
 
-@pytest.mark.parametrize("decode_form,step_form", [(0, "two"), (2, "fused")])
-def test_janus1b_sampled_layers_all_sequences(decode_form, step_form):
+def test_janus1b_sampled_layers_all_sequences():
     cfg = wl.CONFIGS["janus1b"]
     steps = (cfg.n0 + 1, cfg.n0 + 2, cfg.n0 + 25, cfg.n_img)
-    r = run_workload(cfg, [0, 23], list(range(cfg.n_seqs)), steps, check_planted=True, decode_form=decode_form,
-                     step_form=step_form)
+    r = run_workload(cfg, [0, 23], list(range(cfg.n_seqs)), steps, check_planted=True)
     assert r.steps_checked == 2 * len(steps)
 
 
-@pytest.mark.parametrize("decode_form,step_form", [(0, "two"), (0, "fused"), (1, "fused")])
-def test_janus7b_sampled_layers_all_sequences(decode_form, step_form):
-    # at this size (64 sequences x 32 heads) form 0 is the heads-to-blocks kernel
+def test_janus7b_sampled_layers_all_sequences():
     cfg = wl.CONFIGS["janus7b"]
     steps = (cfg.n0 + 1, cfg.n0 + 24, cfg.n_img)
-    r = run_workload(cfg, [0, 29] if decode_form == 0 else [29], list(range(cfg.n_seqs)), steps, check_planted=True,
-                     decode_form=decode_form, step_form=step_form)
-    assert r.steps_checked == (2 if decode_form == 0 else 1) * len(steps)
+    r = run_workload(cfg, [0, 29], list(range(cfg.n_seqs)), steps, check_planted=True)
+    assert r.steps_checked == 2 * len(steps)
 
 
-@pytest.mark.parametrize("decode_form", [0, 2])
-def test_hires7b_one_layer_two_sequences(decode_form):
+def test_hires7b_one_layer_two_sequences():
     cfg = wl.CONFIGS["hires7b"]
     steps = (cfg.n0 + 1, cfg.n0 + 65, cfg.n_img)
-    run_workload(cfg, [0], [0, 1], steps, classify=False, decode_form=decode_form,
-                 step_form="fused" if decode_form else "two")
+    run_workload(cfg, [0], [0, 1], steps, classify=False)
 
 
 def test_sweep_points():
@@ -59,13 +50,12 @@ def test_sweep_points():
         run_workload(cfg, [3], seqs, (cfg.n0 + 1, cfg.n0 + 30, cfg.n_img), classify=False)
 
 
-def _full_cache_case(cfg: wl.Workload, seqs, steps, one_launch=False, decode_form=0):
+def _full_cache_case(cfg: wl.Workload, seqs, steps, one_launch=False):
     """Uncompressed baseline: every head spatial with W = N, prompt loaded with n0 = 0."""
     dev = torch.device("cuda:0")
     L, N, H, S = cfg.prompt_len, cfg.n_img, cfg.n_heads, len(seqs)
     c = B.make_config(1, S, H, L, N, N, 0, 1, cfg.cls_window, cfg.tau)
     cache = B.SsdCache(c)
-    cache.set_decode_form(decode_form)
     cache.set_head_labels(np.zeros(H, np.uint8))
     q, k, v, _ = wl.gen_layer(cfg, 0, seqs, device=dev)
     qu, ku, vu = wl.to_u16(q), wl.to_u16(k), wl.to_u16(v)
@@ -90,8 +80,6 @@ def _full_cache_case(cfg: wl.Workload, seqs, steps, one_launch=False, decode_for
 def test_full_cache_baseline_matches_full_attention():
     _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65))
     _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576))
-    _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65), decode_form=2)
-    _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576), decode_form=2)
     _full_cache_case(wl.CONFIGS["tiny"], [0], steps=range(1, 65), one_launch=True)
     _full_cache_case(wl.CONFIGS["janus7b"], [0, 1, 2], steps=(1, 2, 7, 8, 9, 100, 333, 575, 576), one_launch=True)
 
@@ -115,8 +103,7 @@ def test_random_small_shapes(seed):
         pytest.skip("nothing to load")
     run_workload(cfg, [0], list(range(cfg.n_seqs)), (), classify=False, full_every_step=True,
                  n_obs=min(cfg.n0, seed % 5 + (cfg.n0 if seed % 2 else 0)),
-                 step_form=("two", "fused", "layers")[seed % 3],      # every form of the step sees odd shapes
-                 decode_form=(1, 2)[(seed // 3) % 2])                 # and so does either per-layer kernel
+                 step_form=("two", "fused", "layers")[seed % 3])      # every form of the step sees odd shapes
 
 
 def test_decode_before_any_compress_fills_ring_from_zero():
@@ -304,12 +291,10 @@ def test_other_head_partitions(kind):
         assert r.steps_checked == 3 * len(layers)
 
 
-@pytest.mark.parametrize("decode_form", [1, 2])
 @pytest.mark.parametrize("case", ["tiny_compressed", "tiny_ring_from_zero", "janus7b_slice"])
-def test_fused_append_decode_matches_the_two_calls(case, decode_form):
+def test_fused_append_decode_matches_the_two_calls(case):
     """ssd_append_decode must give the bits of ssd_append + ssd_decode_attn at every step, and leave
-    the same cache behind (later steps read the token that the fused kernel stored); with either
-    per-layer kernel (both merge a head's pieces in an order that does not depend on scheduling)."""
+    the same cache behind (later steps read the token that the fused kernel stored)."""
     dev = torch.device("cuda:0")
     if case == "janus7b_slice":
         cfg, seqs, n_steps = wl.CONFIGS["janus7b"], [0, 1, 2, 3, 4], 30
@@ -320,7 +305,6 @@ def test_fused_append_decode_matches_the_two_calls(case, decode_form):
     caches = []
     for _ in range(2):
         c = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=len(seqs)), device=dev)
-        c.set_decode_form(decode_form)
         c.set_head_labels(wl.sink_mask(cfg, 0))
         if case == "tiny_ring_from_zero":
             t0 = 0                       # no compress: prompt slots unused, rings fill from empty

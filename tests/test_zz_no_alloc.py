@@ -38,10 +38,7 @@ def test_static_scratch_matches_regular_entry_point_on_consecutive_calls(name, s
     for t in (n0 + 1, n0 + 2, n0 + 3):                 # calls in a row reuse the same array
         cache.append(0, k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous())
         qt = q[:, :, t - 1].contiguous()
-        cache.set_decode_form(1)                       # the kernel the static entry point runs: equal shares
         want = cache.decode_attn(0, qt)
-        cache.set_decode_form(2)                       # the other per-layer kernel: same values up to rounding order
-        other = cache.decode_attn(0, qt)
         out_static.fill_(float("nan"))
         torch.cuda.synchronize()
         free_before = torch.cuda.mem_get_info(dev)[0]
@@ -52,8 +49,6 @@ def test_static_scratch_matches_regular_entry_point_on_consecutive_calls(name, s
         err = (got.float() - want.float()).abs()
         assert err.max().item() <= MAX_ABS and err.mean().item() <= MEAN_ABS
         assert torch.equal(got, want), "same kernel, same merge order: expected identical bits"
-        err = (got.float() - other.float()).abs()
-        assert err.max().item() <= MAX_ABS and err.mean().item() <= MEAN_ABS
     assert cache.device_status() == 0
     cache.close()
 
