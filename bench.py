@@ -5,11 +5,13 @@
 
 Prints ONE JSON line.  A "step" is one decoded image token for every sequence: for each layer,
 append the new K/V and attend.  `value` is decoded image tokens per second (one per CFG pair per
-step) over the whole job with inputs resident in HBM and the step issued as one launch
-(ssd_append_decode_layers); `per_layer` is the same step as one launch per layer; `e2e` is the same
-through ssd_step_host_layers with pinned HOST buffers (copies inside the timed region).  Under torchrun
-each rank owns its own block of sequences (weak scaling, no data-path collective); time is the max
-over ranks.  `--impl reference` times the fp64 CPU oracle as it stands on a bounded sample.
+step) over the whole job with inputs resident in HBM and the step issued the way a model issues it:
+one ssd_append_decode call (one kernel launch) per layer.  `one_launch` is the same step as a single
+launch over all layers (ssd_append_decode_layers: an upper bound that needs every layer's inputs up
+front); `e2e` is the step through ssd_step_host_layers with pinned HOST buffers (copies inside the
+timed region).  Under torchrun each rank owns its own block of sequences (weak scaling, no data-path
+collective); time is the max over ranks.  `--impl reference` times the fp64 CPU oracle as it stands on
+a bounded sample.
 """
 from __future__ import annotations
 
@@ -269,6 +271,8 @@ class Stepper:
         self.addr = lambda j, i, layer: base[j] + (i * cfg.n_layers + layer) * per
         self.call = cache.lib.ssd_append_decode
         self.h = cache._h
+        self.args = [[(layer, self.addr(1, i, layer), self.addr(2, i, layer), self.addr(0, i, layer))
+                      for layer in range(cfg.n_layers)] for i in range(self.T)]
 
     def step(self, fused=True, one_launch=False):
         """One decoded token per sequence: for every layer append the new K/V and attend
@@ -287,10 +291,9 @@ class Stepper:
             self.i += 1
             return
         if fused:
-            stream, outp = torch.cuda.current_stream().cuda_stream, self.out.data_ptr()
-            for layer in range(self.cfg.n_layers):
-                rc = self.call(self.h, layer, self.addr(1, i, layer), self.addr(2, i, layer), self.addr(0, i, layer),
-                               outp, stream)
+            stream, outp, call, h = torch.cuda.current_stream().cuda_stream, self.out.data_ptr(), self.call, self.h
+            for layer, ka, va, qa in self.args[i]:
+                rc = call(h, layer, ka, va, qa, outp, stream)
                 if rc != 0:
                     raise RuntimeError(f"ssd_append_decode: status {rc}")
             self.i += 1
@@ -344,29 +347,32 @@ def run_ours(args, cfg):
     out = torch.empty((S, H, 128), dtype=torch.bfloat16, device=device)
     stepper = Stepper(cfg, cache, steps_in, out)
 
-    # ---- device-resident timing (the headline `value`): the whole step as one launch
-    # (ssd_append_decode_layers: every layer's append + attention, heads handed out from a counter)
-    one_step = lambda: stepper.step(one_launch=True)
+    # ---- device-resident timing (the headline `value`): the step as a model issues it, one
+    # ssd_append_decode call (one launch of ssd_decode_kernel) per layer; consecutive launches overlap by
+    # programmatic dependent launch
     for _ in range(W):
-        one_step()
+        stepper.step()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
     l0 = B.kernel_launch_count()
-    ms = timed(one_step, K, barrier)
+    ms = timed(stepper.step, K, barrier)
     launches = B.kernel_launch_count() - l0
     ms = max_over_ranks(ms)
     ms_per_step = ms / K
     value = cfg.images_per_step * world / (ms_per_step * 1e-3)
     # stability: five more passes of the same region, shorter
     Ks = min(K, 50)
-    repeats = [max_over_ranks(timed(one_step, Ks, barrier)) / Ks for _ in range(5)]
-
-    # ---- the same step as one launch per layer (ssd_append_decode; what a model calls, since layer
-    # l+1's inputs depend on layer l's output); consecutive launches overlap by programmatic dependent launch
-    for _ in range(3):
+    repeats = [max_over_ranks(timed(stepper.step, Ks, barrier)) / Ks for _ in range(5)]
+    # what the host needs to issue a launch (Python call + library + driver), measured on a queue that is
+    # never full: if this approaches the launch duration, the number above is the host's, not the GPU's
+    torch.cuda.synchronize()
+    Kh = max(1, min(K, 600 // cfg.n_layers))
+    t_h0 = time.perf_counter()
+    for _ in range(Kh):
         stepper.step()
-    ms_layers = max_over_ranks(timed(stepper.step, K, barrier)) / K
+    host_us = (time.perf_counter() - t_h0) / (Kh * cfg.n_layers) * 1e6
+    torch.cuda.synchronize()
     # the same steps again with a CUDA event on either side of every decode launch (the events stand
     # between the kernels, so these launches do not overlap with their neighbours)
     Kr = min(K, 50)
@@ -374,12 +380,19 @@ def run_ours(args, cfg):
     ms_r = timed(stepper.step, Kr, barrier)
     dec_ms = cache.profile_collect()
     cache.profile_enable(0)
-    clocks = sampler.stop()
-    # and as two launches per layer (ssd_append, ssd_decode_attn), for comparison
+    # as two launches per layer (ssd_append, ssd_decode_attn), for comparison
     Kt = min(K, 50)
     two_step = lambda: stepper.step(fused=False)
     two_step()
     ms_two = max_over_ranks(timed(two_step, Kt, barrier)) / Kt
+
+    # ---- the whole step as ONE launch (ssd_append_decode_layers: every layer's append + attention, heads
+    # handed out from a counter): an upper bound, since it needs all layers' inputs before the first layer runs
+    one_step = lambda: stepper.step(one_launch=True)
+    for _ in range(3):
+        one_step()
+    ms_one = max_over_ranks(timed(one_step, K, barrier)) / K
+    clocks = sampler.stop()
 
     # ---- roofline of the dominant kernel: algorithmic bytes per launch / launch duration (CUDA events)
     slots_layer = int(sum(int(cache.get_lengths(l).sum()) for l in range(cfg.n_layers))) / cfg.n_layers
@@ -388,34 +401,35 @@ def run_ours(args, cfg):
     bytes_step = bytes_launch * cfg.n_layers
     peak, peak_kind = measured_peaks()
     n_calls = (cfg.n_layers + 63) // 64
-    # The timed region holds nothing but launches of ssd_decode_layers_kernel (one per step for up to
-    # 64 layers, each preceded by a 4-byte memset of its unit counter), so its launch duration is the
-    # region time per launch.
-    achieved = bytes_step / (ms_per_step * 1e-3) / 1e9
     traffic = decode_traffic(cfg)
     dec_mean_ms = float(np.mean(dec_ms)) if len(dec_ms) else float("nan")
-    # Per-layer form: its region also holds only one kernel (n_layers launches per step); launches
-    # overlap by design, so timed one at a time (an event between launches forbids the overlap) a
-    # launch takes longer ("isolated").
-    launch_ms = ms_layers / cfg.n_layers
-    ach_l = bytes_launch / (launch_ms * 1e-3) / 1e9
+    # The timed region holds nothing but launches of ssd_decode_kernel (n_layers per step), so its launch
+    # duration is the region time per launch; launches overlap by design, so timed one at a time (an event
+    # between launches forbids the overlap) a launch takes longer ("isolated").
+    launch_ms = ms_per_step / cfg.n_layers
+    achieved = bytes_launch / (launch_ms * 1e-3) / 1e9
     iso = bytes_launch / (dec_mean_ms * 1e-3) / 1e9
-    per_layer = {"value": cfg.images_per_step * world / (ms_layers * 1e-3), "unit": UNIT, "ms_per_step": ms_layers,
-                 "launches_per_step": cfg.n_layers, "ms_per_step_two_launches_per_layer": ms_two,
-                 "roofline": {"bound": "hbm", "kernel": "ssd_decode_kernel (fused append)", "achieved": ach_l, "peak": peak,
-                              "unit": "GB/s", "frac": ach_l / peak, "peak_kind": f"of {peak_kind}",
-                              "traffic": traffic["per_layer"] if traffic else None,
-                              "bytes_per_launch": bytes_launch, "launch_ms_mean": launch_ms,
-                              "isolated": {"launch_ms_mean": dec_mean_ms, "achieved": iso, "frac": iso / peak,
-                                           "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
-                                           "launches_timed": int(len(dec_ms)),
-                                           "ms_per_step_while_timing_launches": ms_r / Kr},
-                              "frac_of_8TBs_nominal": ach_l / 8000.0}}
-    roofline = {"bound": "hbm", "kernel": "ssd_decode_layers_kernel (whole step, fused append)", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "ssd_decode_kernel (one launch per layer, fused append)", "achieved": achieved,
                 "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "traffic": traffic["per_layer_of_step"] * cfg.n_layers / n_calls if traffic else None,
-                "bytes_per_launch": bytes_step / n_calls, "launch_ms_mean": ms_per_step / n_calls,
-                "launches_in_region": K * n_calls, "frac_of_8TBs_nominal": achieved / 8000.0}
+                "traffic": traffic["per_layer"] if traffic else None,
+                "bytes_per_launch": bytes_launch, "launch_ms_mean": launch_ms, "launches_in_region": K * cfg.n_layers,
+                "isolated": {"launch_ms_mean": dec_mean_ms, "achieved": iso, "frac": iso / peak,
+                             "launch_ms_median": float(np.median(dec_ms)) if len(dec_ms) else None,
+                             "launches_timed": int(len(dec_ms)),
+                             "ms_per_step_while_timing_launches": ms_r / Kr},
+                "frac_of_8TBs_nominal": achieved / 8000.0}
+    ach_one = bytes_step / (ms_one * 1e-3) / 1e9
+    one_launch = {"value": cfg.images_per_step * world / (ms_one * 1e-3), "unit": UNIT, "ms_per_step": ms_one,
+                  "launches_per_step": n_calls,
+                  "roofline": {"bound": "hbm", "kernel": "ssd_decode_layers_kernel (whole step, fused append)",
+                               "achieved": ach_one, "peak": peak, "unit": "GB/s", "frac": ach_one / peak,
+                               "peak_kind": f"of {peak_kind}",
+                               "traffic": traffic["per_layer_of_step"] * cfg.n_layers / n_calls if traffic else None,
+                               "bytes_per_launch": bytes_step / n_calls, "launch_ms_mean": ms_one / n_calls,
+                               "frac_of_8TBs_nominal": ach_one / 8000.0}}
+    host = {"enqueue_us_per_launch": host_us, "launches_per_step": cfg.n_layers, "steps": Kh,
+            "share_of_launch_time": host_us / (launch_ms * 1e3),
+            "ms_per_step_two_launches_per_layer": ms_two}
 
     # ---- end to end: the same step through ssd_step_host_layers with pinned host buffers: one call
     # per step takes every layer's q, k_new, v_new from the host and returns every layer's output
@@ -442,7 +456,9 @@ def run_ours(args, cfg):
     e2e_val = cfg.images_per_step * world / (ms_e / Ke * 1e-3)
     tensor_bytes = S * H * 128 * 2
     e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 3 * tensor_bytes * cfg.n_layers,
-           "d2h_bytes_per_step": tensor_bytes * cfg.n_layers, "steps": Ke, "ms_per_step": ms_e / Ke}
+           "d2h_bytes_per_step": tensor_bytes * cfg.n_layers, "steps": Ke, "ms_per_step": ms_e / Ke,
+           "h2d_gbs": 3 * tensor_bytes * cfg.n_layers / (ms_e / Ke * 1e-3) / 1e9,
+           "d2h_gbs": tensor_bytes * cfg.n_layers / (ms_e / Ke * 1e-3) / 1e9}
 
     kv_bytes_per_seq = cache.kv_bytes_per_seq()
     setup_times = cache.setup_times
@@ -464,9 +480,9 @@ def run_ours(args, cfg):
         ms_f = max_over_ranks(timed(f_one, Kf, barrier))                           # one launch per step
         t_mid = n0 + 3 + Kf + 1 + (Kf + 1) / 2
         fbytes = cfg.n_layers * S * H * ((cfg.prompt_len + t_mid) * 512 + 512)
-        full = {"value": cfg.images_per_step * world / (ms_f / Kf * 1e-3), "unit": UNIT, "ms_per_step": ms_f / Kf,
-                "steps": Kf, "image_step": t_mid, "gbs": fbytes / (ms_f / Kf * 1e-3) / 1e9,
-                "ms_per_step_per_layer_launches": ms_fl / Kf,
+        full = {"value": cfg.images_per_step * world / (ms_fl / Kf * 1e-3), "unit": UNIT, "ms_per_step": ms_fl / Kf,
+                "steps": Kf, "image_step": t_mid - Kf - 1, "gbs": (fbytes - cfg.n_layers * S * H * (Kf + 1) * 512) / (ms_fl / Kf * 1e-3) / 1e9,
+                "ms_per_step_one_launch": ms_f / Kf, "gbs_one_launch": fbytes / (ms_f / Kf * 1e-3) / 1e9,
                 "kv_bytes_per_seq": fcache.kv_bytes_per_seq()}
         fcache.close()
         del fcache, fsteps, fst
@@ -478,67 +494,58 @@ def run_ours(args, cfg):
         R = cfg.sink_recent
         Kb = max(R, min(2 * R, (N - n0) // 2 - R) // R * R)   # both forms, each with a warm-up cycle, fit in the image
         rcache, rsteps = build_cache(cfg, device, rank * S, rank, world, t_steps=2 * (Kb + R), row_buffer=True)
-        rstate = {"i": 0}
+        rst = Stepper(cfg, rcache, rsteps, out)          # per-layer calls with precomputed addresses
         rout = torch.empty((cfg.n_layers, S, H, 128), dtype=torch.bfloat16, device=device)
 
+        def reselect(c):
+            for l0 in range(0, cfg.n_layers, 64):
+                c.recompress_layers(l0, min(64, cfg.n_layers - l0))
+
         def rb_step(one_launch):
-            i = rstate["i"]
-            if one_launch:
-                qq, kk, vv = rcache.step_all
-                for l0 in range(0, cfg.n_layers, 64):
-                    l1 = min(l0 + 64, cfg.n_layers)
-                    rcache.append_decode_layers(l0, kk[i, l0:l1], vv[i, l0:l1], qq[i, l0:l1], rout[l0:l1])
-            else:
-                for layer in range(cfg.n_layers):
-                    qq, kk, vv = rsteps[layer]
-                    rcache.append_decode(layer, kk[i], vv[i], qq[i], out)
-            rstate["i"] += 1
-            if rstate["i"] % R == 0:
-                if one_launch:
-                    for l0 in range(0, cfg.n_layers, 64):
-                        rcache.recompress_layers(l0, min(64, cfg.n_layers - l0))
-                else:
-                    for layer in range(cfg.n_layers):
-                        rcache.recompress(layer)
+            # ssd_append_decode per layer (one launch each: the kernel also keeps the scores up to date), or the
+            # whole step in one launch; every R steps ssd_recompress_layers re-selects all layers in one launch
+            rst.step(one_launch=one_launch)
+            if rst.i % R == 0:
+                reselect(rcache)
 
         ms_rb = {}
-        for form in (False, True):    # per-layer launches (append, decode), then the one-launch step
+        for form in (False, True):    # per-layer launches, then the one-launch step
             for _ in range(R):        # one whole cycle as warm-up, so the timed region starts on an empty buffer
                 rb_step(form)
             ms_rb[form] = max_over_ranks(timed(lambda: rb_step(form), Kb, barrier))
-        ms_b = ms_rb[True]
+        ms_b = ms_rb[False]
         rowbuf = {"value": cfg.images_per_step * world / (ms_b / Kb * 1e-3), "unit": UNIT, "ms_per_step": ms_b / Kb,
-                  "steps": Kb, "reselect_every": R, "ms_per_step_per_layer_launches": ms_rb[False] / Kb,
+                  "steps": Kb, "reselect_every": R, "ms_per_step_one_launch": ms_rb[True] / Kb,
                   "device_status": rcache.device_status()}
         rcache.close()
-        del rcache, rsteps
+        del rcache, rsteps, rst
         torch.cuda.empty_cache()
         # Algorithm 1 taken literally: a re-selection after every step = a row buffer of one token with the
         # same number of slots per head (M + R - 1 static, 1 buffered)
         import dataclasses
         ecfg = dataclasses.replace(cfg, sink_budget=cfg.sink_budget + R - 1, sink_recent=1, name=cfg.name + "_evict_every_step")
         Kv = min(K, 48)
-        ecache, _ = build_cache(ecfg, device, rank * S, rank, world, t_steps=Kv + 3, row_buffer=True, classify=False)
-        estate = {"i": 0}
-        eout = torch.empty((cfg.n_layers, S, H, 128), dtype=torch.bfloat16, device=device)
+        ecache, esteps = build_cache(ecfg, device, rank * S, rank, world, t_steps=2 * Kv + 8, row_buffer=True, classify=False)
+        est = Stepper(ecfg, ecache, esteps, out)
 
-        def ev_step():
-            i = estate["i"]
-            qq, kk, vv = ecache.step_all
-            for l0 in range(0, cfg.n_layers, 64):
-                l1 = min(l0 + 64, cfg.n_layers)
-                # with a buffer of one token the launch re-selects as well: one launch per step
-                ecache.append_decode_layers(l0, kk[i, l0:l1], vv[i, l0:l1], qq[i, l0:l1], eout[l0:l1])
-            estate["i"] += 1
+        def ev_step(one_launch):
+            # one launch per layer, then one re-selection launch for all layers; or everything in one launch
+            # (with a buffer of one token the one-launch step re-selects as well)
+            est.step(one_launch=one_launch)
+            if not one_launch:
+                reselect(ecache)
 
-        for _ in range(3):
-            ev_step()
-        ms_ev = max_over_ranks(timed(ev_step, Kv, barrier))
-        rowbuf["evict_every_step"] = {"value": cfg.images_per_step * world / (ms_ev / Kv * 1e-3), "unit": UNIT,
-                                      "ms_per_step": ms_ev / Kv, "steps": Kv, "sink_budget": ecfg.sink_budget,
+        ms_ev = {}
+        for form in (False, True):
+            for _ in range(3):
+                ev_step(form)
+            ms_ev[form] = max_over_ranks(timed(lambda: ev_step(form), Kv, barrier))
+        rowbuf["evict_every_step"] = {"value": cfg.images_per_step * world / (ms_ev[False] / Kv * 1e-3), "unit": UNIT,
+                                      "ms_per_step": ms_ev[False] / Kv, "ms_per_step_one_launch": ms_ev[True] / Kv,
+                                      "steps": Kv, "sink_budget": ecfg.sink_budget,
                                       "sink_recent": 1, "device_status": ecache.device_status()}
         ecache.close()
-        del ecache
+        del ecache, esteps, est
         torch.cuda.empty_cache()
 
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)
@@ -569,9 +576,10 @@ def run_ours(args, cfg):
                        "l2": "inputs larger than L2 (each layer's slab is >126 MB and is touched once per step)",
                        "kv_bytes_per_seq": kv_bytes_per_seq},
             "sequence_tokens_per_s": value * 2 if S > 1 else value,
-            "step_form": "one launch per step (ssd_append_decode_layers); per_layer = one launch per layer",
+            "step_form": "one launch per layer (ssd_append_decode); one_launch = the whole step in one launch",
             "ms_per_step_repeats": repeats,
-            "per_layer": per_layer,
+            "host": host,
+            "one_launch": one_launch,
             "one_time": setup_times,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf,

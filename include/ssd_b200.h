@@ -146,8 +146,10 @@ int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, v
 /* ssd_append followed by ssd_decode_attn for the same layer, in one kernel launch (Algorithm 1's
  * Append and the attention that consumes its output).  Same arguments, results and errors as the two
  * calls; the newest token's rows are read from k_new / v_new by the attention and stored into the
- * ring by the same kernel.  k_new, v_new, q, out 16-byte aligned.  In row-buffer mode the call issues
- * the two launches.  Asynchronous. */
+ * ring by the same kernel.  k_new, v_new, q, out 16-byte aligned.  In row-buffer mode (below) it is still
+ * one launch: the kernel keeps the step's logits in one of two alternating buffers and, at its start, adds
+ * the weights of the layer's previous step to the scores (which nothing reads in between but
+ * ssd_recompress and ssd_cache_get_scores, and those add what is pending themselves).  Asynchronous. */
 int ssd_append_decode(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new,
                       const void *q, void *out, void *stream);
 

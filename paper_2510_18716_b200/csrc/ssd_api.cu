@@ -60,8 +60,10 @@ static Regions plan_regions(const ssd_config& c) {
   // ring slots, and the last decode's (max, exp-sum), per layer
   const size_t mr = (size_t)c.sink_budget + c.sink_recent;
   r.acc = off;       off = align_up(off + (size_t)c.n_layers * pairs_layer * mr * 4);
-  r.logits = off;    off = align_up(off + (size_t)c.n_layers * pairs_layer * mr * 4);
-  r.ml = off;        off = align_up(off + (size_t)c.n_layers * pairs_layer * 8);
+  // two buffers per layer each: a launch that records a step's logits may, at its start, still be adding
+  // those of the step before to the scores
+  r.logits = off;    off = align_up(off + (size_t)c.n_layers * 2 * pairs_layer * mr * 4);
+  r.ml = off;        off = align_up(off + (size_t)c.n_layers * 2 * pairs_layer * 8);
   r.front_bytes = off;
   r.slab = off;
   return r;
@@ -88,9 +90,12 @@ struct ssd_cache {
   // re-selection), -1 if none, -2 if unknown: a decode launch of ANOTHER layer may prefetch its slab
   // before that launch has completed.
   int last_writer = -2;
+  // The same for the layer's score tables of the row-buffer mode (accumulated scores, logits, (max, sum)).
+  int last_scored = -2;
   bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
   std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
   std::vector<uint8_t> pending;       // [layers] last decode's logits not yet added to the scores
+  std::vector<uint8_t> lg_cur;        // [layers] which of the layer's two logit buffers the last decode wrote
   // ssd_step_host_layers: copy streams and per-slot events, created at its first call
   cudaStream_t h_in = nullptr, h_out = nullptr;
   cudaEvent_t h_fork = nullptr, h_loaded[kHostSlots] = {}, h_done[kHostSlots] = {}, h_stored[kHostSlots] = {};
@@ -110,8 +115,12 @@ struct ssd_cache {
   int mr() const { return cfg.sink_budget + cfg.sink_recent; }
   size_t layer_scores(int layer) const { return (size_t)layer * cfg.n_seqs * cfg.n_heads * mr(); }
   float* d_acc(int layer) const { return reinterpret_cast<float*>(base + reg.acc) + layer_scores(layer); }
-  float* d_logits(int layer) const { return reinterpret_cast<float*>(base + reg.logits) + layer_scores(layer); }
-  float2* d_ml(int layer) const { return reinterpret_cast<float2*>(base + reg.ml) + (size_t)layer * cfg.n_seqs * cfg.n_heads; }
+  float* d_logits(int layer, int which) const {
+    return reinterpret_cast<float*>(base + reg.logits) + ((size_t)layer * 2 + which) * cfg.n_seqs * cfg.n_heads * mr();
+  }
+  float2* d_ml(int layer, int which) const {
+    return reinterpret_cast<float2*>(base + reg.ml) + ((size_t)layer * 2 + which) * cfg.n_seqs * cfg.n_heads;
+  }
   // tokens in the rings of semantic heads
   int sem_tokens(int layer) const { return row_buffer ? t_img[layer] - t_base[layer] : t_img[layer]; }
   float* d_partial() const { return reinterpret_cast<float*>(base + reg.partial); }
@@ -200,6 +209,7 @@ int ssd_cache_create(const ssd_config* cfg, void* dev_mem, size_t dev_bytes, ssd
   c->static_valid.assign(cfg->n_layers, 0);
   c->t_base.assign(cfg->n_layers, 0);
   c->pending.assign(cfg->n_layers, 0);
+  c->lg_cur.assign(cfg->n_layers, 0);
   if (cudaMemset(c->base, 0, r.front_bytes) != cudaSuccess ||
       cudaMemset(c->base + r.idx, 0xFF, r.counters - r.idx) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess) {
@@ -458,6 +468,7 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   c->t_base[layer] = n0;
   c->pending[layer] = 0;
   c->last_writer = -2;
+  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -483,10 +494,11 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   p.pending = c->pending[layer];
   p.mr = c->mr();
   p.acc = c->row_buffer ? c->d_acc(layer) : nullptr;
-  p.logits = c->d_logits(layer);
-  p.ml = c->d_ml(layer);
+  p.logits = c->d_logits(layer, c->lg_cur[layer]);
+  p.ml = c->d_ml(layer, c->lg_cur[layer]);
   if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = layer;
+  c->last_scored = c->row_buffer ? layer : -1;
   if (c->row_buffer) c->pending[layer] = 0;
   c->t_img[layer] += 1;
   return SSD_OK;
@@ -506,10 +518,13 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.partial = c->d_partial();
   p.counters = c->d_counters();
   p.status = c->d_status();
-  p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
-  p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
+  const int lg_next = c->lg_cur[layer] ^ 1;
+  p.logits = c->row_buffer ? c->d_logits(layer, lg_next) : nullptr;
+  p.ml = c->row_buffer ? c->d_ml(layer, lg_next) : nullptr;
   p.mr = c->mr();
-  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
+  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1; p.sem_slot = -1;
+  p.fold_acc = nullptr; p.fold_logits = nullptr; p.fold_ml = nullptr;
+  p.fold_pending = 0; p.fold_early = 0; p.fold_static = 0; p.fold_buffered = 0;
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
@@ -519,7 +534,11 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;
-  if (c->row_buffer) c->pending[layer] = 1;
+  c->last_scored = c->row_buffer ? layer : -1;
+  if (c->row_buffer) {
+    c->pending[layer] = 1;
+    c->lg_cur[layer] = (uint8_t)lg_next;
+  }
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -536,11 +555,9 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
-  if (c->row_buffer) {                 // the row buffer's append also maintains the scores: two launches
-    const int rc = ssd_append(c, layer, k_new, v_new, stream);
-    return rc != SSD_OK ? rc : ssd_decode_attn(c, layer, q, out, stream);
-  }
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
+  const bool scored = c->row_buffer && c->n_sink[layer] > 0;
+  if (scored && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;   // Algorithm 2, overflow branch
   DecodeParams p;
   p.slab = c->d_slab(layer);
   p.q = static_cast<const __nv_bfloat16*>(q);
@@ -548,11 +565,24 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   p.partial = c->d_partial();
   p.counters = c->d_counters();
   p.status = c->d_status();
-  p.logits = nullptr; p.ml = nullptr; p.mr = c->mr();
+  // Row-buffer mode (Algorithm 2): the launch records this step's logits in the layer's other buffer and,
+  // at its start, adds the previous step's weights to the scores: still one launch
+  const int lg_next = c->lg_cur[layer] ^ 1;
+  p.logits = scored ? c->d_logits(layer, lg_next) : nullptr;
+  p.ml = scored ? c->d_ml(layer, lg_next) : nullptr;
+  p.mr = c->mr();
+  p.sem_slot = scored ? c->sem_tokens(layer) : -1;
+  p.fold_acc = scored ? c->d_acc(layer) : nullptr;
+  p.fold_logits = c->d_logits(layer, c->lg_cur[layer]);
+  p.fold_ml = c->d_ml(layer, c->lg_cur[layer]);
+  p.fold_pending = scored && c->pending[layer] ? 1 : 0;
+  p.fold_static = c->static_valid[layer];
+  p.fold_buffered = c->sem_tokens(layer);
   p.k_new = static_cast<const unsigned char*>(k_new);
   p.v_new = static_cast<const unsigned char*>(v_new);
   p.new_j = c->t_img[layer];
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
+  p.fold_early = (p.early && c->last_scored >= -1 && c->last_scored != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->t_img[layer] += 1;                // the view describes the layer with the token in place
@@ -565,6 +595,11 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
     return SSD_ERR_CUDA;
   }
   c->last_writer = layer;
+  c->last_scored = scored ? layer : -1;
+  if (scored) {
+    c->pending[layer] = 1;
+    c->lg_cur[layer] = (uint8_t)lg_next;
+  }
   if (timed) {
     cudaEventRecord(c->prof_ev[2 * c->prof_n + 1], st);
     c->prof_n += 1;
@@ -597,7 +632,8 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   for (int i = 0; c->row_buffer && i < n_layers; ++i) {
     const int layer = first_layer + i;
     if (!c->pending[layer] || c->n_sink[layer] == 0) continue;
-    if (launch_fold_pending(c->d_acc(layer), c->d_logits(layer), c->d_ml(layer), c->d_desc(layer), g.n_seqs, g.n_heads,
+    if (launch_fold_pending(c->d_acc(layer), c->d_logits(layer, c->lg_cur[layer]), c->d_ml(layer, c->lg_cur[layer]),
+                            c->d_desc(layer), g.n_seqs, g.n_heads,
                             c->mr(), c->static_valid[layer], c->sem_tokens(layer), st) != cudaSuccess)
       return SSD_ERR_CUDA;
     c->pending[layer] = 0;
@@ -644,6 +680,7 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     }
   }
   c->last_writer = -2;                 // several layers' slabs were written
+  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -840,8 +877,8 @@ int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
     p.desc = c->d_desc(layer);
     p.static_idx = c->d_idx(layer);
     p.acc = c->d_acc(layer);
-    p.logits = c->d_logits(layer);
-    p.ml = c->d_ml(layer);
+    p.logits = c->d_logits(layer, c->lg_cur[layer]);
+    p.ml = c->d_ml(layer, c->lg_cur[layer]);
     p.pending = c->pending[layer];
     p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len; p.M = g.sink_budget; p.mr = c->mr();
     p.static_valid = c->static_valid[layer];
@@ -855,6 +892,7 @@ int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
   c->t_base[layer] = c->t_img[layer];
   c->pending[layer] = 0;
   c->last_writer = -2;
+  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -869,8 +907,8 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
   p.desc = c->d_desc(first_layer);
   p.static_idx = c->d_idx(first_layer);
   p.acc = c->d_acc(first_layer);
-  p.logits = c->d_logits(first_layer);
-  p.ml = c->d_ml(first_layer);
+  p.logits = c->d_logits(first_layer, 0);
+  p.ml = c->d_ml(first_layer, 0);
   p.n_layers = n_layers; p.n_seqs = g.n_seqs; p.H = g.n_heads; p.L = g.prompt_len; p.M = g.sink_budget; p.mr = c->mr();
   bool any = false;
   for (int i = 0; i < n_layers; ++i) {
@@ -882,6 +920,7 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
     ly.buffered = c->sem_tokens(layer);
     ly.t_base = c->t_base[layer];
     ly.pending = c->pending[layer];
+    ly.lg = c->lg_cur[layer];
     ly.todo = (c->n_sink[layer] > 0 && (ly.buffered > 0 || ly.pending)) ? 1 : 0;
     any = any || ly.todo;
   }
@@ -896,6 +935,7 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
     c->pending[layer] = 0;
   }
   c->last_writer = -2;
+  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -909,8 +949,8 @@ int ssd_cache_get_scores(ssd_cache* c, int32_t layer, float* acc_host) {
   std::vector<float2> ml((size_t)g.n_seqs * g.n_heads);
   if (cudaDeviceSynchronize() != cudaSuccess ||
       cudaMemcpy(acc_host, c->d_acc(layer), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-      cudaMemcpy(lg.data(), c->d_logits(layer), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-      cudaMemcpy(ml.data(), c->d_ml(layer), ml.size() * 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaMemcpy(lg.data(), c->d_logits(layer, c->lg_cur[layer]), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(ml.data(), c->d_ml(layer, c->lg_cur[layer]), ml.size() * 8, cudaMemcpyDeviceToHost) != cudaSuccess) {
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }
@@ -1058,16 +1098,23 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.partial = reinterpret_cast<float*>(base);
   p.counters = reinterpret_cast<uint32_t*>(base + kStaticPartialBytes);
   p.status = c->d_status();
-  p.logits = c->row_buffer ? c->d_logits(layer) : nullptr;
-  p.ml = c->row_buffer ? c->d_ml(layer) : nullptr;
+  const int lg_next = c->lg_cur[layer] ^ 1;
+  p.logits = c->row_buffer ? c->d_logits(layer, lg_next) : nullptr;
+  p.ml = c->row_buffer ? c->d_ml(layer, lg_next) : nullptr;
   p.mr = c->mr();
-  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1;
+  p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1; p.sem_slot = -1;
+  p.fold_acc = nullptr; p.fold_logits = nullptr; p.fold_ml = nullptr;
+  p.fold_pending = 0; p.fold_early = 0; p.fold_static = 0; p.fold_buffered = 0;
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;
-  if (c->row_buffer) c->pending[layer] = 1;
+  c->last_scored = c->row_buffer ? layer : -1;
+  if (c->row_buffer) {
+    c->pending[layer] = 1;
+    c->lg_cur[layer] = (uint8_t)lg_next;
+  }
   return SSD_OK;
 }

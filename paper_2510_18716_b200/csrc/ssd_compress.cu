@@ -322,8 +322,8 @@ __global__ void __launch_bounds__(kThreads) ssd_recompress_layers_kernel(const _
   p.desc = q.desc + (size_t)layer * q.H;
   p.static_idx = q.static_idx + (size_t)layer * pairs * (q.M > 0 ? q.M : 1);
   p.acc = q.acc + (size_t)layer * pairs * q.mr;
-  p.logits = q.logits + (size_t)layer * pairs * q.mr;
-  p.ml = q.ml + (size_t)layer * pairs;
+  p.logits = q.logits + ((size_t)layer * 2 + ly.lg) * pairs * q.mr;
+  p.ml = q.ml + ((size_t)layer * 2 + ly.lg) * pairs;
   p.pending = ly.pending;
   p.n_seqs = q.n_seqs; p.H = q.H; p.L = q.L; p.M = q.M; p.mr = q.mr;
   p.static_valid = ly.static_valid;

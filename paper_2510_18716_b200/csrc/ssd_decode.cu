@@ -334,11 +334,64 @@ __device__ __forceinline__ void head_workers(const Split& sp, int wk, int g0, in
 
 // Fused append: valid-slot index, inside head h, of the token being appended (its ring slot holds
 // stale bytes in the slab), and that slot's index from the head's first slot.
-__device__ __forceinline__ void new_token_slot(const LayerView& v, int h, int new_j, int& valid_idx, int& phys) {
+__device__ __forceinline__ void new_token_slot(const LayerView& v, int h, int new_j, int sem_slot, int& valid_idx, int& phys) {
   const HeadRec d = v.head[h];
-  const int r = new_j % d.z;
+  const int r = (d.w && sem_slot >= 0) ? sem_slot : new_j % d.z;   // a row buffer fills from its slot 0
   valid_idx = v.prompt_valid + (d.w ? v.static_valid : 0) + r;
   phys = v.L + d.y + r;
+}
+
+// Algorithm 2, score accumulation, deferred by one step: the weights of the layer's previous decode go into
+// the scores at the start of the layer's next launch (nothing in that launch reads the scores), and the
+// token being appended starts at zero.  Run by the finisher warp of every thread block, which share the
+// pairs; entry c of a score row is static slot c or, from the static capacity on, buffer slot c - capacity.
+__device__ void fold_scores(const DecodeParams& p, int lane) {
+  const LayerView& v = p.view;
+  // Items (pair, entry) are dealt to the lanes kFoldBatch at a time, loads first, so that the warp has
+  // hundreds of independent loads in flight: with HBM saturated by the streaming warps a dependent trip
+  // to memory takes microseconds, and one trip per item would outlast the launch.
+  constexpr int kFoldBatch = 16;
+  const int n_pairs = v.n_seqs * v.H;
+  const int n_mine = (n_pairs - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  float* __restrict__ accp = p.fold_acc;
+  if (p.fold_pending) {
+    const float* __restrict__ lgp = p.fold_logits;
+    const float2* __restrict__ mlp = p.fold_ml;
+    const int total = n_mine * p.mr;
+    for (int it0 = lane; it0 < total; it0 += 32 * kFoldBatch) {
+      float a[kFoldBatch], x[kFoldBatch];
+      float2 ml[kFoldBatch];
+      uint32_t off[kFoldBatch];
+      bool ok[kFoldBatch];
+#pragma unroll
+      for (int u = 0; u < kFoldBatch; ++u) {
+        const int it = it0 + 32 * u;
+        const int k = it / p.mr, c = it - k * p.mr;
+        const int pair = (int)blockIdx.x + k * (int)gridDim.x;
+        ok[u] = false;
+        if (it < total) {
+          const HeadRec d = v.head[pair % v.H];
+          ok[u] = d.w && (c < p.fold_static || (c >= d.y && c < d.y + p.fold_buffered));
+        }
+        off[u] = (uint32_t)pair * (uint32_t)p.mr + (uint32_t)c;      // n_seqs * H * (M + R) < 2^31 (checked at create)
+        if (ok[u]) {
+          a[u] = accp[off[u]];
+          x[u] = lgp[off[u]];
+          ml[u] = mlp[pair];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kFoldBatch; ++u)
+        if (ok[u]) accp[off[u]] = a[u] + ex2(x[u] - ml[u].x) / ml[u].y;
+    }
+  }
+  if (p.sem_slot >= 0) {
+    for (int k = lane; k < n_mine; k += 32) {
+      const int pair = (int)blockIdx.x + k * (int)gridDim.x;
+      const HeadRec d = v.head[pair % v.H];
+      if (d.w) accp[(size_t)pair * p.mr + d.y + p.sem_slot] = 0.f;
+    }
+  }
 }
 
 // The finisher warp of a CTA carries the (at most two) heads that cross the CTA's own range
@@ -376,9 +429,14 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
     }
   }
   unsigned heads = __ballot_sync(FULL, r_pair >= 0);
-  if (!heads) return;
+  if (!heads && p.fold_acc == nullptr) return;
+  // the scores belong to this layer: when the preceding launch worked on another layer's tables nothing can
+  // still be writing them
+  if (p.fold_acc != nullptr && p.fold_early) fold_scores(p, lane);
   pdl_wait_predecessor();                // the scratch below may still be in use by the previous launch
   pdl_allow_successor();
+  if (p.fold_acc != nullptr && !p.fold_early) fold_scores(p, lane);
+  if (!heads) return;
   for (unsigned h = heads; h; h &= h - 1) {
     const int slot = __ffs(h) - 1;       // 0: began in an earlier CTA, 1: begins here and runs on
     if (!mbar_wait(cta_bar0 + 8 * slot, 0)) {
@@ -487,7 +545,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
                                  ((size_t)w.seq * v.seq_slots + v.head[w.head].x) * kSlotBytes;
     if (p.new_j >= 0 && pf_key != w.seq * v.H + w.head) {      // once per head, not per chunk
       pf_key = w.seq * v.H + w.head;
-      new_token_slot(v, w.head, p.new_j, pf_fresh, pf_phys);
+      new_token_slot(v, w.head, p.new_j, p.sem_slot, pf_fresh, pf_phys);
     }
     const int fresh = pf_fresh;
     const bool has_fresh = fresh >= w.i && fresh < w.i + n;
@@ -595,7 +653,7 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
       sink.skip = v.prompt_valid;
       sink.ring_from = v.prompt_valid + v.static_valid;
       sink.ring_shift = d.y - v.static_valid;
-      if (p.new_j >= 0) new_token_slot(v, cons.head, p.new_j, fresh, fresh_phys);
+      if (p.new_j >= 0) new_token_slot(v, cons.head, p.new_j, p.sem_slot, fresh, fresh_phys);
     }
     sink.i0 = cons.i;
     Rows rows;

@@ -40,6 +40,18 @@ struct DecodeParams {
   const unsigned char* k_new;  // [n_seqs, H, 128] bf16: K row of image token new_j
   const unsigned char* v_new;
   int new_j;                // image index of that token; the view already counts it
+  int sem_slot;             // row-buffer mode: buffer slot of that token in semantic heads; else -1 (slot new_j mod R)
+  // Row-buffer mode, fused append (Algorithm 2, score accumulation, one launch per step and layer): before
+  // anything else the launch brings the scores up to date with the layer's PREVIOUS decode, whose logits
+  // and (max, exp-sum) are in fold_logits / fold_ml (the other of two alternating buffers, so that this
+  // launch's own logits do not overwrite them), and starts the new token's score at zero.  fold_acc ==
+  // nullptr: nothing to do.
+  float* fold_acc;          // [n_seqs * H, M + R]
+  const float* fold_logits; // [n_seqs * H, M + R]; read only if fold_pending
+  const float2* fold_ml;    // [n_seqs * H]
+  int fold_pending;         // 1: the previous decode's weights are not yet in the scores
+  int fold_early;           // 1: the launch before this one does not write this layer's score tables either
+  int fold_static, fold_buffered;   // static and buffered entries that held a token at that decode
   int early;                // 1: the launch before this one on the stream does not write this layer's slab
   float scale_log2;         // softmax scale * log2(e)
   Split split;              // how the layer's slots are shared out (set by launch_decode)
@@ -170,6 +182,7 @@ cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st);
 struct RecompressLayer {
   long long first_slot;        // the layer's first slot in the slab
   int seq_slots, static_valid, buffered, t_base, pending;
+  int lg;                      // which of the layer's two logit buffers holds the pending logits
   int todo;                    // 0: nothing buffered and nothing pending in this layer
 };
 struct RecompressLayersParams {
@@ -177,7 +190,7 @@ struct RecompressLayersParams {
   const HeadDesc* desc;        // first layer's [H] records; next layer H records further
   int32_t* static_idx;         // first layer's [n_seqs, H, M]
   float* acc;                  // first layer's [n_seqs * H, mr]
-  const float* logits;
+  const float* logits;         // first layer's first buffer; two buffers per layer
   const float2* ml;
   int n_layers, n_seqs, H, L, M, mr;
   RecompressLayer layer[kMaxLayersPerLaunch];
