@@ -16,8 +16,17 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls enqueue work
  *    on it and return; exceptions are noted per function.  One cache must be driven from one
  *    stream at a time (launches that overlap on the GPU would race on its scratch areas).
+ *  - Host threads: a cache is not synchronised; calls on the SAME cache must not overlap in time
+ *    (its host state, e.g. the token counters, is plain data).  Calls on DIFFERENT caches may run
+ *    on different host threads concurrently: what they share (the per-device set-up of the kernels'
+ *    shared-memory limits, the launch counter, the fixed array of ssd_decode_attn_static) is set
+ *    up or updated atomically.  Every call acts on the calling thread's current device, which must
+ *    be the device that holds the cache's buffer.
  *  - L = prompt_len prompt tokens are retained whole by every head.  Image token j (0-based)
- *    has absolute position L + j; image step t = j + 1.
+ *    has absolute position L + j; image step t = j + 1.  The "initial sink token" that Sec. 3.3
+ *    keeps beside the window of a spatial head is position 0, i.e. the first prompt token, which
+ *    is retained with the prompt; with prompt_len = 0 there is no such token and a spatial head
+ *    keeps exactly its W newest image tokens.
  *  - All sequences advance in lock step: every call acts on all n_seqs sequences of a layer.
  *  - Every function returns an ssd_status (0 = SSD_OK, negative = error) unless noted; all
  *    argument checking happens on the host before anything is launched.
@@ -124,13 +133,18 @@ int ssd_set_head_labels(ssd_cache *cache, const uint8_t *labels_host);
  * tokens among j in [0, n0-R) (ties: lowest j), stored in ascending j, plus the R newest tokens.
  * Spatial heads: keep the W newest tokens.  Every head keeps the whole prompt.
  * 0 <= n0 <= max_image_tokens; 0 <= n_obs <= n0 (q_obs may be NULL when n_obs == 0 or the layer
- * has no semantic head).  Replaces the layer's previous contents.  Asynchronous. */
+ * has no semantic head).  Replaces the layer's previous contents.  Asynchronous.
+ * SSD_ERR_LIMIT if scores are needed (a semantic head, n_obs > 0) and n0 > 7808: a pair's score rows
+ * are kept in shared memory beside the operand tiles.  Should a bounded wait of the scoring kernel
+ * run out, the scores of that pair are written as zeros and bit 2 of the device status word is set
+ * (ssd_cache_device_status): check it after compressing when the selection matters. */
 int ssd_compress(ssd_cache *cache, int32_t layer, const void *q_obs, const void *k_full,
                  const void *v_full, int32_t n0, int32_t n_obs, void *stream);
 
 /* Append the newest token's K/V for every (sequence, head) of a layer: written into the head's
  * ring, overwriting (evicting) the oldest ring entry once the ring is full (Algorithm 1, Append).
- *   k_new, v_new [n_seqs, n_heads, head_dim]
+ *   k_new, v_new [n_seqs, n_heads, head_dim], 16-byte aligned (SSD_ERR_INVALID_ARG otherwise: the
+ *   kernel reads them 16 bytes at a time)
  * SSD_ERR_OVERFLOW once max_image_tokens tokens are held.  Asynchronous. */
 int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v_new, void *stream);
 
@@ -140,7 +154,8 @@ int ssd_append(ssd_cache *cache, int32_t layer, const void *k_new, const void *v
  * out[s,h] = sum_i softmax_i(scale * <q[s,h], K_i>) V_i over the prompt, static and ring slots
  * that hold a token (the token just appended included).  fp32 accumulation, bf16 output.
  *   q, out [n_seqs, n_heads, head_dim], 16-byte aligned
- * SSD_ERR_BAD_STATE if the layer holds no token at all.  Asynchronous. */
+ * SSD_ERR_BAD_STATE if some head of the layer holds no token at all (no prompt loaded and, for that
+ * head's type, nothing in its static set or ring): attention over nothing has no value.  Asynchronous. */
 int ssd_decode_attn(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
 /* ssd_append followed by ssd_decode_attn for the same layer, in one kernel launch (Algorithm 1's
@@ -204,6 +219,13 @@ int ssd_recompress(ssd_cache *cache, int32_t layer, void *stream);
  * SSD_ERR_LIMIT if n_layers > 64. */
 int ssd_recompress_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, void *stream);
 int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
+
+/* The accumulated scores the latest ssd_compress computed (Algorithm 1, AttentionScores summed over the
+ * observed steps), before selection: score_host [n_seqs, n_heads, n0] float, -1 for spatial heads.
+ * The scores live in a buffer that every ssd_compress and ssd_classify_* call reuses, so this works only
+ * for the layer compressed last (SSD_ERR_BAD_STATE otherwise, or if that call needed no scores).
+ * For inspection and parity; synchronises the device. */
+int ssd_cache_get_compress_scores(ssd_cache *cache, int32_t layer, float *score_host);
 
 /* ssd_decode_attn for callers that cannot allocate.  The paper has no counterpart; this is a
  * packaging variant of the same kernel.  ssd_decode_attn keeps the kernel's scratch (partial sums of
@@ -280,11 +302,17 @@ int ssd_cache_kv_bytes(ssd_cache *cache, size_t *bytes_per_seq);
 int ssd_profile_enable(ssd_cache *cache, int32_t max_launches);
 int ssd_profile_collect(ssd_cache *cache, float *ms_host, int32_t *n_out);
 
-/* Device status word of the cache (0 = healthy).  Bit 0: a decode warp gave up a bounded wait
- * for one of its asynchronous copies or for a partial result (each wait is limited to about a
- * second); the outputs of that launch are then incomplete.  The kernels never trap and never spin
- * without a limit, so the CUDA context stays usable.  Synchronises the device.  No paper
- * counterpart. */
+/* Device status word of the cache (0 = healthy).  Every wait inside a kernel is limited to about a
+ * second; a kernel that gives one up sets a bit here and finishes without the missing data:
+ *   bit 0 (1): a decode warp (ssd_decode_attn, ssd_append_decode, ssd_append_decode_layers,
+ *              ssd_decode_attn_static) gave up waiting for one of its asynchronous copies or for a partial
+ *              result; the outputs of that launch are incomplete;
+ *   bit 1 (2): the classifier (ssd_classify_heads / ssd_classify_partial) gave up; its sparsity values
+ *              are incomplete;
+ *   bit 2 (4): the scoring kernel of ssd_compress gave up; the scores of the affected pairs are zero,
+ *              so their top-M is the M lowest candidates.
+ * The bits are sticky until the cache is recreated.  The kernels never trap and never spin without a
+ * limit, so the CUDA context stays usable.  Synchronises the device.  No paper counterpart. */
 int ssd_cache_device_status(ssd_cache *cache, uint32_t *status_host);
 
 /* Inspection of the decode kernel's work decomposition, computed on the host by the same code the

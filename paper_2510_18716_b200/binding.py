@@ -31,7 +31,7 @@ EXPORTS = [
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
-    "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity",
+    "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity", "ssd_cache_get_compress_scores",
 ]
 
 
@@ -84,6 +84,7 @@ def load():
     L.ssd_labels_from_sparsity.argtypes = [vp, C.c_int64, C.c_float, vp]
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
+    L.ssd_cache_get_compress_scores.argtypes = [vp, i32, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_append_decode_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_recompress_layers.argtypes = [vp, i32, i32, vp]
@@ -308,6 +309,13 @@ class SsdCache:
         c = self.cfg
         a = np.empty((c.n_seqs, c.n_heads, c.sink_budget + c.sink_recent), np.float32)
         self._check(self.lib.ssd_cache_get_scores(self._h, layer, a.ctypes.data), "ssd_cache_get_scores")
+        return a
+
+    def get_compress_scores(self, layer: int, n0: int) -> np.ndarray:
+        """Scores of the latest compress call (which must have been on `layer`, at n0 image tokens)."""
+        c = self.cfg
+        a = np.empty((c.n_seqs, c.n_heads, n0), np.float32)
+        self._check(self.lib.ssd_cache_get_compress_scores(self._h, layer, a.ctypes.data), "ssd_cache_get_compress_scores")
         return a
 
     def step_host(self, layer: int, q_host, k_new_host, v_new_host, out_host):

@@ -92,6 +92,7 @@ struct ssd_cache {
   int last_writer = -2;
   // The same for the layer's score tables of the row-buffer mode (accumulated scores, logits, (max, sum)).
   int last_scored = -2;
+  int score_layer = -1, score_n0 = 0; // layer whose prefill scores (ssd_compress) the score buffer holds, -1 if none
   bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
   std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
   std::vector<uint8_t> pending;       // [layers] last decode's logits not yet added to the scores
@@ -132,6 +133,13 @@ struct ssd_cache {
   int max_slots() const {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
     return cfg.prompt_len + (a > b ? a : b);
+  }
+  // True if some head of the layer would hold no token at all with t image tokens in the layer (t_sem of
+  // them in the rings of semantic heads): attention over nothing has no value, so decode refuses.
+  bool empty_head(int layer, int t, int t_sem) const {
+    if (prompt_valid[layer] > 0) return false;
+    if (n_sink[layer] < cfg.n_heads && t == 0) return true;                               // a spatial head
+    return n_sink[layer] > 0 && static_valid[layer] == 0 && t_sem == 0;                   // a semantic head
   }
   // layout and occupancy of a layer, as the decode kernel sees it
   void fill_view(int layer, LayerView& v) const {
@@ -355,6 +363,7 @@ int ssd_classify_partial(ssd_cache* c, const void* q_cal, const void* k_cal, int
   p.N = n_img;
   p.w = g.cls_window;
   p.scale_log2 = c->scale * 1.4426950408889634f;
+  c->score_layer = -1;                 // the partial sums share the score buffer
   if (launch_classify(p, nrb, st) != cudaSuccess) return SSD_ERR_CUDA;
   std::vector<float> part(units * nrb);
   if (cudaMemcpyAsync(part.data(), c->d_score(), part.size() * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
@@ -426,6 +435,8 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   const int sv = g.sink_budget < n_cand ? g.sink_budget : n_cand;
   const bool select = c->n_sink[layer] > 0 && sv > 0;
   if (select && n_obs > 0 && !q_obs) return SSD_ERR_INVALID_ARG;
+  if (select && n_obs > 0 && n0 > score_max_n0()) return SSD_ERR_LIMIT;   // score rows of a pair live in shared memory
+  c->score_layer = -1;
   const HeadDesc* desc = c->d_desc(layer);
   if (select) {
     if (n_obs > 0) {
@@ -449,6 +460,8 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
     sl.mr = c->mr();
     sl.n_seqs = g.n_seqs; sl.H = g.n_heads; sl.M = g.sink_budget; sl.n0 = n0; sl.n_cand = n_cand;
     if (launch_select(sl, st) != cudaSuccess) return SSD_ERR_CUDA;
+    c->score_layer = layer;
+    c->score_n0 = n0;
   }
   GatherParams gp;
   gp.slab = c->d_slab(layer);
@@ -509,7 +522,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
-  if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
+  if (c->empty_head(layer, c->t_img[layer], c->sem_tokens(layer))) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   DecodeParams p;
   p.slab = c->d_slab(layer);
@@ -616,7 +629,7 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   // Row buffer of one token: the launch re-selects as well (Algorithm 1 taken literally)
   const bool evict = c->row_buffer && g.sink_recent == 1;
-  if (c->row_buffer && c->mr() * (evict ? 3 : 1) > decode_layers_max_mr()) return SSD_ERR_LIMIT;
+  if (c->row_buffer && ((c->mr() + 3) & ~3) * (evict ? 3 : 1) > decode_layers_max_mr()) return SSD_ERR_LIMIT;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
@@ -968,6 +981,23 @@ int ssd_cache_get_scores(ssd_cache* c, int32_t layer, float* acc_host) {
   return SSD_OK;
 }
 
+int ssd_cache_get_compress_scores(ssd_cache* c, int32_t layer, float* score_host) {
+  if (!c || !score_host) return SSD_ERR_INVALID_ARG;
+  const ssd_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
+  if (c->score_layer != layer || c->score_n0 < 1) return SSD_ERR_BAD_STATE;
+  const size_t n = (size_t)g.n_seqs * g.n_heads * c->score_n0;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(score_host, c->d_score(), n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SSD_ERR_CUDA;
+  }
+  for (int pr = 0; pr < g.n_seqs * g.n_heads; ++pr)
+    if (!c->desc[(size_t)layer * g.n_heads + pr % g.n_heads].w)
+      for (int j = 0; j < c->score_n0; ++j) score_host[(size_t)pr * c->score_n0 + j] = -1.f;
+  return SSD_OK;
+}
+
 int ssd_cache_device_status(ssd_cache* c, uint32_t* status_host) {
   if (!c || !status_host) return SSD_ERR_INVALID_ARG;
   if (cudaDeviceSynchronize() != cudaSuccess ||
@@ -1056,21 +1086,23 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
-  if (c->prompt_valid[layer] == 0 && c->t_img[layer] == 0) return SSD_ERR_BAD_STATE;
+  if (c->empty_head(layer, c->t_img[layer], c->sem_tokens(layer))) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   const long pairs = (long)g.n_seqs * g.n_heads;
   if (pairs > kStaticPairs) return SSD_ERR_LIMIT;
 
   // Once per device, with that device current: the array's name is only a host-side handle here,
   // so ask the runtime where the array lives on this device.
-  static unsigned char* dev_ptr[64] = {};
-  static int dev_sms[64] = {};
+  // (two host threads that make their first call at once both look the address up and store the same value)
+  static std::atomic<unsigned char*> dev_ptr[64] = {};
+  static std::atomic<int> dev_sms[64] = {};
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }
-  if (!dev_ptr[dev]) {
+  unsigned char* base = dev_ptr[dev].load(std::memory_order_acquire);
+  if (!base) {
     void* ptr = nullptr;
     int sms = 0;
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr ||
@@ -1078,13 +1110,13 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
       cudaGetLastError();
       return SSD_ERR_CUDA;
     }
-    dev_sms[dev] = sms;
-    dev_ptr[dev] = static_cast<unsigned char*>(ptr);
+    dev_sms[dev].store(sms, std::memory_order_relaxed);
+    base = static_cast<unsigned char*>(ptr);
+    dev_ptr[dev].store(base, std::memory_order_release);
   }
-  if (dev_sms[dev] > kStaticCtas) return SSD_ERR_LIMIT;   // the kernel runs one thread block per SM
+  if (dev_sms[dev].load(std::memory_order_relaxed) > kStaticCtas) return SSD_ERR_LIMIT;   // the kernel runs one thread block per SM
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  unsigned char* base = dev_ptr[dev];
   // The array keeps what the previous call left.  Partials are written before they are read, but
   // the arrival counters must start at zero, which a call that was cut short would not guarantee.
   if (cudaMemsetAsync(base + kStaticPartialBytes, 0, (size_t)pairs * 4, st) != cudaSuccess) {

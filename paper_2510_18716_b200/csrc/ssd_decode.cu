@@ -35,6 +35,8 @@
 // during the launch, so no ordering is needed, and the per-layer append launch disappears.
 // Every wait on an mbarrier is bounded: a warp that gives up raises a bit in the status word,
 // waits (bounded again) for its other copies in flight and leaves.
+#include <atomic>
+
 #include "ssd_internal.cuh"
 
 #ifndef SSD_DECODE_WARPS
@@ -1098,24 +1100,24 @@ int decode_max_workers() {
 }
 
 cudaError_t launch_decode(const DecodeParams& p_in, cudaStream_t st) {
-  static bool smem_set[64] = {};
-  static int max_workers[64] = {};
+  // Per-device set-up, done once; two host threads that meet here both do it (the calls are idempotent)
+  // and publish the same value: 0 = not yet set up, else the device's worker count.
+  static std::atomic<int> max_workers[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   const bool cached = dev >= 0 && dev < 64;
-  if (!cached || !smem_set[dev]) {
+  int workers = cached ? max_workers[dev].load(std::memory_order_acquire) : 0;
+  if (workers == 0) {
     e = cudaFuncSetAttribute(ssd_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    if (cached) {
-      smem_set[dev] = true;
-      max_workers[dev] = decode_max_workers();
-    }
+    workers = decode_max_workers();
+    if (cached) max_workers[dev].store(workers, std::memory_order_release);
   }
   DecodeParams p = p_in;
   const long total = (long)p.view.cum[p.view.H] * p.view.n_seqs;
   if (total < 1 || total > 0x7fffffffL) return cudaErrorInvalidValue;
-  const long w = plan_workers(total, cached ? max_workers[dev] : decode_max_workers());
+  const long w = plan_workers(total, workers);
   p.split = make_split(total, w);
   const int grid = (int)((w + kWarps - 1) / kWarps);
   cudaLaunchConfig_t cfg = {};
@@ -1146,14 +1148,13 @@ cudaError_t launch_fold_pending(float* acc, const float* logits, const float2* m
 }
 
 cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
-  static bool smem_set[64] = {};
-  static int n_sm[64] = {};
+  static std::atomic<int> n_sm[64] = {};   // 0 = this device is not set up yet (see launch_decode)
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   const bool cached = dev >= 0 && dev < 64;
-  int sms = cached ? n_sm[dev] : 0;
-  if (!cached || !smem_set[dev]) {
+  int sms = cached ? n_sm[dev].load(std::memory_order_acquire) : 0;
+  if (sms == 0) {
     e = cudaFuncSetAttribute(ssd_decode_layers_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kLayersSmemBytes + kWarps * decode_layers_max_mr() * 4);
     if (e == cudaSuccess)
@@ -1161,10 +1162,7 @@ cudaError_t launch_decode_layers(const DecodeLayersParams& p, cudaStream_t st) {
                                kLayersSmemBytes + kWarps * decode_layers_max_mr() * 4);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    if (cached) {
-      smem_set[dev] = true;
-      n_sm[dev] = sms;
-    }
+    if (cached) n_sm[dev].store(sms, std::memory_order_release);
   }
   const long units = (long)p.n_layers * p.n_seqs * p.H;
   if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;

@@ -161,6 +161,7 @@ int decode_layers_max_mr();
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
+int score_max_n0();   // most image tokens whose score rows fit beside the scoring kernel's tiles in shared memory
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
 struct RecompressParams {
   uint4* slab;

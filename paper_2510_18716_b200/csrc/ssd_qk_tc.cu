@@ -662,9 +662,12 @@ cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStrea
   return cudaGetLastError();
 }
 
+// a pair's four score rows (one per lane quadrant) sit beside the tiles; 8 KB stay free for the static arrays
+int score_max_n0() { return (int)((227 * 1024 - 8192 - 1024 - (1 + kStages) * (size_t)kTileBytes) / (4 * sizeof(float))); }
+
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
   const size_t smem = (1 + kStages) * (size_t)kTileBytes + 4 * (size_t)p.n0 * sizeof(float) + 1024;
-  if (smem + 8192 > 227 * 1024) return cudaErrorInvalidValue;   // 8 KB left for the kernel's static arrays
+  if (p.n0 > score_max_n0()) return cudaErrorInvalidValue;
   CUtensorMap tq, tk;
   const uint64_t pairs = (uint64_t)p.n_seqs * p.H;
   cudaError_t e = make_tile_map(&tq, p.q_obs, (uint64_t)p.n_obs, pairs);

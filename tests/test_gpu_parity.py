@@ -354,3 +354,79 @@ def test_sweep_batch128_full_launch_size_sampled_pairs():
     cfg = wl.sweep(128, 5, 0.5)
     from parity_util import run_sampled
     run_sampled(cfg, 2, _sample_pairs(cfg, 2, 8, 2), (cfg.n0 + 1, cfg.n0 + 26))
+
+
+@pytest.mark.parametrize("name,layer,n_seqs", [("janus7b", 11, 64), ("hires7b", 2, 2)])
+def test_compress_scores_elementwise(name, layer, n_seqs):
+    """Algorithm 1, AttentionScores summed over the observed steps: the score rows ssd_compress selects
+    from, element by element against the oracle (not only through the sets they produce)."""
+    cfg = wl.CONFIGS[name]
+    dev = torch.device("cuda:0")
+    L, n0, M, R, H = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.n_heads
+    labels = wl.sink_mask(cfg, layer)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=n_seqs), device=dev)
+    cache.set_head_labels(labels)
+    with pytest.raises(B.SsdError) as e:
+        cache.get_compress_scores(0, n0)                 # nothing compressed yet
+    assert e.value.code == B.SSD_ERR_BAD_STATE
+    q, k, v, _ = wl.gen_layer(cfg, layer, list(range(n_seqs)), device=dev)
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+    got = cache.get_compress_scores(0, n0)
+    assert cache.device_status() == 0
+    sem = labels[None, :].repeat(n_seqs, 0).astype(np.uint8)
+    want, _, _ = oracle.select_batch(wl.to_u16(q[:, :, :n0]), wl.to_u16(k[:, :, : L + n0]), sem, L, n0, M, R)
+    for h in range(H):
+        if labels[h]:
+            assert np.allclose(got[:, h], want[:, h], rtol=2e-4, atol=1e-7), (h, np.abs(got[:, h] - want[:, h]).max())
+            assert (got[:, h] >= 0).all()
+        else:
+            assert (got[:, h] == -1).all()
+    cache.close()
+
+
+def test_exact_ties_on_the_radix_path_select_the_lowest_indices():
+    """Algorithm 1, IndicesOfTopM with the lowest-index tie rule, where the selection radix-selects the
+    threshold (more than 1024 candidates): with no observed step every score is zero, all candidates tie,
+    and the M lowest must be kept."""
+    cfg = wl.CONFIGS["hires7b"]
+    dev = torch.device("cuda:0")
+    L, n0, M, R, H = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.n_heads
+    assert n0 - R > 1024
+    labels = wl.sink_mask(cfg, 0)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=1), device=dev)
+    cache.set_head_labels(labels)
+    _, k, v, _ = wl.gen_layer(cfg, 0, [0], device=dev)
+    cache.compress(0, None, k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0, 0)
+    gi = cache.get_indices(0)
+    want = oracle.topm(np.zeros(n0 - R), n0 - R, M)
+    assert np.array_equal(want, np.arange(M))
+    for h in range(H):
+        if labels[h]:
+            assert np.array_equal(gi[0, h, L:L + M] - L, want), h
+    assert cache.device_status() == 0
+    cache.close()
+
+
+@pytest.mark.parametrize("frac", [0.25, 0.75])
+def test_sweep_point_through_the_classifier(frac):
+    """A point of the large-batch sweep with a quarter / three quarters of the heads semantic: the
+    classifier has to recover that split (and everything after it is checked as usual)."""
+    cfg = wl.sweep(32, 5, frac)
+    assert cfg.n_sink_heads == round(frac * cfg.n_heads)
+    r = run_workload(cfg, [3, 17], [0, 1], (cfg.n0 + 1, cfg.n_img), classify=True)
+    assert r.steps_checked == 4
+
+
+def test_append_refuses_misaligned_rows_before_any_launch():
+    cfg = wl.CONFIGS["tiny"]
+    dev = torch.device("cuda:0")
+    cache = B.SsdCache(B.config_from_workload(cfg), device=dev)
+    cache.set_head_labels(wl.sink_mask(cfg, 0))
+    x = torch.zeros((cfg.n_seqs * cfg.n_heads * 128 + 8,), dtype=torch.bfloat16, device=dev)
+    lib, st = B.load(), torch.cuda.current_stream().cuda_stream
+    before = B.kernel_launch_count()
+    assert lib.ssd_append(cache._h, 0, x.data_ptr() + 2, x.data_ptr(), st) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_append(cache._h, 0, x.data_ptr(), x.data_ptr() + 2, st) == B.SSD_ERR_INVALID_ARG
+    assert B.kernel_launch_count() == before and cache.tokens(0) == 0
+    assert lib.ssd_append(cache._h, 0, x.data_ptr(), x.data_ptr(), st) == B.SSD_OK
+    cache.close()

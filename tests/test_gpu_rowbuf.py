@@ -267,3 +267,135 @@ def test_eviction_in_the_launch_equals_reselection_after_the_step(case):
     assert general.device_status() == 0 and fused.device_status() == 0
     for c in caches:
         c.close()
+
+
+def _run_full_launch_sampled(cfg, n_layers, seqs, sample, n_steps, form, evict=False):
+    """The launch sizes the benchmark times (all `seqs` x all heads x `n_layers` layers), row-buffer mode;
+    the oracle replays only the sampled (layer, sequence, head) pairs: every step's output, and the static
+    set after every re-selection (exact outside the 1e-5 band, following the GPU's choice inside it).
+    form: "per_layer" (ssd_append_decode per layer; ssd_recompress_layers when the buffer is full, after
+    every step when evict) or "one_launch" (ssd_append_decode_layers; with evict it re-selects itself).
+    Returns (re-selections replayed, of which inside the band)."""
+    import dataclasses
+    if evict:      # Algorithm 1 taken literally: a buffer of one token, same number of slots per head
+        cfg = dataclasses.replace(cfg, sink_budget=cfg.sink_budget + cfg.sink_recent - 1, sink_recent=1,
+                                  name=cfg.name + "_evict")
+    dev = torch.device("cuda:0")
+    L, n0, M, R, W, H, S = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.window, cfg.n_heads, len(seqs)
+    labels = np.stack([wl.sink_mask(cfg, l) for l in range(n_layers)])
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=n_layers, n_seqs=S),
+                       n_sink_heads_total=int(labels.sum()), device=dev)
+    cache.set_row_buffer(True)
+    cache.set_head_labels(labels)
+    step_in = [torch.empty((n_steps, n_layers, S, H, 128), dtype=torch.bfloat16, device=dev) for _ in range(3)]
+    picked = {}
+    for layer in range(n_layers):
+        q, k, v, _ = wl.gen_layer(cfg, layer, seqs, device=dev)
+        cache.compress(layer, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        step_in[0][:, layer] = q[:, :, n0:n0 + n_steps].permute(2, 0, 1, 3)
+        step_in[1][:, layer] = k[:, :, L + n0:L + n0 + n_steps].permute(2, 0, 1, 3)
+        step_in[2][:, layer] = v[:, :, L + n0:L + n0 + n_steps].permute(2, 0, 1, 3)
+        for (l, s, h) in sample:
+            if l == layer:
+                picked[(l, s, h)] = (wl.to_u16(q[s, h]), wl.to_u16(k[s, h]), wl.to_u16(v[s, h]))
+        del q, k, v
+    assert len(picked) == len(sample)
+    sample_layers = sorted({l for (l, _, _) in sample})
+    outs = {key: [] for key in sample}
+    gpu_sets = {}
+    out = torch.empty((S, H, 128), dtype=torch.bfloat16, device=dev)
+    for i in range(n_steps):
+        t = n0 + 1 + i
+        if form == "one_launch":
+            o = cache.append_decode_layers(0, step_in[1][i], step_in[2][i], step_in[0][i])
+            for key in sample:
+                outs[key].append(o[key[0], key[1], key[2]].clone())
+        else:
+            for layer in range(n_layers):
+                cache.append_decode(layer, step_in[1][i, layer], step_in[2][i, layer], step_in[0][i, layer], out)
+                for key in sample:
+                    if key[0] == layer:
+                        outs[key].append(out[key[1], key[2]].clone())
+        if (t - n0) % R == 0:
+            if not (evict and form == "one_launch"):       # that launch has re-selected already
+                cache.recompress_layers(0, n_layers)
+            for layer in sample_layers:
+                gi = cache.get_indices(layer)
+                for (l, s, h) in sample:
+                    if l == layer and labels[l][h]:
+                        st = gi[s, h, L:L + M]
+                        gpu_sets[(l, s, h, t)] = sorted((st[st >= 0] - L).tolist())
+    assert cache.device_status() == 0
+    t_end = n0 + n_steps
+    n_resel, n_band = [0], [0]
+
+    def chooser(key):
+        def choose(t, cand, sc, keep):
+            n_resel[0] += 1
+            got, want = gpu_sets[key + (t,)], [cand[i] for i in keep]
+            if got == want:
+                return keep
+            n_band[0] += 1
+            kth = np.sort(sc)[::-1][len(keep) - 1]
+            sure_in = {cand[i] for i in np.nonzero(sc > kth * (1 + BAND))[0]}
+            band = {cand[i] for i in np.nonzero(np.abs(sc - kth) <= BAND * abs(kth))[0]}
+            assert sure_in <= set(got) <= (sure_in | band) and len(got) == len(want), key
+            return [cand.index(j) for j in got]
+        return choose
+
+    for key, (qu, ku, vu) in picked.items():
+        l, s, h = key
+        got = torch.stack(outs[key]).float().cpu().numpy().astype(np.float64)
+        if labels[l][h]:
+            want, _ = oracle.rowbuf_semantic(qu, ku, vu, L, n0, M, R, t_end, choose=chooser(key))
+        else:
+            want = np.stack([oracle.attend(qu[t - 1], ku, vu, oracle.retained_set(False, L, t, W, R))
+                             for t in range(n0 + 1, t_end + 1)])
+        err = np.abs(got - want)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3, (key, err.max(), err.mean())
+    cache.close()
+    print(f"{cfg.name} {form}: {n_resel[0]} re-selections replayed, {n_band[0]} of them decided inside the tie band")
+    return n_resel[0], n_band[0]
+
+
+def _sample_of(cfg, layers, n_seqs, n_per_layer, seed):
+    rng = np.random.default_rng(seed)
+    sample = []
+    for layer in layers:
+        labels = wl.sink_mask(cfg, layer)
+        for i in range(n_per_layer):
+            heads = np.nonzero(labels == (1 if i % 3 else 0))[0]     # two semantic heads for every spatial one
+            sample.append((layer, int(rng.integers(0, n_seqs)), int(rng.choice(heads))))
+    return sorted(set(sample))
+
+
+@pytest.mark.parametrize("form", ["per_layer", "one_launch"])
+def test_rowbuf_janus7b_launch_size_sampled_pairs(form):
+    """Algorithm 2 at the sizes the benchmark times: 30 layers x 64 sequences x 32 heads, one full buffer
+    cycle and two steps of the next, ten sampled pairs against the oracle."""
+    cfg = wl.CONFIGS["janus7b"]
+    sample = _sample_of(cfg, (0, 7, 14, 22, 29), cfg.n_seqs, 3, seed=3)
+    assert len(sample) >= 8
+    n_resel, n_band = _run_full_launch_sampled(cfg, cfg.n_layers, list(range(cfg.n_seqs)), sample,
+                                               cfg.sink_recent + 2, form)
+    assert n_resel >= 8 and 0 <= n_band <= n_resel
+
+
+@pytest.mark.parametrize("form", ["per_layer", "one_launch"])
+def test_evict_every_step_janus7b_launch_size_sampled_pairs(form):
+    """Algorithm 1 taken literally (a re-selection after every step) at the benchmark's sizes, ten steps."""
+    cfg = wl.CONFIGS["janus7b"]
+    sample = _sample_of(cfg, (0, 11, 19, 29), cfg.n_seqs, 3, seed=4)
+    assert len(sample) >= 8
+    n_resel, n_band = _run_full_launch_sampled(cfg, cfg.n_layers, list(range(cfg.n_seqs)), sample, 10, form, evict=True)
+    assert n_resel >= 60 and 0 <= n_band <= n_resel
+
+
+@pytest.mark.parametrize("form", ["per_layer", "one_launch"])
+def test_rowbuf_hires7b_slice(form):
+    """The 4096-token grid (M + R = 320 entries per score row): two layers, four sequences, a full buffer
+    cycle of 64 steps and three more; four sampled pairs."""
+    cfg = wl.CONFIGS["hires7b"]
+    sample = _sample_of(cfg, (0, 1), 4, 2, seed=5)
+    n_resel, n_band = _run_full_launch_sampled(cfg, 2, [0, 1, 2, 3], sample, cfg.sink_recent + 3, form)
+    assert n_resel >= 2 and 0 <= n_band <= n_resel
