@@ -548,6 +548,25 @@ def run_ours(args, cfg):
         del ecache, esteps, est
         torch.cuda.empty_cache()
 
+    # ---- analysis utility (Sec. 3.2, MSE_token): per-token divergence of two uncompressed caches of one layer
+    analysis = None
+    if rank == 0 and world == 1:
+        g = torch.Generator(device=device).manual_seed(1)
+        shape = (S, H, cfg.prompt_len + N, 128)
+        t4 = [torch.randn(shape, generator=g, device=device).to(torch.bfloat16) for _ in range(4)]
+        mo = torch.empty(shape[:-1], dtype=torch.float32, device=device)
+        mse = lambda: B.kv_token_mse(*t4, out=mo)
+        for _ in range(3):
+            mse()
+        ms_m = timed(mse, 20, barrier) / 20
+        mbytes = mo.numel() * (4 * 256 + 4)
+        analysis = {"kernel": "ssd_kv_token_mse_kernel", "rows": mo.numel(), "ms": ms_m,
+                    "roofline": {"bound": "hbm", "achieved": mbytes / (ms_m * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                                 "frac": mbytes / (ms_m * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
+                                 "bytes_per_launch": mbytes, "traffic": None}}
+        del t4, mo
+        torch.cuda.empty_cache()
+
     # ---- CPU oracle on the host cores (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -582,7 +601,7 @@ def run_ours(args, cfg):
             "one_launch": one_launch,
             "one_time": setup_times,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf,
+            "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf, "analysis": analysis,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -247,6 +247,17 @@ int ssd_cache_get_compress_scores(ssd_cache *cache, int32_t layer, float *score_
  * cache's status word like those of ssd_decode_attn. */
 int ssd_decode_attn_static(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
+/* Per-token divergence of two KV caches (Sec. 3.2, the MSE_token equation; the paper compares the cache of
+ * the guided branch with that of the native branch of one prompt, position by position):
+ *   mse_out[r] = ||k_a[r] - k_b[r]||^2 + ||v_a[r] - v_b[r]||^2,  r = 0 .. n_rows-1
+ * where a row is one token of one head: k_a, v_a, k_b, v_b [n_rows, head_dim = 128] bf16 on the device,
+ * dense, 16-byte aligned (any leading shape, e.g. [n_seqs, n_heads, tokens], flattened); mse_out [n_rows]
+ * float on the device.  The sum is as printed: no division by head_dim.  fp32 arithmetic on the exactly
+ * widened inputs.  Needs no cache.  SSD_ERR_INVALID_ARG on null or misaligned pointers or n_rows < 0;
+ * n_rows = 0 does nothing.  Asynchronous. */
+int ssd_kv_token_mse(const void *k_a, const void *v_a, const void *k_b, const void *v_b, int64_t n_rows,
+                     float *mse_out, void *stream);
+
 /* One decode step of one layer from HOST buffers (pinned memory recommended): copies q, k_new and
  * v_new to the device, appends, attends, and copies the output back, all enqueued on `stream`.
  *   q_host, k_new_host, v_new_host, out_host [n_seqs, n_heads, head_dim] bf16 on the host

@@ -31,7 +31,7 @@ EXPORTS = [
     "ssd_cache_kv_bytes", "ssd_kernel_launch_count", "ssd_profile_enable", "ssd_profile_collect",
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
-    "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity", "ssd_cache_get_compress_scores",
+    "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity", "ssd_cache_get_compress_scores", "ssd_kv_token_mse",
 ]
 
 
@@ -85,6 +85,7 @@ def load():
     L.ssd_recompress.argtypes = [vp, i32, vp]
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_cache_get_compress_scores.argtypes = [vp, i32, vp]
+    L.ssd_kv_token_mse.argtypes = [vp, vp, vp, vp, C.c_int64, vp, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_append_decode_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_recompress_layers.argtypes = [vp, i32, i32, vp]
@@ -152,6 +153,26 @@ def labels_from_sparsity(s, tau: float):
     if rc != SSD_OK:
         raise SsdError(rc, "ssd_labels_from_sparsity")
     return lab
+
+
+def kv_token_mse(k_a: torch.Tensor, v_a: torch.Tensor, k_b: torch.Tensor, v_b: torch.Tensor,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Per-token divergence of two KV caches (Sec. 3.2): tensors [..., 128] bf16 on one CUDA device, all
+    of one shape; returns float32 [...] on that device."""
+    shape = tuple(k_a.shape)
+    for t in (k_a, v_a, k_b, v_b):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and tuple(t.shape) == shape and shape[-1] == 128):
+            raise ValueError("kv_token_mse: want four contiguous CUDA bf16 tensors [..., 128] of one shape")
+    if out is None:
+        out = torch.empty(shape[:-1], dtype=torch.float32, device=k_a.device)
+    n_rows = k_a.numel() // 128
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() == n_rows
+    with torch.cuda.device(k_a.device):
+        rc = load().ssd_kv_token_mse(k_a.data_ptr(), v_a.data_ptr(), k_b.data_ptr(), v_b.data_ptr(), n_rows,
+                                     out.data_ptr(), _stream())
+    if rc != SSD_OK:
+        raise SsdError(rc, "ssd_kv_token_mse")
+    return out
 
 
 def required_bytes(cfg: SsdConfig, n_sink_heads_total: int = -1) -> int:
