@@ -235,6 +235,15 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
                 cache.append(layer, k[:, :, L + j].contiguous(), v[:, :, L + j].contiguous())
         else:
             args_c = (q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous())
+            if layer == 0:
+                # the same call without observed queries does everything but the scoring (scores all zero):
+                # the difference to the full call is the scoring kernel's time
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+                cache.compress(layer, None, args_c[1], args_c[2], n0, 0)
+                ev[0].record()
+                cache.compress(layer, None, args_c[1], args_c[2], n0, 0)
+                ev[1].record()
+                noscore_events = ev
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             cache.compress(layer, *args_c, n0)          # score (tcgen05), select, gather
@@ -250,9 +259,48 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
         ms_c = [a.elapsed_time(b) for a, b in comp_events]
         setup["compress_ms_per_layer_median"] = float(np.median(ms_c))
         setup["compress_ms_all_layers"] = float(np.sum(ms_c))
+        setup.update(one_time_rooflines(cfg, S, float(np.median(ms_c)), noscore_events[0].elapsed_time(noscore_events[1])))
     cache.step_all = step_all
     cache.setup_times = setup
     return cache, steps_in
+
+
+def one_time_rooflines(cfg, S, compress_ms, noscore_ms):
+    """Rooflines of the one-time kernels of ssd_compress on one layer: the scoring contraction (tcgen05;
+    flops after causal skipping, i.e. of the 128 x 128 tiles it computes, in both sweeps) against the bf16
+    peak, and select + gather as a copy against the HBM peak."""
+    L, n0, H = cfg.prompt_len, cfg.n0, cfg.n_heads
+    tiles = 0
+    for r0 in range(0, n0, 128):
+        ctx = L + min(r0 + 128, n0)
+        tiles += -(-ctx // 128) + -(-(ctx - (L // 128) * 128) // 128)
+    pairs = S * cfg.n_sink_heads
+    flops = tiles * 2 * 128 ** 3 * pairs
+    exps = tiles * 128 * 128 * pairs
+    score_ms = max(compress_ms - noscore_ms, 1e-6)
+    tf_peak = 1620.8
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            tf_peak = float(json.load(f)["bf16_tflops"])
+    except Exception:
+        pass
+    sms, mhz = 148, 1965.0
+    exp_peak = 16 * sms * mhz * 1e6            # 16 special-function results per clock and SM
+    n_sp = H - cfg.n_sink_heads
+    slots = n_sp * (L + min(cfg.window, n0)) + cfg.n_sink_heads * (L + min(cfg.sink_budget, max(n0 - cfg.sink_recent, 0)) + min(cfg.sink_recent, n0))
+    gbytes = S * slots * 512 * 2
+    hbm, kind = measured_peaks()
+    return {"score": {"kernel": "ssd_score_kernel (tcgen05)", "ms_per_layer": score_ms, "tiles_per_pair": tiles,
+                      "roofline": {"bound": "tensor", "achieved": flops / (score_ms * 1e-3) / 1e12, "peak": tf_peak,
+                                   "unit": "TFLOP/s", "frac": flops / (score_ms * 1e-3) / 1e12 / tf_peak,
+                                   "peak_kind": f"of {kind} (burst)", "traffic": None,
+                                   "co_limit": {"what": "exponentials (special-function unit), one per logit and sweep",
+                                                "achieved_per_s": exps / (score_ms * 1e-3), "peak_per_s": exp_peak,
+                                                "frac": exps / (score_ms * 1e-3) / exp_peak}}},
+            "select_gather": {"kernels": "memset + ssd_select_kernel + ssd_gather_kernel", "ms_per_layer": noscore_ms,
+                              "roofline": {"bound": "hbm", "achieved": gbytes / (noscore_ms * 1e-3) / 1e9, "peak": hbm,
+                                           "unit": "GB/s", "frac": gbytes / (noscore_ms * 1e-3) / 1e9 / hbm,
+                                           "peak_kind": f"of {kind}", "bytes_per_layer": gbytes, "traffic": None}}}
 
 
 class Stepper:

@@ -134,10 +134,9 @@ int ssd_set_head_labels(ssd_cache *cache, const uint8_t *labels_host);
  * Spatial heads: keep the W newest tokens.  Every head keeps the whole prompt.
  * 0 <= n0 <= max_image_tokens; 0 <= n_obs <= n0 (q_obs may be NULL when n_obs == 0 or the layer
  * has no semantic head).  Replaces the layer's previous contents.  Asynchronous.
- * SSD_ERR_LIMIT if scores are needed (a semantic head, n_obs > 0) and n0 > 7808: a pair's score rows
- * are kept in shared memory beside the operand tiles.  Should a bounded wait of the scoring kernel
- * run out, the scores of that pair are written as zeros and bit 2 of the device status word is set
- * (ssd_cache_device_status): check it after compressing when the selection matters. */
+ * Should a bounded wait of the scoring kernel run out, the scores of that pair are incomplete and bit 2
+ * of the device status word is set (ssd_cache_device_status): check it after compressing when the
+ * selection matters. */
 int ssd_compress(ssd_cache *cache, int32_t layer, const void *q_obs, const void *k_full,
                  const void *v_full, int32_t n0, int32_t n_obs, void *stream);
 
@@ -320,8 +319,8 @@ int ssd_profile_collect(ssd_cache *cache, float *ms_host, int32_t *n_out);
  *              result; the outputs of that launch are incomplete;
  *   bit 1 (2): the classifier (ssd_classify_heads / ssd_classify_partial) gave up; its sparsity values
  *              are incomplete;
- *   bit 2 (4): the scoring kernel of ssd_compress gave up; the scores of the affected pairs are zero,
- *              so their top-M is the M lowest candidates.
+ *   bit 2 (4): the scoring kernel of ssd_compress gave up; the scores of the affected pairs are
+ *              incomplete, and so is the selection made from them.
  * The bits are sticky until the cache is recreated.  The kernels never trap and never spin without a
  * limit, so the CUDA context stays usable.  Synchronises the device.  No paper counterpart. */
 int ssd_cache_device_status(ssd_cache *cache, uint32_t *status_host);

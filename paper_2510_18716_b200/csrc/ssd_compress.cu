@@ -50,7 +50,22 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
   const int head = pair % p.H;
   if (!p.desc[head].w) return;
   const int tid = threadIdx.x;
-  const uint32_t* sc = reinterpret_cast<const uint32_t*>(p.score + (size_t)pair * p.n0);
+  // the score row arrives in 4 * n_parts pieces (one per lane quadrant of every thread block that shared the
+  // pair's query blocks): add them in a fixed order, so the row is reproducible bit for bit
+  float* row = p.score + (size_t)pair * kScoreQuads * p.n0;
+  {
+    const size_t stride = (size_t)gridDim.x * kScoreQuads * p.n0;
+    for (int i = tid; i < p.n0; i += kThreads) {
+      float s = 0.f;
+      for (int part = 0; part < p.n_parts; ++part) {
+        const float* r = row + (size_t)part * stride + i;
+        s += (r[0] + r[p.n0]) + (r[2 * (size_t)p.n0] + r[3 * (size_t)p.n0]);
+      }
+      row[i] = s;
+    }
+    __syncthreads();
+  }
+  const uint32_t* sc = reinterpret_cast<const uint32_t*>(row);
   int32_t* out = p.static_idx + (size_t)pair * p.M;
   const int n = p.n_cand;
   const int k = min(p.M, n);

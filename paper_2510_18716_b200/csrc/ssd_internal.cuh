@@ -127,14 +127,18 @@ struct ScoreParams {
   const __nv_bfloat16* q_obs;  // [n_seqs, H, n_obs, 128]
   const __nv_bfloat16* k_full; // [n_seqs, H, L + n0, 128]
   const HeadDesc* desc;
-  float* score;                // [n_seqs, H, n0]
+  float* score;                // [n_parts][n_seqs, H][4][n0], zero at launch: row (part, pair, quadrant) gets the
+                               // sums over the query rows of that lane quadrant in the query blocks of that part
   uint32_t* status;            // device status word (bit 2: a bounded wait of the scoring ran out)
   int n_seqs, H, L, n0, n_obs;
+  int n_parts;                 // thread blocks that share the query blocks of one (sequence, head)
   float scale_log2;
 };
 
 struct SelectParams {
-  const float* score;          // [n_seqs, H, n0]
+  float* score;                // [n_parts][n_seqs, H][4][n0]; a pair's 4 * n_parts rows are first added, in a
+                               // fixed order, into its row (part 0, quadrant 0), which is the pair's score row
+  int n_parts;
   const HeadDesc* desc;
   int32_t* static_idx;         // [n_seqs, H, M]
   float* acc;                  // row-buffer mode: [n_seqs * H, mr], gets the selected tokens' scores; else null
@@ -161,7 +165,9 @@ int decode_layers_max_mr();
 cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
-int score_max_n0();   // most image tokens whose score rows fit beside the scoring kernel's tiles in shared memory
+constexpr int kScoreMaxParts = 4;
+constexpr int kScoreQuads = 4;   // score rows a scoring thread block keeps per pair: one per TMEM lane quadrant
+int score_parts(int n_sem_pairs, int n_obs);   // thread blocks per (sequence, head) the scoring kernel should use
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
 struct RecompressParams {
   uint4* slab;

@@ -10,8 +10,9 @@
 // block of 128 observed queries, a first sweep over the key tiles gives every row its maximum and
 // exp-sum, a second sweep recomputes the tiles, normalises, and adds the columns up.  The sum over
 // the 32 rows of a warp is a shuffle transpose-reduction; each TMEM lane quadrant keeps its own
-// score array in shared memory and the four are added in a fixed order at the end, so scores are
-// bitwise reproducible from run to run, which the selection relies on.
+// score row in global memory (it stays in L2; every element belongs to one lane of one warp, which
+// adds to it with reductions that return nothing), and the selection adds the rows in a fixed order,
+// so scores are bitwise reproducible from run to run, which it relies on.
 //
 // A CTA is a pipeline of three roles that meet only at mbarriers:
 //   warp 0, one lane   producer: TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the query tile
@@ -473,7 +474,16 @@ __device__ __forceinline__ ScoreBlock score_block(const ScoreParams& p, int r0) 
   return b;
 }
 
-// One CTA per (sequence, semantic head); loops over blocks of 128 observed queries.
+// Which of n_parts thread blocks takes query block b of a pair: dealt back and forth (0, 1, .., P-1, P-1, ..,
+// 1, 0, 0, ..), so that every part gets short and long contexts alike.
+__device__ __forceinline__ int block_owner(int b, int n_parts) {
+  const int r = b % n_parts;
+  return ((b / n_parts) & 1) ? n_parts - 1 - r : r;
+}
+
+// n_parts CTAs per (sequence, semantic head), each looping over its blocks of 128 observed queries; a
+// part writes its own score row (zeros where it had nothing to add), and the selection adds the parts up
+// in a fixed order.
 __global__ void __launch_bounds__(kTcThreads, 2)
 ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, const __grid_constant__ CUtensorMap tk) {
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -481,7 +491,10 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float s_half[2][2][2][kRows];   // [block parity][column half][m, exp-sum][row]: sweep-1 statistics
-  const int pair = blockIdx.x;
+  const int n_pairs = p.n_seqs * p.H;
+  // the parts of a pair are neighbours in launch order, so they run at the same time and find each other's
+  // key tiles in L2
+  const int pair = blockIdx.x / p.n_parts, part = blockIdx.x % p.n_parts;
   const int head = pair % p.H;
   if (!p.desc[head].w) return;            // before any tensor-memory allocation
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -490,14 +503,13 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   Pipe pipe;
   const uint32_t q_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe), k_s = q_s + kTileBytes;
   const uint32_t tmem = s_tmem;
-  // [4 lane quadrants][n0], behind the tiles
-  float* s_score = reinterpret_cast<float*>(smem + (q_s - smem_u32(smem)) + (1 + kStages) * kTileBytes);
 
   if (warp == 0) {
     if (lane == 0) {
       Producer pr;
       pr.p = pipe; pr.abort = &s_abort; pr.q_s = q_s; pr.k_s = k_s; pr.tq = &tq; pr.tk = &tk;
       for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
+        if (block_owner(r0 / kRows, p.n_parts) != part) continue;
         const ScoreBlock b = score_block(p, r0);
         pr.query_block(r0, pair);
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) pr.key_tile(k0, pair);
@@ -510,6 +522,7 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
       Issuer is;
       is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem;
       for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
+        if (block_owner(r0 / kRows, p.n_parts) != part) continue;
         const ScoreBlock b = score_block(p, r0);
         is.query_block();
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
@@ -522,11 +535,12 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
     const int rl = quad * 32 + lane;                     // row inside a block of queries
     Consumer co;
     co.p = pipe; co.abort = &s_abort; co.tmem_lane = tmem + ((uint32_t)(quad * 32) << 16); co.lane = lane;
-    float* my_score = s_score + (size_t)quad * p.n0;     // the two warps of a quadrant write disjoint keys
-    for (int j = tid - 64; j < 4 * p.n0; j += kEpiThreads) s_score[j] = 0.f;   // ordered before its use by the barrier below
+    // this quadrant's score row; the two warps of a quadrant own disjoint keys, a key always the same lane
+    float* my_score = p.score + ((((size_t)part * n_pairs + pair) * kScoreQuads) + quad) * p.n0;
 
-    int blk = 0;
-    for (int r0 = 0; r0 < p.n_obs; r0 += kRows, ++blk) {
+    int blk = 0;                           // blocks this part has done
+    for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
+      if (block_owner(r0 / kRows, p.n_parts) != part) continue;
       const ScoreBlock b = score_block(p, r0);
       const int row = r0 + rl;
       const int ctx_r = row < p.n_obs ? p.L + t_first + row : 0;          // keys [0, ctx_r) are visible
@@ -597,19 +611,18 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
           }
           const float col = warp_column_sums(v, lane);
           const int key = base + lane;
-          if (key >= p.L && key < b.ctx_max) my_score[key - p.L] += col;
+          // an addition that returns nothing, so nothing waits for it; this lane is the only one that ever
+          // adds to this element, and its additions arrive in program order: the sum is reproducible
+          if (key >= p.L && key < b.ctx_max) atomicAdd(my_score + (key - p.L), col);
         }
         if (!released) co.release();
       }
+      ++blk;
     }
   }
 
   __syncthreads();
-  const bool ok = s_abort == 0;
-  float* out = p.score + (size_t)pair * p.n0;
-  for (int j = tid; j < p.n0; j += kTcThreads)
-    out[j] = ok ? (s_score[j] + s_score[p.n0 + j]) + (s_score[2 * p.n0 + j] + s_score[3 * p.n0 + j]) : 0.f;
-  if (tid == 0 && !ok) atomicOr(p.status, 4u);
+  if (tid == 0 && s_abort != 0) atomicOr(p.status, 4u);    // the pair's rows are incomplete
   cta_teardown(tmem);
 }
 
@@ -662,19 +675,40 @@ cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStrea
   return cudaGetLastError();
 }
 
-// a pair's four score rows (one per lane quadrant) sit beside the tiles; 8 KB stay free for the static arrays
-int score_max_n0() { return (int)((227 * 1024 - 8192 - 1024 - (1 + kStages) * (size_t)kTileBytes) / (4 * sizeof(float))); }
+// Two scoring CTAs fit an SM.  With P parts per pair the launch needs ceil(pairs * P / slots) rounds of CTAs,
+// each 1/P of a pair's work long: take the P that makes that product smallest (the smaller P on ties), as
+// long as every part still gets at least two query blocks.
+int score_parts(int n_sem_pairs, int n_obs) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    sms = 148;
+  }
+  const long slots = 2L * sms;
+  const int n_blocks = (n_obs + kRows - 1) / kRows;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int parts = 1; parts <= kScoreMaxParts && 2 * parts <= (n_blocks > 2 ? n_blocks : 2); ++parts) {
+    const long rounds = ((long)n_sem_pairs * parts + slots - 1) / slots;
+    const double cost = (double)rounds / parts;
+    if (cost < best_cost * (1.0 - 1e-9)) {
+      best_cost = cost;
+      best = parts;
+    }
+  }
+  return best;
+}
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
-  const size_t smem = (1 + kStages) * (size_t)kTileBytes + 4 * (size_t)p.n0 * sizeof(float) + 1024;
-  if (p.n0 > score_max_n0()) return cudaErrorInvalidValue;
+  const size_t smem = (1 + kStages) * (size_t)kTileBytes + 1024;
   CUtensorMap tq, tk;
   const uint64_t pairs = (uint64_t)p.n_seqs * p.H;
   cudaError_t e = make_tile_map(&tq, p.q_obs, (uint64_t)p.n_obs, pairs);
   if (e == cudaSuccess) e = make_tile_map(&tk, p.k_full, (uint64_t)p.L + p.n0, pairs);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(ssd_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  ssd_score_kernel<<<p.n_seqs * p.H, kTcThreads, smem, st>>>(p, tq, tk);
+  if (p.n_parts < 1 || p.n_parts > kScoreMaxParts) return cudaErrorInvalidValue;
+  ssd_score_kernel<<<p.n_seqs * p.H * p.n_parts, kTcThreads, smem, st>>>(p, tq, tk);
   count_launch();
   return cudaGetLastError();
 }

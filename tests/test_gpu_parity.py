@@ -373,6 +373,9 @@ def test_compress_scores_elementwise(name, layer, n_seqs):
     cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
     got = cache.get_compress_scores(0, n0)
     assert cache.device_status() == 0
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+    assert np.array_equal(got, cache.get_compress_scores(0, n0)), "scores must be reproducible bit for bit"
+
     sem = labels[None, :].repeat(n_seqs, 0).astype(np.uint8)
     want, _, _ = oracle.select_batch(wl.to_u16(q[:, :, :n0]), wl.to_u16(k[:, :, : L + n0]), sem, L, n0, M, R)
     for h in range(H):
