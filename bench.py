@@ -36,8 +36,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.39e6, "per_layer_of_step": 160.84e6,
-                  "sha256": "897dd95c647319ed9b92ff857ce2835f7195184c50e275e7842b45dbdb885b7a"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.26e6, "per_layer_of_step": 160.89e6,
+                  "sha256": "8ae52eb6b67ee40171d816382324d6a8221d36a9c956d2adab099f68e092f47c"}
 
 
 def decode_traffic(cfg):
