@@ -241,6 +241,73 @@ def kv_token_mse(K_a, V_a, K_b, V_b):
     return (dk * dk).sum(-1) + (dv * dv).sum(-1)
 
 
+# ---- 8-bit K/V (an extension the paper only cites as related work, Sec. 2 "KV Cache Compression")
+# Format: OCP 8-bit floating point, E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no
+# infinities, S.1111.111 is NaN, largest finite magnitude 448, subnormals 2^-6 * m/8).
+
+def e4m3_decode(codes):
+    """E4M3 bit patterns (uint8) -> float64, from the format's definition."""
+    c = np.asarray(codes, np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = c & 0x7
+    mag = np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return sign * mag
+
+
+def e4m3_encode(x):
+    """float32 values -> E4M3 bit patterns: the nearest finite value, ties to the even bit pattern, magnitudes
+    beyond 448 to 448 (round to nearest even, saturating).  Written as a search over the 127 finite
+    magnitudes, not as bit manipulation."""
+    x = np.asarray(x, np.float32)
+    table = e4m3_decode(np.arange(127, dtype=np.uint8))          # ascending magnitudes, code = index
+    a = np.abs(x.astype(np.float64)).reshape(-1)
+    out = np.empty(a.shape, np.uint8)
+    for i, v in enumerate(a):
+        if v >= table[-1]:
+            k = 126
+        else:
+            hi = int(np.searchsorted(table, v, side="left"))     # table[hi-1] < v <= table[hi]
+            lo = max(hi - 1, 0)
+            dl, dh = v - table[lo], table[hi] - v
+            k = hi if dh < dl else lo if dl < dh else (lo if lo % 2 == 0 else hi)
+        out[i] = k
+    out = out.reshape(x.shape)
+    return np.where(np.signbit(x), out | 0x80, out).astype(np.uint8)
+
+
+def kv_quantize_rows(rows_u16):
+    """Per-row (one token of one head) 8-bit quantisation of K or V rows [..., D] (uint16 bf16):
+    scale = max|x| / 448 and code = E4M3(x / scale), both in float32 arithmetic (the precision in which the
+    library decides the codes); a row of zeros gets scale 0 and codes 0.  Returns (codes uint8 [..., D],
+    scale float32 [...])."""
+    x = (_u16(rows_u16).astype(np.uint32) << 16).view(np.float32)
+    amax = np.abs(x).max(axis=-1)
+    scale = (amax / np.float32(448.0)).astype(np.float32)
+    safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
+    y = (x / safe[..., None]).astype(np.float32)
+    return e4m3_encode(y), scale
+
+
+def kv_dequantize(codes, scale):
+    """codes [..., D] uint8, scale [...] float32 -> float64 values code * scale."""
+    return e4m3_decode(codes) * np.asarray(scale, np.float32).astype(np.float64)[..., None]
+
+
+def attend_values(q, K, V, pos, scale=None):
+    """softmax(scale * K[pos] q) V[pos] for a query q [D] (uint16 bf16) over float64 rows K, V [n, D]: the
+    attention of Sec. 3.1 over an explicit set of positions, for caches whose rows are not bf16."""
+    qv = _widen(q)
+    K, V = np.asarray(K, np.float64), np.asarray(V, np.float64)
+    pos = np.asarray(pos, np.int64)
+    sc = default_scale(qv.shape[-1]) if scale is None else scale
+    logits = (K[pos] @ qv) * sc
+    w = np.exp(logits - logits.max())
+    w = w / w.sum()
+    return w @ V[pos]
+
+
 class RowBufferOverflow(RuntimeError):
     """Algorithm 2: a token was appended to a row buffer that already holds R tokens."""
 

@@ -506,3 +506,70 @@ def test_kv_token_mse_pins():
         assert math.isclose(m[1, 0, j], acc, rel_tol=1e-12)
     assert np.array_equal(m, oracle.kv_token_mse(ub, uvb, ua, uva))
     assert (m > 0).all()
+
+
+def test_e4m3_decode_and_encode_pins():
+    """The 8-bit format of the quantised cache: the decode table against the library's float8_e4m3fn and the
+    format's closed form; encode against the library cast on in-range values, exact ties to the even bit
+    pattern, saturation at 448, every finite code a fixed point, monotonicity."""
+    codes = np.arange(256, dtype=np.uint8)
+    lib = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    got = oracle.e4m3_decode(codes)
+    assert np.array_equal(np.isnan(got), np.isnan(lib)) and np.isnan(got).sum() == 2
+    ok = ~np.isnan(got)
+    assert np.array_equal(got[ok], lib[ok])
+    assert got[0x7E] == 448.0 and got[0x01] == 2.0 ** -9 and got[0x08] == 2.0 ** -6 and got[0x38] == 1.0 and got[0xB8] == -1.0
+    finite = codes[ok]
+    assert np.array_equal(oracle.e4m3_encode(got[ok].astype(np.float32)) & 0x7F, finite & 0x7F)     # fixed points (+-0 aside)
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(0, 100, 4000), rng.normal(0, 1, 4000), rng.uniform(-448, 448, 4000),
+                        rng.normal(0, 0.01, 2000)]).astype(np.float32)
+    x = x[np.abs(x) <= 448]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(oracle.e4m3_encode(x), want)
+    # midpoints of neighbouring magnitudes go to the even bit pattern
+    mags = got[:127]
+    mid = ((mags[:-1] + mags[1:]) / 2).astype(np.float32)
+    assert np.array_equal(mid.astype(np.float64), (mags[:-1] + mags[1:]) / 2)                     # exact in float32
+    enc = oracle.e4m3_encode(mid)
+    assert np.array_equal(enc, np.where(np.arange(126) % 2 == 0, np.arange(126), np.arange(1, 127)).astype(np.uint8))
+    assert np.array_equal(oracle.e4m3_encode(np.array([449, 480, 1e6, -1e9], np.float32)), np.array([0x7E, 0x7E, 0x7E, 0xFE], np.uint8))
+    xs = np.sort(x)
+    assert (np.diff(oracle.e4m3_decode(oracle.e4m3_encode(xs))) >= 0).all()
+
+
+def test_kv_quantize_rows_pins():
+    """Per-row scale = max|x| / 448: the largest element is reproduced (up to float32 rounding of the scale),
+    every element within half a step of its binade (relative error <= 2^-4 for normal codes, absolute
+    <= scale * 2^-10 below), zero rows stay zero, and scaling a row by a power of two scales the scale only."""
+    g = torch.Generator().manual_seed(3)
+    rows = (torch.randn((5, 7, 128), generator=g) * torch.logspace(-3, 2, 7)[None, :, None]).to(torch.bfloat16)
+    rows[2, 3] = 0
+    u = wl.to_u16(rows)
+    codes, scale = oracle.kv_quantize_rows(u)
+    assert codes.shape == (5, 7, 128) and scale.shape == (5, 7) and codes.dtype == np.uint8 and scale.dtype == np.float32
+    x = rows.double().numpy()
+    dq = oracle.kv_dequantize(codes, scale)
+    amax = np.abs(x).max(-1)
+    assert np.allclose(np.abs(dq).max(-1), amax, rtol=1e-6) and np.array_equal(scale, (amax.astype(np.float32) / np.float32(448)))
+    err = np.abs(dq - x)
+    assert (err <= np.maximum(np.abs(x) * 2.0 ** -4, scale[..., None].astype(np.float64) * 2.0 ** -10) * (1 + 1e-6)).all()
+    assert (codes[2, 3] == 0).all() and scale[2, 3] == 0 and (dq[2, 3] == 0).all()
+    c2, s2 = oracle.kv_quantize_rows(wl.to_u16((rows * 4).to(torch.bfloat16)))
+    assert np.array_equal(c2, codes) and np.array_equal(s2, scale * np.float32(4))
+
+
+def test_attend_values_equals_attend_on_bf16_rows():
+    """attend_values on exactly widened bf16 rows is the attention the C routine computes (and, through its own
+    pin, the library's masked SDPA)."""
+    g = torch.Generator().manual_seed(5)
+    q, K, V = (torch.randn(s, generator=g).to(torch.bfloat16) for s in ((128,), (40, 128), (40, 128)))
+    pos = np.array([0, 1, 2, 7, 9, 30, 39], np.int32)
+    a = oracle.attend(wl.to_u16(q), wl.to_u16(K), wl.to_u16(V), pos)
+    b = oracle.attend_values(wl.to_u16(q), K.double().numpy(), V.double().numpy(), pos)
+    assert np.allclose(a, b, rtol=1e-12, atol=1e-14)
+    # the quantised cache changes the result by the quantisation error only: a few percent of |V|
+    ck, sk = oracle.kv_quantize_rows(wl.to_u16(K))
+    cv, sv = oracle.kv_quantize_rows(wl.to_u16(V))
+    c = oracle.attend_values(wl.to_u16(q), oracle.kv_dequantize(ck, sk), oracle.kv_dequantize(cv, sv), pos)
+    assert 0 < np.abs(c - a).max() < 0.1
