@@ -246,6 +246,24 @@ int ssd_cache_get_compress_scores(ssd_cache *cache, int32_t layer, float *score_
  * cache's status word like those of ssd_decode_attn. */
 int ssd_decode_attn_static(ssd_cache *cache, int32_t layer, const void *q, void *out, void *stream);
 
+/* 8-bit K/V.  The paper does not quantise; it cites quantisation as the orthogonal line of work (Sec. 2, "KV
+ * Cache Compression").  This is that extension on the same head-decoupled store: every cached row is held as
+ * 128 E4M3 codes (OCP 8-bit floating point: 4 exponent bits, bias 7, 3 mantissa bits, largest magnitude 448) and
+ * one float32 scale per row, scale = max|x| / 448, code = E4M3(x / scale) with round to nearest even, saturating,
+ * decided in float32 arithmetic; a slot is 272 bytes instead of 512.  A row is quantised once, when it enters the
+ * cache.  Attention runs in float32 on the exactly widened codes; the K row's scale multiplies the logit, the V
+ * row's the softmax weight.
+ *   ssd_cache_set_kv_format(cache, 1) switches a cache to that format (0 = bf16, the default) and resets every
+ *   layer to the empty state; call it before ssd_compress.  In that format the cache serves ssd_compress,
+ *   ssd_append_decode_layers, ssd_append_decode (the same kernel on one layer), ssd_step_host(_layers) and the
+ *   inspection calls; ssd_append, ssd_decode_attn, ssd_decode_attn_static and the row-buffer mode return
+ *   SSD_ERR_BAD_STATE (so does switching the format while the row buffer is on, and vice versa).  The device buffer
+ *   is sized as for bf16 (ssd_cache_required_bytes); ssd_cache_kv_bytes reports the bytes actually held.
+ *   ssd_quantize_rows_e4m3 is the quantiser on its own: rows [n_rows, 128] bf16 -> codes_out [n_rows, 128] uint8 and
+ *   scales_out [n_rows] float (all on the device; rows and codes_out 16-byte aligned).  Asynchronous. */
+int ssd_cache_set_kv_format(ssd_cache *cache, int32_t format);
+int ssd_quantize_rows_e4m3(const void *rows, int64_t n_rows, void *codes_out, float *scales_out, void *stream);
+
 /* Per-token divergence of two KV caches (Sec. 3.2, the MSE_token equation; the paper compares the cache of
  * the guided branch with that of the native branch of one prompt, position by position):
  *   mse_out[r] = ||k_a[r] - k_b[r]||^2 + ||v_a[r] - v_b[r]||^2,  r = 0 .. n_rows-1

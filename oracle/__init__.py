@@ -258,23 +258,18 @@ def e4m3_decode(codes):
 
 def e4m3_encode(x):
     """float32 values -> E4M3 bit patterns: the nearest finite value, ties to the even bit pattern, magnitudes
-    beyond 448 to 448 (round to nearest even, saturating).  Written as a search over the 127 finite
-    magnitudes, not as bit manipulation."""
+    beyond 448 to 448 (round to nearest even, saturating).  Written as a search over the table of the 127
+    finite magnitudes (the two neighbours of |x|, the nearer one, the even one on a tie), not as bit
+    manipulation."""
     x = np.asarray(x, np.float32)
     table = e4m3_decode(np.arange(127, dtype=np.uint8))          # ascending magnitudes, code = index
-    a = np.abs(x.astype(np.float64)).reshape(-1)
-    out = np.empty(a.shape, np.uint8)
-    for i, v in enumerate(a):
-        if v >= table[-1]:
-            k = 126
-        else:
-            hi = int(np.searchsorted(table, v, side="left"))     # table[hi-1] < v <= table[hi]
-            lo = max(hi - 1, 0)
-            dl, dh = v - table[lo], table[hi] - v
-            k = hi if dh < dl else lo if dl < dh else (lo if lo % 2 == 0 else hi)
-        out[i] = k
-    out = out.reshape(x.shape)
-    return np.where(np.signbit(x), out | 0x80, out).astype(np.uint8)
+    a = np.abs(x.astype(np.float64))
+    hi = np.minimum(np.searchsorted(table, a, side="left"), 126)  # table[hi-1] < a <= table[hi] (a below 448)
+    lo = np.maximum(hi - 1, 0)
+    dl, dh = a - table[lo], table[hi] - a
+    k = np.where(dh < dl, hi, np.where(dl < dh, lo, np.where(lo % 2 == 0, lo, hi)))   # ties: the even pattern
+    k = np.where(a >= table[-1], 126, k).astype(np.uint8)
+    return np.where(np.signbit(x), k | 0x80, k).astype(np.uint8)
 
 
 def kv_quantize_rows(rows_u16):

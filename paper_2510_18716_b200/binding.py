@@ -32,6 +32,7 @@ EXPORTS = [
     "ssd_cache_device_status", "ssd_debug_decode_plan", "ssd_decode_attn_static",
     "ssd_cache_set_row_buffer", "ssd_recompress", "ssd_cache_get_scores", "ssd_append_decode",
     "ssd_labels_from_ratio_sums", "ssd_labels_from_sparsity", "ssd_cache_get_compress_scores", "ssd_kv_token_mse",
+    "ssd_cache_set_kv_format", "ssd_quantize_rows_e4m3",
 ]
 
 
@@ -86,6 +87,8 @@ def load():
     L.ssd_cache_get_scores.argtypes = [vp, i32, vp]
     L.ssd_cache_get_compress_scores.argtypes = [vp, i32, vp]
     L.ssd_kv_token_mse.argtypes = [vp, vp, vp, vp, C.c_int64, vp, vp]
+    L.ssd_cache_set_kv_format.argtypes = [vp, i32]
+    L.ssd_quantize_rows_e4m3.argtypes = [vp, C.c_int64, vp, vp, vp]
     L.ssd_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.ssd_append_decode_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.ssd_recompress_layers.argtypes = [vp, i32, i32, vp]
@@ -173,6 +176,20 @@ def kv_token_mse(k_a: torch.Tensor, v_a: torch.Tensor, k_b: torch.Tensor, v_b: t
     if rc != SSD_OK:
         raise SsdError(rc, "ssd_kv_token_mse")
     return out
+
+
+def quantize_rows_e4m3(rows: torch.Tensor):
+    """The library's 8-bit row quantiser: rows [..., 128] bf16 on a CUDA device -> (codes uint8 [..., 128],
+    scales float32 [...])."""
+    if not (rows.is_cuda and rows.dtype == torch.bfloat16 and rows.is_contiguous() and rows.shape[-1] == 128):
+        raise ValueError("quantize_rows_e4m3: want a contiguous CUDA bf16 tensor [..., 128]")
+    codes = torch.empty(rows.shape, dtype=torch.uint8, device=rows.device)
+    scales = torch.empty(rows.shape[:-1], dtype=torch.float32, device=rows.device)
+    with torch.cuda.device(rows.device):
+        rc = load().ssd_quantize_rows_e4m3(rows.data_ptr(), rows.numel() // 128, codes.data_ptr(), scales.data_ptr(), _stream())
+    if rc != SSD_OK:
+        raise SsdError(rc, "ssd_quantize_rows_e4m3")
+    return codes, scales
 
 
 def required_bytes(cfg: SsdConfig, n_sink_heads_total: int = -1) -> int:
@@ -315,6 +332,10 @@ class SsdCache:
         self._check(self.lib.ssd_decode_attn_static(self._h, layer, _dev(q, shp, "q"), _dev(out, shp, "out"),
                                                     _stream()), "ssd_decode_attn_static")
         return out
+
+    def set_kv_format(self, fmt: int):
+        """0: bf16 rows (default); 1: 8-bit rows (E4M3 codes and a float32 scale per row)."""
+        self._check(self.lib.ssd_cache_set_kv_format(self._h, int(fmt)), "ssd_cache_set_kv_format")
 
     # -- Algorithm 2 (row buffer)
     def set_row_buffer(self, enable: bool = True):

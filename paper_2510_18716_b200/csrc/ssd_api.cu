@@ -130,7 +130,11 @@ struct ssd_cache {
   char* d_staging(int slot = 0) const {
     return base + reg.staging + (size_t)slot * kHostGroup * 4 * cfg.n_seqs * cfg.n_heads * kHeadDim * 2;
   }
-  uint4* d_slab(int layer) const { return reinterpret_cast<uint4*>(base + reg.slab) + (size_t)layer_base[layer] * kSlotU4; }
+  bool kv_q8 = false;                 // 8-bit K/V: slots of 272 bytes (E4M3 codes and row scales) instead of 512
+  int slot_bytes() const { return kv_q8 ? q8_slot_bytes() : kSlotBytes; }
+  uint4* d_slab(int layer) const {
+    return reinterpret_cast<uint4*>(base + reg.slab + (size_t)layer_base[layer] * slot_bytes());
+  }
   int max_slots() const {
     int a = cfg.window, b = cfg.sink_budget + cfg.sink_recent;
     return cfg.prompt_len + (a > b ? a : b);
@@ -480,7 +484,8 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   gp.n_seqs = g.n_seqs; gp.H = g.n_heads; gp.L = g.prompt_len; gp.M = g.sink_budget; gp.n0 = n0;
   gp.static_valid = select ? sv : 0;
   gp.seq_slots = c->seq_slots[layer];
-  if (launch_gather(gp, c->max_slots(), st) != cudaSuccess) return SSD_ERR_CUDA;
+  if ((c->kv_q8 ? launch_gather_q8(gp, c->max_slots(), st) : launch_gather(gp, c->max_slots(), st)) != cudaSuccess)
+    return SSD_ERR_CUDA;
   c->t_img[layer] = n0;
   c->n0[layer] = n0;
   c->prompt_valid[layer] = g.prompt_len;
@@ -497,7 +502,7 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
-  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (!c->labels_set || c->kv_q8) return SSD_ERR_BAD_STATE;   // 8-bit caches append inside the decode launch only
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
   if (c->row_buffer && c->n_sink[layer] > 0 && c->sem_tokens(layer) >= g.sink_recent)
     return SSD_ERR_OVERFLOW;            // Algorithm 2, overflow branch: call ssd_recompress first
@@ -528,7 +533,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (!c || !q || !out) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
-  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (!c->labels_set || c->kv_q8) return SSD_ERR_BAD_STATE;
   if (c->empty_head(layer, c->t_img[layer], c->sem_tokens(layer))) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   DecodeParams p;
@@ -575,6 +580,8 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
+  if (c->kv_q8)      // 8-bit K/V: the one kernel of that format, on one layer
+    return ssd_append_decode_layers(c, layer, 1, k_new, v_new, q, out, stream);
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
   const bool scored = c->row_buffer && c->n_sink[layer] > 0;
   if (scored && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;   // Algorithm 2, overflow branch
@@ -686,7 +693,8 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     ls.sem_slot = c->sem_tokens(layer);
     ls.t_sem = ls.sem_slot + 1;
   }
-  if (cudaMemsetAsync(p.work, 0, 4, st) != cudaSuccess || launch_decode_layers(p, st) != cudaSuccess) {
+  if (cudaMemsetAsync(p.work, 0, 4, st) != cudaSuccess ||
+      (c->kv_q8 ? launch_decode_layers_q8(p, st) : launch_decode_layers(p, st)) != cudaSuccess) {
     cudaGetLastError();
     return SSD_ERR_CUDA;
   }
@@ -871,12 +879,34 @@ int ssd_cache_kv_bytes(ssd_cache* c, size_t* bytes_per_seq) {
   if (!c->labels_set) return SSD_ERR_BAD_STATE;
   size_t slots = 0;
   for (int l = 0; l < c->cfg.n_layers; ++l) slots += (size_t)c->seq_slots[l];
-  *bytes_per_seq = slots * kSlotBytes;
+  *bytes_per_seq = slots * (size_t)c->slot_bytes();
   return SSD_OK;
+}
+
+int ssd_cache_set_kv_format(ssd_cache* c, int32_t format) {
+  if (!c || (format != 0 && format != 1)) return SSD_ERR_INVALID_ARG;
+  if (format == 1 && c->row_buffer) return SSD_ERR_BAD_STATE;
+  c->kv_q8 = format == 1;
+  for (int l = 0; l < c->cfg.n_layers; ++l) {
+    c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = c->t_base[l] = 0;
+    c->pending[l] = 0;
+  }
+  return SSD_OK;
+}
+
+int ssd_quantize_rows_e4m3(const void* rows, int64_t n_rows, void* codes_out, float* scales_out, void* stream) {
+  if (!rows || !codes_out || !scales_out || n_rows < 0 || n_rows > (int64_t)1 << 36) return SSD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(rows) | reinterpret_cast<uintptr_t>(codes_out)) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(scales_out) % 4 != 0)
+    return SSD_ERR_INVALID_ARG;
+  if (n_rows == 0) return SSD_OK;
+  return launch_quantize_rows(rows, n_rows, codes_out, scales_out, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? SSD_OK : SSD_ERR_CUDA;
 }
 
 int ssd_cache_set_row_buffer(ssd_cache* c, int32_t enable) {
   if (!c) return SSD_ERR_INVALID_ARG;
+  if (enable && c->kv_q8) return SSD_ERR_BAD_STATE;
   c->row_buffer = enable != 0;
   for (int l = 0; l < c->cfg.n_layers; ++l) {
     c->t_img[l] = c->n0[l] = c->prompt_valid[l] = c->static_valid[l] = c->t_base[l] = 0;
@@ -1093,7 +1123,7 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   if (!c || !q || !out) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
-  if (!c->labels_set) return SSD_ERR_BAD_STATE;
+  if (!c->labels_set || c->kv_q8) return SSD_ERR_BAD_STATE;
   if (c->empty_head(layer, c->t_img[layer], c->sem_tokens(layer))) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   const long pairs = (long)g.n_seqs * g.n_heads;

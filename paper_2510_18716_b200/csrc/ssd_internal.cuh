@@ -184,6 +184,11 @@ struct RecompressParams {
   int seq_slots;
 };
 cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st);
+// 8-bit K/V (slots of 272 bytes: 128 + 128 E4M3 codes and two float32 row scales)
+cudaError_t launch_quantize_rows(const void* rows, long long n_rows, void* codes, float* scales, cudaStream_t st);
+cudaError_t launch_gather_q8(const GatherParams& p, int max_slots, cudaStream_t st);
+cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st);
+int q8_slot_bytes();
 // The same for several layers in one launch: what differs from layer to layer, and the first layer's
 // tables (a layer's tables follow the previous layer's at fixed strides).
 struct RecompressLayer {

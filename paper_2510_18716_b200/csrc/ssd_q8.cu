@@ -1,0 +1,465 @@
+// 8-bit K/V: an extension the paper only cites as related work (Sec. 2, "KV Cache Compression").  The same
+// head-decoupled store, with every cached row held as 128 E4M3 codes (OCP 8-bit floating point: 4 exponent
+// bits, bias 7, 3 mantissa bits, largest magnitude 448) and one float32 scale per row,
+//   scale = max|x| / 448,   code = E4M3(x / scale)   (round to nearest even, saturating; float32 arithmetic),
+// so a slot is [K codes 128 B | V codes 128 B | K scale | V scale | 8 B unused] = 272 bytes instead of 512.
+// A row is quantised once, when it enters the cache (by the gather of ssd_compress, or by the decode launch
+// that appends it), so what later steps read does not depend on when they read it.
+//   ssd_quantize_rows_kernel   the quantiser on its own (parity of the codes, bit for bit)
+//   ssd_gather_q8_kernel       ssd_compress's gather, quantising on the way into the slab
+//   ssd_decode_layers_q8_kernel  fused append + decode attention of every layer in one launch: whole heads
+//                              handed out to warps from a counter, as in ssd_decode_layers_kernel; codes are
+//                              widened with cvt.rn.f16x2.e4m3x2 (exact), all arithmetic in float32, the row
+//                              scales applied to the logit and to the softmax weight
+#include <cuda_fp16.h>
+
+#include <atomic>
+
+#include "ssd_internal.cuh"
+#include "ssd_device.cuh"
+
+namespace ssd {
+
+namespace {
+
+constexpr int kQ8SlotBytes = 272;
+constexpr int kQ8SlotU4 = kQ8SlotBytes / 16;   // 17
+
+// two floats -> two E4M3 codes (a in the low byte)
+__device__ __forceinline__ uint32_t e4m3x2(float a, float b) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(b), "f"(a));
+  return r;
+}
+
+// 8 bf16 values of a row (one uint4) -> 8 codes (uint2), given the row's scale
+__device__ __forceinline__ uint2 quantize8(const uint4& raw, float scale) {
+  const float s = scale > 0.f ? scale : 1.f;
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  uint32_t c[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    c[i] = e4m3x2(__fdiv_rn(__uint_as_float(w[i] << 16), s), __fdiv_rn(__uint_as_float(w[i] & 0xffff0000u), s));
+  return make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
+}
+
+__device__ __forceinline__ float amax8(const uint4& raw) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    m = fmaxf(m, fmaxf(fabsf(__uint_as_float(w[i] << 16)), fabsf(__uint_as_float(w[i] & 0xffff0000u))));
+  return m;
+}
+
+// A row is held by 16 consecutive lanes (8 values each): its scale, the same in all 16 lanes.
+__device__ __forceinline__ float row_scale16(const uint4& raw) {
+  float m = amax8(raw);
+#pragma unroll
+  for (int o = 8; o >= 1; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  return __fdiv_rn(m, 448.f);
+}
+
+// ----------------------------------------------------------------------------- the quantiser on its own
+__global__ void __launch_bounds__(256) ssd_quantize_rows_kernel(const uint4* __restrict__ rows, long long n_rows,
+                                                                uint2* __restrict__ codes, float* __restrict__ scales) {
+  const long long hw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // one half-warp per row
+  const int l16 = threadIdx.x & 15;
+  const bool ok = hw < n_rows;
+  const uint4 raw = ok ? rows[hw * 16 + l16] : make_uint4(0, 0, 0, 0);
+  const float scale = row_scale16(raw);
+  if (!ok) return;
+  codes[hw * 16 + l16] = quantize8(raw, scale);
+  if (l16 == 0) scales[hw] = scale;
+}
+
+// ----------------------------------------------------------------------------- gather into 272-byte slots
+// One warp per destination slot: lanes 0-15 quantise the K row, lanes 16-31 the V row.
+__global__ void __launch_bounds__(256) ssd_gather_q8_kernel(const GatherParams p, int max_slots) {
+  const int pair = blockIdx.x;
+  const int seq = pair / p.H, head = pair - seq * p.H;
+  const HeadDesc d = p.desc[head];
+  const int cap = p.L + d.y + d.z;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int ctx = p.L + p.n0;
+  unsigned char* dst0 = reinterpret_cast<unsigned char*>(p.slab) + ((size_t)seq * p.seq_slots + d.x) * kQ8SlotBytes;
+  const uint4* src = (lane < 16 ? p.k_full : p.v_full) + (size_t)pair * ctx * 16 + (lane & 15);
+  for (int s = blockIdx.y * 8 + warp; s < cap; s += gridDim.y * 8) {
+    int pos = -1;
+    if (s < p.L) {
+      pos = s;
+    } else if (s < p.L + d.y) {
+      const int mm = s - p.L;
+      if (d.w && mm < p.static_valid) {
+        const int j = p.static_idx[(size_t)pair * p.M + mm];
+        if (j >= 0 && j < p.n0) pos = p.L + j;
+      }
+    } else {
+      const int r = s - p.L - d.y;                 // ring slot r holds the newest j = r (mod cap)
+      if (p.n0 - 1 >= r && (p.sem_ring || !d.w)) pos = p.L + ((p.n0 - 1 - r) / d.z) * d.z + r;
+    }
+    if (pos < 0) continue;                         // the same for the whole warp
+    const uint4 raw = src[(size_t)pos * 16];
+    const float scale = row_scale16(raw);
+    unsigned char* dst = dst0 + (size_t)s * kQ8SlotBytes;
+    reinterpret_cast<uint2*>(dst)[lane] = quantize8(raw, scale);           // K codes at 0, V codes at 128
+    if ((lane & 15) == 0) reinterpret_cast<float*>(dst + 256)[lane >> 4] = scale;
+  }
+}
+
+// ----------------------------------------------------------------------------- decode over 272-byte slots
+constexpr int kWarps = 8;                  // streaming warps per CTA, each an independent worker
+constexpr int kStages = 2;
+constexpr int kChunk = 32;                 // slots per stage: 8704 bytes per copy in steady state
+constexpr int kGroups = 4;                 // 8-lane groups of a warp; group g takes slots g, g + 4, ..
+constexpr int kPer = kChunk / kGroups;
+constexpr int kU = 4;                      // slots a group folds in at a time
+constexpr int kRowBytes = kHeadDim * 2;    // a bf16 row of q, k_new, v_new, out
+constexpr int kStageQ = kChunk * kQ8SlotBytes;            // where the query row sits in a stage
+constexpr int kStageNew = kStageQ + kRowBytes;            // and the new token's K and V rows (bf16, as they arrive)
+constexpr int kStageBytes = kStageNew + 2 * kRowBytes;
+constexpr int kRingBytes = kWarps * kStages * kStageBytes;
+constexpr int kQ8SmemBytes = kRingBytes + kWarps * kStages * 8 + kWarps * 4 * 4;
+static_assert(kPer % kU == 0 && kQ8SmemBytes <= 227 * 1024 && kStageBytes % 16 == 0, "stage rings");
+
+struct Q8Unit {
+  const unsigned char* hbase;   // the head's first slot
+  size_t row;                   // byte offset of the head's row in q, k_new, v_new and out
+  int vh;                       // slots that hold a token
+  int pv, sv;                   // of which prompt slots and static slots (the rest is the ring)
+  int y;                        // static capacity
+  int fresh, phys;              // valid-slot index of the token being appended, and its slot in the head
+  int contig;
+};
+
+__device__ __forceinline__ void q8_unit_load(const DecodeLayersParams& p, int u, Q8Unit& U) {
+  const int pairs = p.n_seqs * p.H;
+  const int layer = u / pairs, pair = u - layer * pairs;
+  const int seq = pair / p.H, head = pair - seq * p.H;
+  const LayerState& ls = p.layer[layer];
+  const HeadDesc d = __ldg(ls.desc + head);
+  const int r = ls.new_j % d.z;
+  U.pv = ls.prompt_valid;
+  U.sv = d.w ? ls.static_valid : 0;
+  U.y = d.y;
+  U.vh = U.pv + U.sv + (ls.t_img < d.z ? ls.t_img : d.z);
+  U.fresh = U.pv + U.sv + r;
+  U.phys = p.L + d.y + r;
+  U.contig = (U.pv == p.L && U.sv == d.y) ? 1 : 0;
+  U.hbase = reinterpret_cast<const unsigned char*>(p.slab) +
+            ((size_t)ls.first_slot + (size_t)seq * ls.seq_slots + d.x) * kQ8SlotBytes;
+  U.row = ((size_t)layer * pairs + pair) * kRowBytes;
+}
+
+// 4 codes (one 32-bit word) -> 4 floats, exactly
+__device__ __forceinline__ void widen4(uint32_t w, float2& lo, float2& hi) {
+  uint32_t a, b;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(a) : "h"((uint16_t)(w & 0xffffu)));
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(b) : "h"((uint16_t)(w >> 16)));
+  lo = __half22float2(*reinterpret_cast<const __half2*>(&a));
+  hi = __half22float2(*reinterpret_cast<const __half2*>(&b));
+}
+
+// The rows of a stage as one lane holds them: slot 4*u + grp, 16 codes of K and of V (dimensions
+// [16*l8, 16*l8 + 16)) and the two row scales.
+struct Q8Rows {
+  uint4 k[kPer], v[kPer];
+  float ks[kPer], vs[kPer];
+};
+
+__device__ __forceinline__ void q8_load_stage(const unsigned char* __restrict__ sb, int n, int grp, int l8, Q8Rows& r) {
+#pragma unroll
+  for (int u = 0; u < kPer; ++u) {
+    const int slot = kGroups * u + grp;
+    const unsigned char* s = sb + slot * kQ8SlotBytes;
+    if (slot < n) {
+      r.k[u] = reinterpret_cast<const uint4*>(s)[l8];
+      r.v[u] = reinterpret_cast<const uint4*>(s + 128)[l8];
+      const float2 sc = *reinterpret_cast<const float2*>(s + 256);
+      r.ks[u] = sc.x;
+      r.vs[u] = sc.y;
+    } else {
+      r.k[u] = r.v[u] = make_uint4(0, 0, 0, 0);
+      r.ks[u] = r.vs[u] = 0.f;
+    }
+  }
+}
+
+__device__ __forceinline__ float q8_dot16(const uint4& k, const float2 (&q)[8]) {
+  const uint32_t w[4] = {k.x, k.y, k.z, k.w};
+  float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 lo, hi;
+    widen4(w[i], lo, hi);
+    a = __ffma2_rn(lo, q[2 * i], a);
+    b = __ffma2_rn(hi, q[2 * i + 1], b);
+  }
+  return (a.x + a.y) + (b.x + b.y);
+}
+
+__device__ __forceinline__ void q8_axpy16(float p, const uint4& v, float2 (&acc)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const float2 pp = make_float2(p, p);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 lo, hi;
+    widen4(w[i], lo, hi);
+    acc[2 * i] = __ffma2_rn(pp, lo, acc[2 * i]);
+    acc[2 * i + 1] = __ffma2_rn(pp, hi, acc[2 * i + 1]);
+  }
+}
+
+__device__ __forceinline__ void q8_fold_stage(const Q8Rows& r, int n, int grp, const float2 (&q)[8], State& st) {
+#pragma unroll
+  for (int s = 0; s < kPer; s += kU) {
+    if (kGroups * s >= n) break;
+    float x[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) x[u] = q8_dot16(r.k[s + u], q);
+#pragma unroll
+    for (int off = 4; off >= 1; off >>= 1) {
+#pragma unroll
+      for (int u = 0; u < kU; ++u) x[u] += __shfl_xor_sync(0xffffffffu, x[u], off);
+    }
+    float mn = st.m;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      x[u] = kGroups * (s + u) + grp < n ? x[u] * r.ks[s + u] : kNegBig;     // the K row's scale
+      mn = fmaxf(mn, x[u]);
+    }
+    const float corr = ex2(st.m - mn);
+    float p[kU], psum = 0.f;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      p[u] = kGroups * (s + u) + grp < n ? ex2(x[u] - mn) : 0.f;
+      psum += p[u];
+    }
+    st.l = st.l * corr + psum;
+    st.m = mn;
+    const float2 cc = make_float2(corr, corr);
+#pragma unroll
+    for (int d = 0; d < 8; ++d) st.acc[d] = __fmul2_rn(st.acc[d], cc);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) q8_axpy16(p[u] * r.vs[s + u], r.v[s + u], st.acc);   // the V row's scale
+  }
+}
+
+// One warp streams a whole head; heads (units, in the order layer, sequence, head) come from a global counter, the
+// next one asked for while the current one streams; its copy pipeline runs on across unit boundaries; the unit
+// ids travel from the warp's producer side to its consumer side through a 4-entry shared-memory FIFO.
+__global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(const __grid_constant__ DecodeLayersParams p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = lane >> 3, l8 = lane & 7;
+  const uint32_t FULL = 0xffffffffu;
+  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
+  const uint32_t ring_s = smem_u32(ring);
+  const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
+  volatile int* fifo = reinterpret_cast<volatile int*>(smem + kRingBytes + kWarps * kStages * 8) + warp * 4;
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    mbar_init_fence();
+  }
+  __syncwarp();
+  const int n_units = p.n_layers * p.n_seqs * p.H;
+
+  int raw_next = 0;
+  auto ask = [&]() {
+    if (lane == 0) raw_next = (int)atomicAdd(p.work, 1u);
+  };
+  ask();
+  int u = __shfl_sync(FULL, raw_next, 0);
+  if (u >= n_units) return;
+  ask();
+
+  Q8Unit PU, CU;               // the producer's and the consumer's current head
+  int pi = 0, ci = 0;          // and their positions in it
+  int produced = 0, consumed = 0, ahead = 0;
+  bool feeding = true;
+  q8_unit_load(p, u, PU);
+  if (lane == 0) fifo[0] = u;
+  produced = 1;
+  __syncwarp();
+
+  // Lane 0 starts the copies of the producer's next chunk into `stage`; every lane advances.
+  auto issue = [&](int stage) {
+    const int n = PU.vh - pi < kChunk ? PU.vh - pi : kChunk;
+    if (lane == 0) {
+      const bool begin = pi == 0;
+      const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
+      const bool has_fresh = PU.fresh >= pi && PU.fresh < pi + n;
+      // order the warp's reads (and the writes of a quantised row) of this stage before the asynchronous writes
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_expect_tx(bar, (uint32_t)(n * kQ8SlotBytes + (begin ? kRowBytes : 0) + (has_fresh ? 2 * kRowBytes : 0)));
+      if (PU.contig) {
+        bulk_g2s(dst, PU.hbase + (size_t)pi * kQ8SlotBytes, (uint32_t)n * kQ8SlotBytes, bar);
+      } else {
+        const int l0[3] = {0, PU.pv, PU.pv + PU.sv};          // logical start of each run
+        const int l1[3] = {PU.pv, PU.pv + PU.sv, PU.vh};      // and end
+        const int p0[3] = {0, p.L, p.L + PU.y};               // physical start
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+          const int lo = pi > l0[r] ? pi : l0[r], hi = pi + n < l1[r] ? pi + n : l1[r];
+          if (hi > lo)
+            bulk_g2s(dst + (uint32_t)(lo - pi) * kQ8SlotBytes, PU.hbase + (size_t)(p0[r] + lo - l0[r]) * kQ8SlotBytes,
+                     (uint32_t)(hi - lo) * kQ8SlotBytes, bar);
+        }
+      }
+      // the slot of the token being appended holds stale codes: its rows come from the caller, unquantised
+      if (has_fresh) {
+        bulk_g2s(dst + kStageNew, p.k_new + PU.row, kRowBytes, bar);
+        bulk_g2s(dst + kStageNew + kRowBytes, p.v_new + PU.row, kRowBytes, bar);
+      }
+      if (begin) bulk_g2s(dst + kStageQ, p.q + PU.row, kRowBytes, bar);
+    }
+    pi += n;
+    ++ahead;
+    if (pi == PU.vh) {                   // on to the unit asked for earlier, and ask for the one after
+      const int nu = __shfl_sync(FULL, raw_next, 0);
+      if (nu < n_units) {
+        ask();
+        q8_unit_load(p, nu, PU);
+        pi = 0;
+        if (lane == 0) fifo[produced & 3] = nu;
+        ++produced;
+        __syncwarp();
+      } else {
+        feeding = false;
+      }
+    }
+  };
+
+#pragma unroll 1
+  for (int s = 0; s < kStages && feeding; ++s) issue(s);
+
+  int stage = 0;
+  uint32_t parity = 0;
+  float2 q[8];
+  State st;
+  bool begin = true;
+
+#pragma unroll 1
+  for (;;) {
+    if (begin) {
+      if (consumed == produced) break;
+      q8_unit_load(p, fifo[consumed & 3], CU);
+      ++consumed;
+      ci = 0;
+    }
+    const int n = CU.vh - ci < kChunk ? CU.vh - ci : kChunk;
+    if (!mbar_wait(bar0 + 8 * stage, parity)) {
+      // give up: flag it, let the copies still in flight land (bounded), and leave
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int k = 0; k < ahead; ++k) {
+        mbar_wait(bar0 + 8 * stage, parity);
+        if (++stage == kStages) { stage = 0; parity ^= 1u; }
+      }
+      return;
+    }
+    unsigned char* sb = ring + (size_t)stage * kStageBytes;
+    if (begin) {
+      // the lane's 16 dimensions of the query, widened and scaled
+      const uint4* qs = reinterpret_cast<const uint4*>(sb + kStageQ) + 2 * l8;
+      const uint4 qa = qs[0], qb = qs[1];
+      const float2 sc = make_float2(p.scale_log2, p.scale_log2);
+      q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
+      q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
+      q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
+      q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
+      state_init(st);
+      begin = false;
+    }
+    {
+      // the chunk that carries the newest token: quantise its rows (lanes 0-15 the K row, 16-31 the V row), put the
+      // slot in its place in the stage and in the slab; later steps read what this step has attended to
+      const int s_new = CU.fresh - ci;
+      if (s_new >= 0 && s_new < n) {
+        const uint4 raw = reinterpret_cast<const uint4*>(sb + kStageNew)[lane];
+        const float scale = row_scale16(raw);
+        const uint2 codes = quantize8(raw, scale);
+        unsigned char* in_stage = sb + s_new * kQ8SlotBytes;
+        unsigned char* in_slab = const_cast<unsigned char*>(CU.hbase) + (size_t)CU.phys * kQ8SlotBytes;
+        reinterpret_cast<uint2*>(in_stage)[lane] = codes;
+        reinterpret_cast<uint2*>(in_slab)[lane] = codes;
+        if ((lane & 15) == 0) {
+          reinterpret_cast<float*>(in_stage + 256)[lane >> 4] = scale;
+          reinterpret_cast<float*>(in_slab + 256)[lane >> 4] = scale;
+        }
+        __syncwarp();
+      }
+    }
+    Q8Rows rows;
+    q8_load_stage(sb, n, grp, l8, rows);
+    __syncwarp();          // every lane has its rows in registers: the stage may be refilled
+    --ahead;
+    if (feeding) issue(stage);
+    q8_fold_stage(rows, n, grp, q, st);
+    ci += n;
+    if (ci == CU.vh) {
+      // the head is complete: merge the four groups and write the output row (lane l8 of group 0 holds
+      // dimensions [16 * l8, 16 * l8 + 16))
+      State tot = st;
+      state_merge_lane(tot, 8);
+      state_merge_lane(tot, 16);
+      if (grp == 0) {
+        const float inv = 1.f / tot.l;
+        uint32_t o[8];
+#pragma unroll
+        for (int d = 0; d < 8; ++d) {
+          __nv_bfloat162 t = __floats2bfloat162_rn(tot.acc[d].x * inv, tot.acc[d].y * inv);
+          o[d] = *reinterpret_cast<uint32_t*>(&t);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.out) + CU.row) + 2 * l8;
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+      }
+      begin = true;
+    }
+    if (++stage == kStages) { stage = 0; parity ^= 1u; }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_rows(const void* rows, long long n_rows, void* codes, float* scales, cudaStream_t st) {
+  const long long threads = n_rows * 16;
+  ssd_quantize_rows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(static_cast<const uint4*>(rows), n_rows,
+                                                                               static_cast<uint2*>(codes), scales);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_q8(const GatherParams& p, int max_slots, cudaStream_t st) {
+  dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
+  ssd_gather_q8_kernel<<<grid, 256, 0, st>>>(p, max_slots);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st) {
+  static std::atomic<int> n_sm[64] = {};   // 0 = this device is not set up yet
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < 64;
+  int sms = cached ? n_sm[dev].load(std::memory_order_acquire) : 0;
+  if (sms == 0) {
+    e = cudaFuncSetAttribute(ssd_decode_layers_q8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQ8SmemBytes);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (cached) n_sm[dev].store(sms, std::memory_order_release);
+  }
+  const long units = (long)p.n_layers * p.n_seqs * p.H;
+  if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  const long want = (units + kWarps - 1) / kWarps;
+  const int grid = (int)(want < sms ? want : sms);
+  ssd_decode_layers_q8_kernel<<<grid, kWarps * 32, kQ8SmemBytes, st>>>(p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+int q8_slot_bytes() { return kQ8SlotBytes; }
+
+}  // namespace ssd
