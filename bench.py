@@ -184,7 +184,7 @@ def run_reference(args, cfg):
 
 # ----------------------------------------------------------------------------- our arm
 def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False, t_steps=0, row_buffer=False,
-                classify=True):
+                classify=True, kv_format=0):
     """Create, classify, load and compress every layer; returns the cache and per-layer step inputs."""
     from paper_2510_18716_b200 import binding as B
     from paper_2510_18716_b200 import dist as D
@@ -199,6 +199,8 @@ def build_cache(cfg: wl.Workload, device, seq_lo, rank, world, full_cache=False,
         cache = B.SsdCache(ccfg, n_sink_heads_total=cfg.n_layers * cfg.n_sink_heads, device=device)
         if row_buffer:
             cache.set_row_buffer(True)
+        if kv_format:
+            cache.set_kv_format(kv_format)
         if not classify:
             cache.set_head_labels(np.stack([wl.sink_mask(cfg, l) for l in range(cfg.n_layers)]))
         mine = D.shard_calibration(cfg.n_cal, rank, world) if classify else None
@@ -596,6 +598,32 @@ def run_ours(args, cfg):
         del ecache, esteps, est
         torch.cuda.empty_cache()
 
+    # ---- 8-bit K/V (an extension the paper only cites, Sec. 2): a leg of its own, never the headline.  The same
+    # steps over a cache of 272-byte slots; per-layer form = the format's one kernel launched on one layer at a time
+    q8 = None
+    if not args.no_q8:
+        Kq = min(K, 40)
+        qcache, qsteps = build_cache(cfg, device, rank * S, rank, world, t_steps=2 * Kq + 8, classify=False, kv_format=1)
+        qst = Stepper(cfg, qcache, qsteps, out)
+        ms_q = {}
+        for form in (False, True):
+            for _ in range(3):
+                qst.step(one_launch=form)
+            ms_q[form] = max_over_ranks(timed(lambda: qst.step(one_launch=form), Kq, barrier)) / Kq
+        slots_q = int(sum(int(qcache.get_lengths(l).sum()) for l in range(cfg.n_layers))) / cfg.n_layers
+        # codes and scales of the valid slots, q in and out, the new token's bf16 rows read and its slot written
+        qbytes = S * (slots_q * 272 + H * 2 * 256 + H * (512 + 272)) * cfg.n_layers
+        q8 = {"kv_dtype": "e4m3 codes + float32 scale per row (272 B per slot)", "unit": UNIT,
+              "value": cfg.images_per_step * world / (ms_q[False] * 1e-3), "ms_per_step": ms_q[False],
+              "ms_per_step_one_launch": ms_q[True], "steps": Kq, "kv_bytes_per_seq": qcache.kv_bytes_per_seq(),
+              "roofline_one_launch": {"bound": "hbm", "kernel": "ssd_decode_layers_q8_kernel", "achieved": qbytes / (ms_q[True] * 1e-3) / 1e9,
+                                      "peak": peak, "unit": "GB/s", "frac": qbytes / (ms_q[True] * 1e-3) / 1e9 / peak,
+                                      "peak_kind": f"of {peak_kind}", "bytes_per_launch": qbytes, "traffic": None},
+              "device_status": qcache.device_status()}
+        qcache.close()
+        del qcache, qsteps, qst
+        torch.cuda.empty_cache()
+
     # ---- analysis utility (Sec. 3.2, MSE_token): per-token divergence of two uncompressed caches of one layer
     analysis = None
     if rank == 0 and world == 1:
@@ -652,7 +680,7 @@ def run_ours(args, cfg):
             "one_launch": one_launch,
             "one_time": setup_times,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf, "analysis": analysis,
+            "cpu_baseline": cpu, "full_cache": full, "row_buffer": rowbuf, "kv_8bit": q8, "analysis": analysis,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -719,6 +747,7 @@ def main():
     ap.add_argument("--no-full-cache", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-row-buffer", action="store_true")
+    ap.add_argument("--no-q8", action="store_true", help="skip the 8-bit K/V leg")
     ap.add_argument("--sweep", action="store_true", help="large-batch sweep on the 7B shape: one JSON line per point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
