@@ -108,12 +108,21 @@ __global__ void __launch_bounds__(256) ssd_gather_q8_kernel(const GatherParams p
 }
 
 // ----------------------------------------------------------------------------- decode over 272-byte slots
-constexpr int kWarps = 8;                  // streaming warps per CTA, each an independent worker
-constexpr int kStages = 2;
-constexpr int kChunk = 32;                 // slots per stage: 8704 bytes per copy in steady state
+#ifndef SSD_Q8_WARPS
+#define SSD_Q8_WARPS 12
+#endif
+#ifndef SSD_Q8_STAGES
+#define SSD_Q8_STAGES 2
+#endif
+#ifndef SSD_Q8_CHUNK
+#define SSD_Q8_CHUNK 24
+#endif
+constexpr int kWarps = SSD_Q8_WARPS;       // streaming warps per CTA, each an independent worker
+constexpr int kStages = SSD_Q8_STAGES;
+constexpr int kChunk = SSD_Q8_CHUNK;       // slots per stage: 6528 bytes per copy in steady state
 constexpr int kGroups = 4;                 // 8-lane groups of a warp; group g takes slots g, g + 4, ..
 constexpr int kPer = kChunk / kGroups;
-constexpr int kU = 4;                      // slots a group folds in at a time
+constexpr int kU = kPer % 4 == 0 ? 4 : (kPer % 3 == 0 ? 3 : 2);   // slots a group folds in at a time
 constexpr int kRowBytes = kHeadDim * 2;    // a bf16 row of q, k_new, v_new, out
 constexpr int kStageQ = kChunk * kQ8SlotBytes;            // where the query row sits in a stage
 constexpr int kStageNew = kStageQ + kRowBytes;            // and the new token's K and V rows (bf16, as they arrive)
