@@ -37,13 +37,13 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
 DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.26e6, "per_layer_of_step": 160.89e6,
-                  "sha256": "8ae52eb6b67ee40171d816382324d6a8221d36a9c956d2adab099f68e092f47c"}
+                  "sha256": "84da792082f7f46c4738632fb55b6c193e1b20c81b9428dc87b46f5c96855332"}
 
 
 def decode_traffic(cfg):
     import hashlib
     h = hashlib.sha256()
-    for f in ("ssd_decode.cu", "ssd_plan.h", "ssd_internal.cuh"):
+    for f in ("ssd_decode.cu", "ssd_device.cuh", "ssd_plan.h", "ssd_internal.cuh"):
         with open(os.path.join(ROOT, "paper_2510_18716_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     if h.hexdigest() != DECODE_TRAFFIC["sha256"] or not cfg.name.startswith(DECODE_TRAFFIC["workload"]):
