@@ -974,7 +974,10 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
     ly.todo = (c->n_sink[layer] > 0 && (ly.buffered > 0 || ly.pending)) ? 1 : 0;
     any = any || ly.todo;
   }
-  if (any && launch_recompress_layers(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
+  // a buffer of one token (Algorithm 1 taken literally) needs no ranking: drop the lowest score
+  if (any && (g.sink_recent == 1 ? launch_evict_one_layers(p, static_cast<cudaStream_t>(stream))
+                                 : launch_recompress_layers(p, static_cast<cudaStream_t>(stream))) != cudaSuccess)
+    return SSD_ERR_CUDA;
   for (int i = 0; i < n_layers; ++i) {
     const int layer = first_layer + i;
     if (p.layer[i].todo) {

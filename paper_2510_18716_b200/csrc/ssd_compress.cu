@@ -348,6 +348,66 @@ __global__ void __launch_bounds__(kThreads) ssd_recompress_layers_kernel(const _
   recompress_pair(p, blockIdx.x);
 }
 
+// Re-selection with a row buffer of ONE token (Algorithm 1 taken literally, one step): the token appended in
+// the step just attended to either takes a still unused static slot, or the slot of the lowest-scoring static
+// token (among equal scores the highest position leaves, so the new token loses ties), or is dropped itself.
+// The same result as recompress_pair with one buffered token, without its rank counting and block-wide
+// barriers: one warp per (layer, pair), which first adds the pending weights of the layer's last decode.
+__global__ void __launch_bounds__(kThreads) ssd_evict_one_kernel(const __grid_constant__ RecompressLayersParams q) {
+  const int lane = threadIdx.x & 31;
+  const long long w = ((long long)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int pairs = q.n_seqs * q.H;
+  if (w >= (long long)q.n_layers * pairs) return;
+  const int layer = (int)(w / pairs), pair = (int)(w - (long long)layer * pairs);
+  const RecompressLayer& ly = q.layer[layer];
+  if (!ly.todo) return;
+  const int seq = pair / q.H, head = pair - seq * q.H;
+  const HeadDesc d = q.desc[(size_t)layer * q.H + head];
+  if (!d.w) return;
+  const size_t pr = (size_t)layer * pairs + pair;
+  float* acc = q.acc + pr * q.mr;
+  int32_t* idx = q.static_idx + pr * (q.M > 0 ? q.M : 1);
+  const float* lg = q.logits + (((size_t)layer * 2 + ly.lg) * pairs + pair) * q.mr;
+  float mx = 0.f, inv = 0.f;
+  if (ly.pending) {
+    const float2 ml = q.ml[((size_t)layer * 2 + ly.lg) * pairs + pair];
+    mx = ml.x;
+    inv = 1.f / ml.y;
+  }
+  const int sv = ly.static_valid;
+  float worst = 3.0e38f;
+  int worst_pos = -1, worst_e = -1;
+  for (int i = lane; i < sv; i += 32) {
+    float sc = acc[i];
+    if (ly.pending) {
+      sc += ex2(lg[i] - mx) * inv;
+      acc[i] = sc;
+    }
+    const int pos = idx[i];
+    if (sc < worst || (sc == worst && pos > worst_pos)) { worst = sc; worst_pos = pos; worst_e = i; }
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const float w2 = __shfl_xor_sync(0xffffffffu, worst, off);
+    const int p2 = __shfl_xor_sync(0xffffffffu, worst_pos, off), e2 = __shfl_xor_sync(0xffffffffu, worst_e, off);
+    if (w2 < worst || (w2 == worst && p2 > worst_pos)) { worst = w2; worst_pos = p2; worst_e = e2; }
+  }
+  if (ly.buffered < 1) return;                       // nothing buffered: only the pending weights were due
+  float w_new = acc[d.y];                            // entry of buffer slot 0
+  if (ly.pending) w_new += ex2(lg[d.y] - mx) * inv;
+  int dest = -1;
+  if (sv < q.M) dest = sv;
+  else if (sv > 0 && !(w_new <= worst)) dest = worst_e;
+  __syncwarp();                                      // the scores written above, before the one written below
+  if (dest < 0) return;
+  if (lane == 0) {
+    acc[dest] = w_new;
+    idx[dest] = ly.t_base;
+  }
+  uint4* hb = q.slab + ((size_t)ly.first_slot + (size_t)seq * ly.seq_slots + d.x + q.L) * kSlotU4;
+  hb[(size_t)dest * kSlotU4 + lane] = hb[(size_t)d.y * kSlotU4 + lane];
+}
+
 }  // namespace
 
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
@@ -369,6 +429,14 @@ cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream
   cudaError_t e = cudaFuncSetAttribute(ssd_recompress_layers_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   ssd_recompress_layers_kernel<<<dim3(p.n_seqs * p.H, p.n_layers), kThreads, smem, st>>>(p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_evict_one_layers(const RecompressLayersParams& p, cudaStream_t st) {
+  if (p.n_layers < 1 || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
+  const long long warps = (long long)p.n_layers * p.n_seqs * p.H;
+  ssd_evict_one_kernel<<<(unsigned)((warps * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }

@@ -208,6 +208,8 @@ struct RecompressLayersParams {
   RecompressLayer layer[kMaxLayersPerLaunch];
 };
 cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream_t st);
+// the same for a row buffer of one token (every layer has at most one token buffered): one warp per pair
+cudaError_t launch_evict_one_layers(const RecompressLayersParams& p, cudaStream_t st);
 cudaError_t launch_classify(const ClassifyParams& p, int n_row_blocks, cudaStream_t st);
 int classify_rows_per_block();
 int decode_max_workers();
