@@ -91,8 +91,6 @@ struct ssd_cache {
   // re-selection), -1 if none, -2 if unknown: a decode launch of ANOTHER layer may prefetch its slab
   // before that launch has completed.
   int last_writer = -2;
-  // The same for the layer's score tables of the row-buffer mode (accumulated scores, logits, (max, sum)).
-  int last_scored = -2;
   int score_layer = -1, score_n0 = 0; // layer whose prefill scores (ssd_compress) the score buffer holds, -1 if none
   bool row_buffer = false;            // Algorithm 2: rings of semantic heads are row buffers
   std::vector<int32_t> t_base;        // [layers] image tokens held when the buffer was last emptied
@@ -493,7 +491,6 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   c->t_base[layer] = n0;
   c->pending[layer] = 0;
   c->last_writer = -2;
-  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -523,7 +520,6 @@ int ssd_append(ssd_cache* c, int32_t layer, const void* k_new, const void* v_new
   p.ml = c->d_ml(layer, c->lg_cur[layer]);
   if (launch_append(p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = layer;
-  c->last_scored = c->row_buffer ? layer : -1;
   if (c->row_buffer) c->pending[layer] = 0;
   c->t_img[layer] += 1;
   return SSD_OK;
@@ -549,7 +545,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   p.mr = c->mr();
   p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1; p.sem_slot = -1;
   p.fold_acc = nullptr; p.fold_logits = nullptr; p.fold_ml = nullptr;
-  p.fold_pending = 0; p.fold_early = 0; p.fold_static = 0; p.fold_buffered = 0;
+  p.fold_pending = 0; p.fold_static = 0; p.fold_buffered = 0;
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
@@ -559,7 +555,6 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;
-  c->last_scored = c->row_buffer ? layer : -1;
   if (c->row_buffer) {
     c->pending[layer] = 1;
     c->lg_cur[layer] = (uint8_t)lg_next;
@@ -609,7 +604,6 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   p.v_new = static_cast<const unsigned char*>(v_new);
   p.new_j = c->t_img[layer];
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
-  p.fold_early = (p.early && c->last_scored >= -1 && c->last_scored != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->t_img[layer] += 1;                // the view describes the layer with the token in place
@@ -622,7 +616,6 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
     return SSD_ERR_CUDA;
   }
   c->last_writer = layer;
-  c->last_scored = scored ? layer : -1;
   if (scored) {
     c->pending[layer] = 1;
     c->lg_cur[layer] = (uint8_t)lg_next;
@@ -708,7 +701,6 @@ int ssd_append_decode_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers
     }
   }
   c->last_writer = -2;                 // several layers' slabs were written
-  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -942,7 +934,6 @@ int ssd_recompress(ssd_cache* c, int32_t layer, void* stream) {
   c->t_base[layer] = c->t_img[layer];
   c->pending[layer] = 0;
   c->last_writer = -2;
-  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -988,7 +979,6 @@ int ssd_recompress_layers(ssd_cache* c, int32_t first_layer, int32_t n_layers, v
     c->pending[layer] = 0;
   }
   c->last_writer = -2;
-  c->last_scored = -2;
   return SSD_OK;
 }
 
@@ -1177,14 +1167,13 @@ extern "C" int ssd_decode_attn_static(ssd_cache* c, int32_t layer, const void* q
   p.mr = c->mr();
   p.k_new = nullptr; p.v_new = nullptr; p.new_j = -1; p.sem_slot = -1;
   p.fold_acc = nullptr; p.fold_logits = nullptr; p.fold_ml = nullptr;
-  p.fold_pending = 0; p.fold_early = 0; p.fold_static = 0; p.fold_buffered = 0;
+  p.fold_pending = 0; p.fold_static = 0; p.fold_buffered = 0;
   p.early = (c->last_writer >= -1 && c->last_writer != layer) ? 1 : 0;
   p.scale_log2 = c->scale * 1.4426950408889634f;
   p.split = Split{0, 0, 0, 0, 0.f};
   c->fill_view(layer, p.view);
   if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;
-  c->last_scored = c->row_buffer ? layer : -1;
   if (c->row_buffer) {
     c->pending[layer] = 1;
     c->lg_cur[layer] = (uint8_t)lg_next;

@@ -60,7 +60,7 @@ constexpr int kStages = SSD_DECODE_STAGES;
 constexpr int kChunk = SSD_DECODE_CHUNK;             // slots per stage
 constexpr int kGroups = 4;                           // 8-lane groups of a warp
 constexpr int kPer = kChunk / kGroups;               // slots of a stage each group takes
-constexpr int kU = kPer < 4 ? kPer : 4;              // slots a group folds in at a time
+constexpr int kU = kPer % 4 == 0 ? 4 : (kPer % 3 == 0 ? 3 : (kPer % 2 == 0 ? 2 : 1));   // slots a group folds in at a time
 constexpr int kQBytes = kHeadDim * 2;
 constexpr int kStageBytes = kChunk * kSlotBytes + kQBytes;
 constexpr int kRingBytes = kWarps * kStages * kStageBytes;
@@ -238,49 +238,65 @@ __device__ __forceinline__ void new_token_slot(const LayerView& v, int h, int ne
 // pairs; entry c of a score row is static slot c or, from the static capacity on, buffer slot c - capacity.
 __device__ void fold_scores(const DecodeParams& p, int lane) {
   const LayerView& v = p.view;
-  // Items (pair, entry) are dealt to the lanes kFoldBatch at a time, loads first, so that the warp has
-  // hundreds of independent loads in flight: with HBM saturated by the streaming warps a dependent trip
-  // to memory takes microseconds, and one trip per item would outlast the launch.
-  constexpr int kFoldBatch = 16;
+  const uint32_t FULL = 0xffffffffu;
+  // This block's pairs are b, b + grid, ..; lane k looks at pair k, and the semantic ones are then taken four
+  // at a time, all their loads issued before the first use: with HBM saturated by the streaming warps a
+  // dependent trip to memory takes microseconds, so the trips must overlap; and the loop is kept free of
+  // divisions, because this warp shares its scheduler with two streaming warps.
+  constexpr int kFoldPairs = 4;
   const int n_pairs = v.n_seqs * v.H;
   const int n_mine = (n_pairs - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int n_old = p.fold_pending ? p.fold_static + p.fold_buffered : 0;
   float* __restrict__ accp = p.fold_acc;
-  if (p.fold_pending) {
-    const float* __restrict__ lgp = p.fold_logits;
-    const float2* __restrict__ mlp = p.fold_ml;
-    const int total = n_mine * p.mr;
-    for (int it0 = lane; it0 < total; it0 += 32 * kFoldBatch) {
-      float a[kFoldBatch], x[kFoldBatch];
-      float2 ml[kFoldBatch];
-      uint32_t off[kFoldBatch];
-      bool ok[kFoldBatch];
+  const float* __restrict__ lgp = p.fold_logits;
+  const float2* __restrict__ mlp = p.fold_ml;
+  for (int k0 = 0; k0 < n_mine; k0 += 32) {
+    const int my_pair = (int)blockIdx.x + (k0 + lane) * (int)gridDim.x;
+    const bool sem = k0 + lane < n_mine && v.head[my_pair % v.H].w != 0;
+    unsigned todo = __ballot_sync(FULL, sem);
+    while (todo) {
+      int pair[kFoldPairs], ycap[kFoldPairs], np = 0;
 #pragma unroll
-      for (int u = 0; u < kFoldBatch; ++u) {
-        const int it = it0 + 32 * u;
-        const int k = it / p.mr, c = it - k * p.mr;
-        const int pair = (int)blockIdx.x + k * (int)gridDim.x;
-        ok[u] = false;
-        if (it < total) {
-          const HeadRec d = v.head[pair % v.H];
-          ok[u] = d.w && (c < p.fold_static || (c >= d.y && c < d.y + p.fold_buffered));
-        }
-        off[u] = (uint32_t)pair * (uint32_t)p.mr + (uint32_t)c;      // n_seqs * H * (M + R) < 2^31 (checked at create)
-        if (ok[u]) {
-          a[u] = accp[off[u]];
-          x[u] = lgp[off[u]];
-          ml[u] = mlp[pair];
+      for (int j = 0; j < kFoldPairs; ++j) {
+        pair[j] = 0;
+        ycap[j] = 0;
+        if (todo) {
+          const int src = __ffs(todo) - 1;
+          todo &= todo - 1;
+          pair[j] = __shfl_sync(FULL, my_pair, src);
+          ycap[j] = v.head[pair[j] % v.H].y;
+          np = j + 1;
         }
       }
+      if (n_old > 0) {
+        float2 ml[kFoldPairs];
 #pragma unroll
-      for (int u = 0; u < kFoldBatch; ++u)
-        if (ok[u]) accp[off[u]] = a[u] + ex2(x[u] - ml[u].x) / ml[u].y;
-    }
-  }
-  if (p.sem_slot >= 0) {
-    for (int k = lane; k < n_mine; k += 32) {
-      const int pair = (int)blockIdx.x + k * (int)gridDim.x;
-      const HeadRec d = v.head[pair % v.H];
-      if (d.w) accp[(size_t)pair * p.mr + d.y + p.sem_slot] = 0.f;
+        for (int j = 0; j < kFoldPairs; ++j) ml[j] = j < np ? mlp[pair[j]] : make_float2(0.f, 1.f);
+        for (int i = lane; i < n_old; i += 32) {
+          float a[kFoldPairs], x[kFoldPairs];
+          uint32_t off[kFoldPairs];
+#pragma unroll
+          for (int j = 0; j < kFoldPairs; ++j) {
+            // entry of the i-th scored token: static slot i, or buffer slot i - static behind the static capacity
+            const int c = i < p.fold_static ? i : ycap[j] + (i - p.fold_static);
+            off[j] = (uint32_t)pair[j] * (uint32_t)p.mr + (uint32_t)c;     // n_seqs * H * (M + R) < 2^31 (checked at create)
+            if (j < np) {
+              a[j] = accp[off[j]];
+              x[j] = lgp[off[j]];
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < kFoldPairs; ++j)
+            if (j < np) accp[off[j]] = a[j] + ex2(x[j] - ml[j].x) / ml[j].y;
+        }
+      }
+      if (p.sem_slot >= 0 && lane < np) {
+        int pj = pair[0], yj = ycap[0];
+#pragma unroll
+        for (int j = 1; j < kFoldPairs; ++j)
+          if (lane == j) { pj = pair[j]; yj = ycap[j]; }
+        accp[(size_t)pj * p.mr + yj + p.sem_slot] = 0.f;       // the token being appended starts at zero
+      }
     }
   }
 }
@@ -321,12 +337,9 @@ __device__ void finisher(const DecodeParams& p, const unsigned char* smem, int l
   }
   unsigned heads = __ballot_sync(FULL, r_pair >= 0);
   if (!heads && p.fold_acc == nullptr) return;
-  // the scores belong to this layer: when the preceding launch worked on another layer's tables nothing can
-  // still be writing them
-  if (p.fold_acc != nullptr && p.fold_early) fold_scores(p, lane);
   pdl_wait_predecessor();                // the scratch below may still be in use by the previous launch
   pdl_allow_successor();
-  if (p.fold_acc != nullptr && !p.fold_early) fold_scores(p, lane);
+  if (p.fold_acc != nullptr) fold_scores(p, lane);
   if (!heads) return;
   for (unsigned h = heads; h; h &= h - 1) {
     const int slot = __ffs(h) - 1;       // 0: began in an earlier CTA, 1: begins here and runs on
@@ -423,60 +436,75 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
   Walk cons = prod;
   int ahead = 0;   // chunks issued and not yet consumed
 
-  // Lane 0 starts copies of the chunk at walk position `w` into `stage`.  what & 1: the slab part
-  // (and the barrier's byte count for the whole chunk); what & 2: the caller's inputs that travel with
-  // the chunk (the head's query row with its first chunk, the newest token's rows in place of its slot).
+  // Lane 0 starts copies of the chunk at a walk position into a stage, in two steps: planning (everything that
+  // needs the layout tables: where the head starts, where the newest token sits, the rows of the caller's
+  // inputs) and firing (fence, byte count, the copies).  The main loop plans the next chunk while it waits for
+  // the current one's data, so that between "the stage is free" and "its refill is on its way" only the firing
+  // remains.  what & 1: the slab part (and the barrier's byte count for the whole chunk); what & 2: the caller's
+  // inputs that travel with the chunk (the head's query row with its first chunk, the newest token's rows in
+  // place of its slot).
+  struct Plan {
+    const unsigned char* hbase;   // the head's first slot
+    size_t row;                   // byte offset of the head's row in q, k_new, v_new
+    int head, i, n;               // valid slots [i, i + n) of the head
+    int fresh;                    // valid-slot index of the newest token in this head (-1: none)
+    bool begin;                   // the chunk carries the head's query row
+  };
   int pf_key = -1, pf_fresh = -1, pf_phys = 0;     // producer side: newest token's slot in the current head
-  auto copy_chunk = [&](const Walk& w, int stage, int what) {
-    const int n = walk_chunk(w, kChunk);
+  auto plan_chunk = [&](const Walk& w, Plan& pl) {
+    pl.n = walk_chunk(w, kChunk);
+    pl.i = w.i;
+    pl.head = w.head;
+    pl.begin = w.i == 0 || w.g == g_begin;
     if (lane != 0) return;
-    const bool begin = w.i == 0 || w.g == g_begin;
-    const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
-    const unsigned char* hbase = reinterpret_cast<const unsigned char*>(p.slab) +
-                                 ((size_t)w.seq * v.seq_slots + v.head[w.head].x) * kSlotBytes;
+    pl.hbase = reinterpret_cast<const unsigned char*>(p.slab) + ((size_t)w.seq * v.seq_slots + v.head[w.head].x) * kSlotBytes;
     if (p.new_j >= 0 && pf_key != w.seq * v.H + w.head) {      // once per head, not per chunk
       pf_key = w.seq * v.H + w.head;
       new_token_slot(v, w.head, p.new_j, p.sem_slot, pf_fresh, pf_phys);
     }
-    const int fresh = pf_fresh;
-    const bool has_fresh = fresh >= w.i && fresh < w.i + n;
+    pl.fresh = pf_fresh;
+    pl.row = ((size_t)w.seq * v.H + w.head) * kQBytes;
+  };
+  auto fire_chunk = [&](const Plan& pl, int stage, int what) {
+    if (lane != 0) return;
+    const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
+    const int fresh = pl.fresh, n = pl.n;
+    const bool has_fresh = fresh >= pl.i && fresh < pl.i + n;
     if (what & 1) {
       // order the warp's reads of this stage (made visible to this lane by __syncwarp) before
       // the asynchronous writes that follow
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + (begin ? kQBytes : 0)));
+      mbar_expect_tx(bar, (uint32_t)(n * kSlotBytes + (pl.begin ? kQBytes : 0)));
       // valid slots [a, a + len) of the head into the stage from slot `at` on
       auto copy_range = [&](int a, int len, int at) {
         if (len <= 0) return;
         if (v.contig) {
-          bulk_g2s(dst + (uint32_t)at * kSlotBytes, hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
+          bulk_g2s(dst + (uint32_t)at * kSlotBytes, pl.hbase + (size_t)a * kSlotBytes, (uint32_t)len * kSlotBytes, bar);
         } else {
-          chunk_runs(v, w.head, a, len, [&](int src, int d, int l) {
-            bulk_g2s(dst + (uint32_t)(at + d) * kSlotBytes, hbase + (size_t)src * kSlotBytes, (uint32_t)l * kSlotBytes, bar);
+          chunk_runs(v, pl.head, a, len, [&](int src, int d, int l) {
+            bulk_g2s(dst + (uint32_t)(at + d) * kSlotBytes, pl.hbase + (size_t)src * kSlotBytes, (uint32_t)l * kSlotBytes, bar);
           });
         }
       };
       if (has_fresh) {                   // the slab is copied around the newest token's slot
-        copy_range(w.i, fresh - w.i, 0);
-        copy_range(fresh + 1, w.i + n - fresh - 1, fresh + 1 - w.i);
+        copy_range(pl.i, fresh - pl.i, 0);
+        copy_range(fresh + 1, pl.i + n - fresh - 1, fresh + 1 - pl.i);
       } else {
-        copy_range(w.i, n, 0);
+        copy_range(pl.i, n, 0);
       }
     }
     if (what & 2) {
-      const size_t row = ((size_t)w.seq * v.H + w.head) * kQBytes;
       if (has_fresh) {
-        bulk_g2s(dst + (uint32_t)(fresh - w.i) * kSlotBytes, p.k_new + row, kQBytes, bar);
-        bulk_g2s(dst + (uint32_t)(fresh - w.i) * kSlotBytes + kQBytes, p.v_new + row, kQBytes, bar);
+        bulk_g2s(dst + (uint32_t)(fresh - pl.i) * kSlotBytes, p.k_new + pl.row, kQBytes, bar);
+        bulk_g2s(dst + (uint32_t)(fresh - pl.i) * kSlotBytes + kQBytes, p.v_new + pl.row, kQBytes, bar);
       }
-      if (begin) bulk_g2s(dst + kChunk * kSlotBytes, reinterpret_cast<const unsigned char*>(p.q) + row, kQBytes, bar);
+      if (pl.begin) bulk_g2s(dst + kChunk * kSlotBytes, reinterpret_cast<const unsigned char*>(p.q) + pl.row, kQBytes, bar);
     }
   };
-  // the producer's current chunk, whole; every lane advances
-  auto issue = [&](int stage) {
-    copy_chunk(prod, stage, 3);
-    advance(prod, walk_chunk(prod, kChunk));
-    ++ahead;
+  auto copy_chunk = [&](const Walk& w, int stage, int what) {
+    Plan pl;
+    plan_chunk(w, pl);
+    fire_chunk(pl, stage, what);
   };
 
   // Prologue.  Everything above read only the launch parameters.  The slab holds nothing that the
@@ -518,6 +546,9 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
 #pragma unroll 1
   while (cons.g < cons.g_end) {
     const int n = walk_chunk(cons, kChunk);
+    Plan next;                                     // the chunk that will refill this stage, planned while its data is awaited
+    const bool more = prod.g < prod.g_end;
+    if (more) plan_chunk(prod, next);
     if (!mbar_wait(bar0 + 8 * stage, parity)) {
       // give up: flag it, let the copies still in flight land (bounded), and leave
       if (lane == 0) atomicOr(p.status, 1u);
@@ -560,7 +591,11 @@ __global__ void __launch_bounds__(kThreads, 1) ssd_decode_kernel(const __grid_co
     }
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
-    if (prod.g < prod.g_end) issue(stage);
+    if (more) {
+      fire_chunk(next, stage, 3);
+      advance(prod, next.n);
+      ++ahead;
+    }
     fold_stage(rows, n, grp, l8, q, st, sink);
 
     const int i1 = cons.i + n;

@@ -50,7 +50,6 @@ struct DecodeParams {
   const float* fold_logits; // [n_seqs * H, M + R]; read only if fold_pending
   const float2* fold_ml;    // [n_seqs * H]
   int fold_pending;         // 1: the previous decode's weights are not yet in the scores
-  int fold_early;           // 1: the launch before this one does not write this layer's score tables either
   int fold_static, fold_buffered;   // static and buffered entries that held a token at that decode
   int early;                // 1: the launch before this one on the stream does not write this layer's slab
   float scale_log2;         // softmax scale * log2(e)

@@ -23,7 +23,6 @@ namespace ssd {
 namespace {
 
 constexpr int kQ8SlotBytes = 272;
-constexpr int kQ8SlotU4 = kQ8SlotBytes / 16;   // 17
 
 // two floats -> two E4M3 codes (a in the low byte)
 __device__ __forceinline__ uint32_t e4m3x2(float a, float b) {
