@@ -36,8 +36,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.26e6, "per_layer_of_step": 160.89e6,
-                  "sha256": "84da792082f7f46c4738632fb55b6c193e1b20c81b9428dc87b46f5c96855332"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.41e6, "per_layer_of_step": 160.98e6,
+                  "sha256": "4a845e3ac2a81a26e8916864b946d0f3387db3a95adacbf34dc0522cc8e20692"}
 
 
 def decode_traffic(cfg):
