@@ -584,7 +584,8 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
         st.all = lo_l * ex2(lo_m - mn) + hi_l * ex2(hi_m - mn);
         st.m = mn;
       }
-      const float inv = st.all > 0.f ? 1.f / st.all : 0.f;
+      // the normaliser goes into the exponent: p = 2^(x - (m + log2 l)), one multiplication less per logit
+      const float m_l = st.all > 0.f ? st.m + __log2f(st.all) : 1.0e30f;
 
       // sweep 2: normalised probabilities, column sums over the block's rows
       for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) {
@@ -603,11 +604,11 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
           }
           if (warp_full && base + 32 <= lo_ctx) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv;
+            for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], p.scale_log2, -m_l));
           } else {
             const int nv = clamp32(ctx_r - base);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -st.m)) * inv : 0.f;
+            for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -m_l)) : 0.f;
           }
           const float col = warp_column_sums(v, lane);
           const int key = base + lane;
