@@ -97,3 +97,25 @@ def test_null_and_bad_arguments_are_rejected_on_the_host():
     assert lib.ssd_cache_max_slots(None) == -1
     assert lib.ssd_cache_tokens(None, 0) == -1
     assert isinstance(B.kernel_launch_count(), int)
+
+
+def test_threshold_rule_exports_need_no_gpu():
+    """Sec. 3.3: s = ratio sum / (P * N) in float32, semantic iff s > tau (equality is spatial); host arithmetic."""
+    lib = B.load()
+    P, N = 3, 10
+    sums = np.array([0.45 * P * N, 0.46 * P * N, 0.0, float(P * N)], np.float64)
+    s, lab = B.labels_from_ratio_sums(sums, P, N, 0.45)
+    assert s.dtype == np.float32 and lab.tolist() == [int(np.float32(0.45 * P * N / (P * N)) > np.float32(0.45)), 1, 0, 1]
+    assert np.array_equal(s, (sums / (P * N)).astype(np.float32))
+    assert B.labels_from_sparsity(np.array([0.45, 0.4500001, 0.2], np.float32), 0.45).tolist() == [0, 1, 0]
+    x = np.zeros(4, np.float64)
+    out = np.zeros(4, np.uint8)
+    assert lib.ssd_labels_from_ratio_sums(None, 4, 1, 1, C.c_float(0.5), None, out.ctypes.data) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_labels_from_ratio_sums(x.ctypes.data, 4, 0, 1, C.c_float(0.5), None, out.ctypes.data) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_labels_from_ratio_sums(x.ctypes.data, 4, 1, 1, C.c_float(float("nan")), None, out.ctypes.data) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_labels_from_sparsity(None, 4, C.c_float(0.5), out.ctypes.data) == B.SSD_ERR_INVALID_ARG
+    p = x.ctypes.data
+    assert lib.ssd_kv_token_mse(None, p, p, p, 1, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_quantize_rows_e4m3(None, 1, p, p, None) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_cache_set_kv_format(None, 1) == B.SSD_ERR_INVALID_ARG
+    assert lib.ssd_cache_get_compress_scores(None, 0, p) == B.SSD_ERR_INVALID_ARG

@@ -123,6 +123,18 @@ def test_layers_launch_argument_errors():
     assert lib.ssd_append_decode_layers(c._h, 0, 2, x.data_ptr() + 2, *args[1:]) == B.SSD_ERR_INVALID_ARG   # misaligned
     assert B.kernel_launch_count() == before
     c.close()
+    # a score row that a warp cannot keep in shared memory is a documented limit, not a launch failure: with a
+    # buffer of one token the one-launch step needs three rows of M + 1 entries (rounded up to 4) per warp
+    big = B.make_config(1, 1, 2, 4, 1300, 8, 1100, 1)
+    c = B.SsdCache(big, device=dev)
+    c.set_row_buffer(True)
+    c.set_head_labels(np.ones(2, np.uint8))
+    y = torch.zeros((1, 1, 2, 128), dtype=torch.bfloat16, device=dev)
+    before = B.kernel_launch_count()
+    assert lib.ssd_append_decode_layers(c._h, 0, 1, y.data_ptr(), y.data_ptr(), y.data_ptr(), y.data_ptr(),
+                                        torch.cuda.current_stream().cuda_stream) == B.SSD_ERR_LIMIT
+    assert B.kernel_launch_count() == before
+    c.close()
 
 
 def test_janus7b_whole_step_launch_size_sampled_pairs():
