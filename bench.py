@@ -116,6 +116,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def config_dict(cfg, world, kv_bytes_per_seq=None):
+    """The `config` object of the JSON line, the same for both arms."""
+    slots = cfg.n_sink_heads * (cfg.prompt_len + cfg.sink_budget + cfg.sink_recent) + \
+        (cfg.n_heads - cfg.n_sink_heads) * (cfg.prompt_len + cfg.window)
+    layer_mb = cfg.n_seqs * slots * 512 / 1e6
+    return {"workload": cfg.name, "n_layers": cfg.n_layers, "n_seqs_per_gpu": cfg.n_seqs, "n_heads": cfg.n_heads,
+            "prompt_len": cfg.prompt_len, "image_tokens": cfg.n_img, "compressed_at": cfg.n0, "window": cfg.window,
+            "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent, "sink_heads_per_layer": cfg.n_sink_heads,
+            "kv_dtype": "bf16", "parallelism": f"sequence-sharded x{world}",
+            "l2": f"no flush: a layer's slab ({layer_mb:.0f} MB) is touched once per step and a step touches "
+                  f"{layer_mb * cfg.n_layers / 1e3:.2f} GB, against 126 MB of L2",
+            "kv_bytes_per_seq": cfg.n_layers * slots * 512 if kv_bytes_per_seq is None else kv_bytes_per_seq}
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -172,9 +186,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "n_layers": cfg.n_layers, "n_seqs": cfg.n_seqs, "n_heads": cfg.n_heads,
-                   "prompt_len": cfg.prompt_len, "image_tokens": cfg.n_img, "window": cfg.window,
-                   "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent},
+        "config": config_dict(cfg, args.gpus),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -667,12 +679,7 @@ def run_ours(args, cfg):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": cfg.name, "n_layers": cfg.n_layers, "n_seqs_per_gpu": S, "n_heads": H,
-                       "prompt_len": cfg.prompt_len, "image_tokens": N, "compressed_at": n0, "window": cfg.window,
-                       "sink_budget": cfg.sink_budget, "sink_recent": cfg.sink_recent,
-                       "sink_heads_per_layer": cfg.n_sink_heads, "kv_dtype": "bf16", "parallelism": f"sequence-sharded x{world}",
-                       "l2": "inputs larger than L2 (each layer's slab is >126 MB and is touched once per step)",
-                       "kv_bytes_per_seq": kv_bytes_per_seq},
+            "config": config_dict(cfg, world, kv_bytes_per_seq),
             "sequence_tokens_per_s": value * 2 if S > 1 else value,
             "step_form": "one launch per layer (ssd_append_decode); one_launch = the whole step in one launch",
             "ms_per_step_repeats": repeats,
