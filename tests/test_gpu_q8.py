@@ -127,3 +127,44 @@ def test_q8_unsupported_calls_are_refused():
     cache.set_row_buffer(True)
     assert lib.ssd_cache_set_kv_format(cache._h, 1) == B.SSD_ERR_BAD_STATE
     cache.close()
+
+
+@pytest.mark.parametrize("mode", ["q8", "row_buffer"])
+def test_step_from_host_buffers_in_the_other_modes(mode):
+    """ssd_step_host_layers issues the per-layer calls itself, so it serves the 8-bit format and the row-buffer mode
+    too: same bits as the per-layer calls on device tensors, several steps in a row."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], n_layers=6, n_seqs=2)
+    dev = torch.device("cuda:0")
+    L, n0, nl = cfg.prompt_len, cfg.n0, cfg.n_layers
+    data = [wl.gen_layer(cfg, l, range(cfg.n_seqs), device=dev) for l in range(nl)]
+    labels = np.concatenate([wl.sink_mask(cfg, l) for l in range(nl)])
+    caches = []
+    for _ in range(2):
+        cache = B.SsdCache(B.config_from_workload(cfg), device=dev)
+        if mode == "q8":
+            cache.set_kv_format(1)
+        else:
+            cache.set_row_buffer(True)
+        cache.set_head_labels(labels)
+        for l, (q, k, v, _) in enumerate(data):
+            cache.compress(l, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(cache)
+    dev_cache, host_cache = caches
+    for t in range(n0 + 1, n0 + 6):
+        qs = torch.stack([data[l][0][:, :, t - 1] for l in range(nl)]).contiguous()
+        ks = torch.stack([data[l][1][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        vs = torch.stack([data[l][2][:, :, L + t - 1] for l in range(nl)]).contiguous()
+        want = torch.stack([dev_cache.append_decode(l, ks[l], vs[l], qs[l]) for l in range(nl)]).cpu()
+        hq, hk, hv = (x.cpu().pin_memory() for x in (qs, ks, vs))
+        ho = torch.zeros_like(hq).pin_memory()
+        host_cache.step_host_layers(0, hq, hk, hv, ho)
+        torch.cuda.synchronize()
+        assert torch.equal(ho, want), t
+    for l in range(nl):
+        assert np.array_equal(dev_cache.get_indices(l), host_cache.get_indices(l))
+    if mode == "row_buffer":
+        assert np.allclose(dev_cache.get_scores(2), host_cache.get_scores(2), rtol=0, atol=0)
+    assert dev_cache.device_status() == 0 and host_cache.device_status() == 0
+    for c in caches:
+        c.close()
