@@ -137,12 +137,15 @@ def test_layers_launch_argument_errors():
     c.close()
 
 
-def test_janus7b_whole_step_launch_size_sampled_pairs():
-    """The launch the benchmark times: all 30 layers x 64 sequences x 32 heads of janus7b in one
-    launch.  The oracle recomputes sampled (layer, sequence, head) pairs one by one: their selected
-    sets (exact outside the tie band) and their outputs at three steps."""
+@pytest.mark.parametrize("name,form", [("janus7b", "one_launch"), ("janus7b", "per_layer"), ("janus1b", "per_layer"),
+                                       ("hires7b", "per_layer"), ("hires7b", "one_launch")])
+def test_whole_step_launch_size_sampled_pairs(name, form):
+    """The launches the benchmark times, at every workload's full size (all layers x all sequences x all heads):
+    one launch per layer (ssd_append_decode, the headline form) or the whole step in one launch.  The oracle
+    recomputes sampled (layer, sequence, head) pairs one by one: their selected sets (exact outside the tie
+    band) and their outputs at three steps."""
     from parity_util import MAX_ABS, MEAN_ABS, bf16_to_f64, check_index_sets
-    cfg = wl.CONFIGS["janus7b"]
+    cfg = wl.CONFIGS[name]
     dev = torch.device("cuda:0")
     L, N, n0, W, M, R, H, S, NL = (cfg.prompt_len, cfg.n_img, cfg.n0, cfg.window, cfg.sink_budget, cfg.sink_recent,
                                    cfg.n_heads, cfg.n_seqs, cfg.n_layers)
@@ -150,7 +153,8 @@ def test_janus7b_whole_step_launch_size_sampled_pairs():
     labels = np.stack([wl.sink_mask(cfg, l) for l in range(NL)])
     rng = np.random.default_rng(42)
     sample = {}
-    for i, layer in enumerate((0, 0, 9, 9, 17, 17, 29, 29)):
+    some_layers = sorted({0, NL // 3, (2 * NL) // 3, NL - 1})
+    for i, layer in enumerate(sorted(some_layers * (2 if name != "hires7b" else 1))):
         heads = np.nonzero(labels[layer] == (i % 2))[0]         # alternately a spatial and a semantic head
         sample.setdefault(layer, []).append((int(rng.integers(0, S)), int(rng.choice(heads))))
     cache = B.SsdCache(B.config_from_workload(cfg), n_sink_heads_total=int(labels.sum()), device=dev)
@@ -177,10 +181,14 @@ def test_janus7b_whole_step_launch_size_sampled_pairs():
                     check_index_sets(gidx, sc, oidx, ocnt, sem, n_cand, M)
                 picked[(layer, s, h)] = (qu, ku, vu, sem, gidx, (gidx >= 0).sum(-1).astype(np.int32))
         del q, k, v
-    assert len(picked) == 8
+    assert len(picked) == (8 if name != "hires7b" else 4)
     for i in range(n_steps):
         t = n0 + 1 + i
-        out = bf16_to_f64(cache.append_decode_layers(0, step_in[1][i], step_in[2][i], step_in[0][i]))
+        if form == "one_launch":
+            out = bf16_to_f64(cache.append_decode_layers(0, step_in[1][i], step_in[2][i], step_in[0][i]))
+        else:
+            out = bf16_to_f64(torch.stack([cache.append_decode(l, step_in[1][i, l], step_in[2][i, l], step_in[0][i, l])
+                                           for l in range(NL)]))
         for (layer, s, h), (qu, ku, vu, sem, gidx, gcnt) in picked.items():
             want = oracle.decode_batch(qu[None, None, t - 1], ku[None, None], vu[None, None], sem, gidx, gcnt, L, t, W, M, R)
             err = np.abs(out[layer, s, h] - want[0, 0])
