@@ -1,10 +1,13 @@
 """fp64 CPU oracle for the SSD hot path -- TEST INFRASTRUCTURE ONLY.
 
 Thin ctypes wrapper around ``ssd_oracle.c`` (plain C, double precision, written
-from the paper).  Only the tests, the smoke check and the benchmark's
-CPU-baseline leg may import this package; the CUDA library never does, and this
-package never imports the CUDA library.  bf16 tensors travel as numpy ``uint16``
-bit patterns.
+from the paper), plus a few functions in plain numpy: the buffered variant of the
+method (Algorithm 2), the per-token divergence of two caches (Sec. 3.2) and the
+8-bit K/V extension (E4M3 encode / decode from the format's definition, per-row
+quantisation, attention over dequantised rows).  Only the tests, the smoke check
+and the benchmark's CPU-baseline leg may import this package; the CUDA library
+never does, and this package never imports the CUDA library.  bf16 tensors travel
+as numpy ``uint16`` bit patterns.
 
 Every function cites the passage of the paper it follows in ``ssd_oracle.c``.
 Parity status: all functions are pinned by ``tests/test_oracle_pins.py``
