@@ -215,6 +215,8 @@ int ssd_recompress(ssd_cache *cache, int32_t layer, void *stream);
 /* ssd_recompress for n_layers consecutive layers in one launch (same results, layer by layer): with
  * ssd_append_decode_layers, a buffer cycle of Algorithm 2 is R + 1 launches for all layers.  Layers
  * with an empty buffer and nothing pending are skipped (no launch at all if that is all of them).
+ * With sink_recent = 1 (Algorithm 1 taken literally: a re-selection after every step) no ranking is needed
+ * and a lighter kernel, one warp per (sequence, head), drops the lowest score; same results.
  * SSD_ERR_LIMIT if n_layers > 64. */
 int ssd_recompress_layers(ssd_cache *cache, int32_t first_layer, int32_t n_layers, void *stream);
 int ssd_cache_get_scores(ssd_cache *cache, int32_t layer, float *acc_host);
