@@ -285,7 +285,7 @@ int ssd_step_host(ssd_cache *cache, int32_t layer, const void *q_host, const voi
                   const void *v_new_host, void *out_host, void *stream);
 
 /* The same for n_layers consecutive layers in one call, with the copies running beside the kernels:
- * layers move in groups of 4 (one copy per tensor and group); a group's inputs are copied on a
+ * layers move in groups of 10 (one copy per tensor and group); a group's inputs are copied on a
  * stream of the library's own while the group before it is attended to, and its outputs go back
  * on another while the next group runs (a ring of 3 staging slots inside the cache buffer; the
  * streams and events are created at the first call).

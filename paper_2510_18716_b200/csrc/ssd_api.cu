@@ -18,7 +18,7 @@ static size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 // ssd_step_host_layers moves layers in groups of kHostGroup (one copy per tensor and group: a copy
 // of one layer's 0.5 MB costs about as much in set-up as in transfer) through a ring of kHostSlots
 // staging slots; a slot holds q, k_new, v_new and out of a whole group.
-constexpr int kHostGroup = 4;
+constexpr int kHostGroup = 10;
 constexpr int kHostSlots = 3;
 
 struct Regions {

@@ -195,11 +195,11 @@ def test_step_host_matches_device_path():
 
 
 def test_step_host_layers_matches_device_path():
-    """Fourteen layers (four groups: more than the staging ring holds, the last group short) from
+    """Thirty-four layers (four groups: more than the staging ring holds, the last group short) from
     pinned host arrays in one call, several steps in a row, against per-layer calls on device
     tensors: bit-identical outputs."""
     import dataclasses
-    cfg = dataclasses.replace(wl.CONFIGS["tiny"], n_layers=14, n_seqs=2)
+    cfg = dataclasses.replace(wl.CONFIGS["tiny"], n_layers=34, n_seqs=2)
     dev = torch.device("cuda:0")
     L, n0, nl, steps = cfg.prompt_len, cfg.n0, cfg.n_layers, 5
     data = [wl.gen_layer(cfg, l, range(cfg.n_seqs), device=dev) for l in range(nl)]
@@ -229,7 +229,7 @@ def test_step_host_layers_matches_device_path():
     torch.cuda.synchronize()
     assert host_cache.tokens(2) == host_cache.tokens(0) + 1 and host_cache.tokens(4) == host_cache.tokens(0)
     lib = B.load()
-    assert lib.ssd_step_host_layers(host_cache._h, 13, 2, hq1.data_ptr(), hk1.data_ptr(), hv1.data_ptr(), ho1.data_ptr(),
+    assert lib.ssd_step_host_layers(host_cache._h, 33, 2, hq1.data_ptr(), hk1.data_ptr(), hv1.data_ptr(), ho1.data_ptr(),
                                     None) == B.SSD_ERR_INVALID_ARG
     assert host_cache.device_status() == 0
     for c in caches:
