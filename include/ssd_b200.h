@@ -257,8 +257,9 @@ int ssd_decode_attn_static(ssd_cache *cache, int32_t layer, const void *q, void 
  * row's the softmax weight.
  *   ssd_cache_set_kv_format(cache, 1) switches a cache to that format (0 = bf16, the default) and resets every
  *   layer to the empty state; call it before ssd_compress.  In that format the cache serves ssd_compress,
- *   ssd_append_decode_layers, ssd_append_decode (the same kernel on one layer), ssd_step_host(_layers) and the
- *   inspection calls; ssd_append, ssd_decode_attn, ssd_decode_attn_static and the row-buffer mode return
+ *   ssd_append_decode_layers, ssd_append_decode and ssd_decode_attn (the equal-shares kernel of the bf16 path
+ *   with this format's arithmetic), ssd_step_host(_layers) and the inspection calls; ssd_append (a row is
+ *   quantised by the launch that first attends to it), ssd_decode_attn_static and the row-buffer mode return
  *   SSD_ERR_BAD_STATE (so does switching the format while the row buffer is on, and vice versa).  The device buffer
  *   is sized as for bf16 (ssd_cache_required_bytes); ssd_cache_kv_bytes reports the bytes actually held.
  *   ssd_quantize_rows_e4m3 is the quantiser on its own: rows [n_rows, 128] bf16 -> codes_out [n_rows, 128] uint8 and

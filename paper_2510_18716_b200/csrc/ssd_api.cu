@@ -529,7 +529,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   if (!c || !q || !out) return SSD_ERR_INVALID_ARG;
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
-  if (!c->labels_set || c->kv_q8) return SSD_ERR_BAD_STATE;
+  if (!c->labels_set) return SSD_ERR_BAD_STATE;
   if (c->empty_head(layer, c->t_img[layer], c->sem_tokens(layer))) return SSD_ERR_BAD_STATE;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return SSD_ERR_INVALID_ARG;
   DecodeParams p;
@@ -553,7 +553,7 @@ int ssd_decode_attn(ssd_cache* c, int32_t layer, const void* q, void* out, void*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
-  if (launch_decode(p, st) != cudaSuccess) return SSD_ERR_CUDA;
+  if ((c->kv_q8 ? launch_decode_q8(p, st) : launch_decode(p, st)) != cudaSuccess) return SSD_ERR_CUDA;
   c->last_writer = -1;
   if (c->row_buffer) {
     c->pending[layer] = 1;
@@ -575,8 +575,6 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
        reinterpret_cast<uintptr_t>(v_new)) % 16 != 0)
     return SSD_ERR_INVALID_ARG;
-  if (c->kv_q8)      // 8-bit K/V: the one kernel of that format, on one layer
-    return ssd_append_decode_layers(c, layer, 1, k_new, v_new, q, out, stream);
   if (c->t_img[layer] >= g.max_image_tokens) return SSD_ERR_OVERFLOW;
   const bool scored = c->row_buffer && c->n_sink[layer] > 0;
   if (scored && c->sem_tokens(layer) >= g.sink_recent) return SSD_ERR_OVERFLOW;   // Algorithm 2, overflow branch
@@ -611,7 +609,7 @@ int ssd_append_decode(ssd_cache* c, int32_t layer, const void* k_new, const void
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool timed = (size_t)(2 * c->prof_n + 1) < c->prof_ev.size();
   if (timed) cudaEventRecord(c->prof_ev[2 * c->prof_n], st);
-  if (launch_decode(p, st) != cudaSuccess) {
+  if ((c->kv_q8 ? launch_decode_q8(p, st) : launch_decode(p, st)) != cudaSuccess) {
     c->t_img[layer] -= 1;
     return SSD_ERR_CUDA;
   }

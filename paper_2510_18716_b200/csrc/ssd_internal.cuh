@@ -187,6 +187,7 @@ cudaError_t launch_recompress(const RecompressParams& p, cudaStream_t st);
 cudaError_t launch_quantize_rows(const void* rows, long long n_rows, void* codes, float* scales, cudaStream_t st);
 cudaError_t launch_gather_q8(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st);
+cudaError_t launch_decode_q8(const DecodeParams& p, cudaStream_t st);   // one layer, 8-bit slots (no row-buffer fields)
 int q8_slot_bytes();
 // The same for several layers in one launch: what differs from layer to layer, and the first layer's
 // tables (a layer's tables follow the previous layer's at fixed strides).

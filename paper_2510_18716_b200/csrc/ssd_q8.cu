@@ -11,12 +11,13 @@
 //                              handed out to warps from a counter, as in ssd_decode_layers_kernel; codes are
 //                              widened with cvt.rn.f16x2.e4m3x2 (exact), all arithmetic in float32, the row
 //                              scales applied to the logit and to the softmax weight
+//   ssd_decode_kernel<Q8Slots>   one layer per launch: the equal-shares kernel of ssd_decode_layer.cuh with the
+//                              arithmetic of this format (decode alone, or fused with the append)
 #include <cuda_fp16.h>
 
 #include <atomic>
 
-#include "ssd_internal.cuh"
-#include "ssd_device.cuh"
+#include "ssd_decode_layer.cuh"
 
 namespace ssd {
 
@@ -253,6 +254,76 @@ __device__ __forceinline__ void q8_fold_stage(const Q8Rows& r, int n, int grp, c
   }
 }
 
+// the lane's 16 dimensions of the query row ([16 * l8, 16 * l8 + 16)), widened and scaled
+__device__ __forceinline__ void q8_load_q(const unsigned char* qrow, int l8, float scale_log2, float2 (&q)[8]) {
+  const uint4* qs = reinterpret_cast<const uint4*>(qrow) + 2 * l8;
+  const uint4 qa = qs[0], qb = qs[1];
+  const float2 sc = make_float2(scale_log2, scale_log2);
+  q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
+  q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
+  q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
+  q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
+}
+
+// The newest token: quantise its rows as the caller passed them (lanes 0-15 the K row, 16-31 the V row) and put
+// the slot in its place in the stage and in the slab; later steps read what this step attends to.
+__device__ __forceinline__ void q8_store_new(unsigned char* in_stage, const unsigned char* new_rows, unsigned char* in_slab,
+                                             int lane) {
+  const uint4 raw = reinterpret_cast<const uint4*>(new_rows)[lane];
+  const float scale = row_scale16(raw);
+  const uint2 codes = quantize8(raw, scale);
+  reinterpret_cast<uint2*>(in_stage)[lane] = codes;
+  reinterpret_cast<uint2*>(in_slab)[lane] = codes;
+  if ((lane & 15) == 0) {
+    reinterpret_cast<float*>(in_stage + 256)[lane >> 4] = scale;
+    reinterpret_cast<float*>(in_slab + 256)[lane >> 4] = scale;
+  }
+  __syncwarp();
+}
+
+// lanes 0..7 write the output row: lane l8 holds dimensions [16 * l8, 16 * l8 + 16)
+__device__ __forceinline__ void q8_write_out(unsigned char* out_row, const State& tot, int l8) {
+  const float inv = 1.f / tot.l;
+  uint4* dst = reinterpret_cast<uint4*>(out_row) + 2 * l8;
+  dst[0] = make_uint4(pack_bf16(tot.acc[0], inv), pack_bf16(tot.acc[1], inv), pack_bf16(tot.acc[2], inv),
+                      pack_bf16(tot.acc[3], inv));
+  dst[1] = make_uint4(pack_bf16(tot.acc[4], inv), pack_bf16(tot.acc[5], inv), pack_bf16(tot.acc[6], inv),
+                      pack_bf16(tot.acc[7], inv));
+}
+
+// The 272-byte slot format as the one-layer kernel sees it.
+#ifndef SSD_Q8_LAYER_WARPS
+#define SSD_Q8_LAYER_WARPS 11
+#endif
+struct Q8Slots {
+  static constexpr int kWarps = SSD_Q8_LAYER_WARPS, kStages = ssd::kStages, kChunk = ssd::kChunk;
+  static constexpr int kSlot = kQ8SlotBytes;
+  static constexpr int kNewBytes = 2 * kRowBytes;     // the newest token's bf16 rows travel behind the query row
+  using Rows = Q8Rows;
+  static __device__ __forceinline__ void load_q(const unsigned char* qrow, int l8, float scale_log2, float2 (&q)[8]) {
+    q8_load_q(qrow, l8, scale_log2, q);
+  }
+  static __device__ __forceinline__ void load_stage(const unsigned char* sb, int n, int grp, int l8, Rows& r) {
+    q8_load_stage(sb, n, grp, l8, r);
+  }
+  static __device__ __forceinline__ void fold_stage(const Rows& r, int n, int grp, int, const float2 (&q)[8], State& st,
+                                                    const LogitSink&) {
+    q8_fold_stage(r, n, grp, q, st);
+  }
+  static __device__ __forceinline__ void store_new(unsigned char* in_stage, const unsigned char* new_rows,
+                                                   unsigned char* in_slab, int lane) {
+    q8_store_new(in_stage, new_rows, in_slab, lane);
+  }
+  static __device__ __forceinline__ void post_acc(float* acc128, const State& tot, int l8) {
+    float4* d = reinterpret_cast<float4*>(acc128 + 16 * l8);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) d[j] = make_float4(tot.acc[2 * j].x, tot.acc[2 * j].y, tot.acc[2 * j + 1].x, tot.acc[2 * j + 1].y);
+  }
+  static __device__ __forceinline__ void write_out(__nv_bfloat16* out, const State& tot, int l8) {
+    q8_write_out(reinterpret_cast<unsigned char*>(out), tot, l8);
+  }
+};
+
 // One warp streams a whole head; heads (units, in the order layer, sequence, head) come from a global counter, the
 // next one asked for while the current one streams; its copy pipeline runs on across unit boundaries; the unit
 // ids travel from the warp's producer side to its consumer side through a 4-entry shared-memory FIFO.
@@ -369,13 +440,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(co
     unsigned char* sb = ring + (size_t)stage * kStageBytes;
     if (begin) {
       // the lane's 16 dimensions of the query, widened and scaled
-      const uint4* qs = reinterpret_cast<const uint4*>(sb + kStageQ) + 2 * l8;
-      const uint4 qa = qs[0], qb = qs[1];
-      const float2 sc = make_float2(p.scale_log2, p.scale_log2);
-      q[0] = __fmul2_rn(widen2(qa.x), sc); q[1] = __fmul2_rn(widen2(qa.y), sc);
-      q[2] = __fmul2_rn(widen2(qa.z), sc); q[3] = __fmul2_rn(widen2(qa.w), sc);
-      q[4] = __fmul2_rn(widen2(qb.x), sc); q[5] = __fmul2_rn(widen2(qb.y), sc);
-      q[6] = __fmul2_rn(widen2(qb.z), sc); q[7] = __fmul2_rn(widen2(qb.w), sc);
+      q8_load_q(sb + kStageQ, l8, p.scale_log2, q);
       state_init(st);
       begin = false;
     }
@@ -384,18 +449,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(co
       // slot in its place in the stage and in the slab; later steps read what this step has attended to
       const int s_new = CU.fresh - ci;
       if (s_new >= 0 && s_new < n) {
-        const uint4 raw = reinterpret_cast<const uint4*>(sb + kStageNew)[lane];
-        const float scale = row_scale16(raw);
-        const uint2 codes = quantize8(raw, scale);
-        unsigned char* in_stage = sb + s_new * kQ8SlotBytes;
-        unsigned char* in_slab = const_cast<unsigned char*>(CU.hbase) + (size_t)CU.phys * kQ8SlotBytes;
-        reinterpret_cast<uint2*>(in_stage)[lane] = codes;
-        reinterpret_cast<uint2*>(in_slab)[lane] = codes;
-        if ((lane & 15) == 0) {
-          reinterpret_cast<float*>(in_stage + 256)[lane >> 4] = scale;
-          reinterpret_cast<float*>(in_slab + 256)[lane >> 4] = scale;
-        }
-        __syncwarp();
+        q8_store_new(sb + s_new * kQ8SlotBytes, sb + kStageNew,
+                     const_cast<unsigned char*>(CU.hbase) + (size_t)CU.phys * kQ8SlotBytes, lane);
       }
     }
     Q8Rows rows;
@@ -411,18 +466,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(co
       State tot = st;
       state_merge_lane(tot, 8);
       state_merge_lane(tot, 16);
-      if (grp == 0) {
-        const float inv = 1.f / tot.l;
-        uint32_t o[8];
-#pragma unroll
-        for (int d = 0; d < 8; ++d) {
-          __nv_bfloat162 t = __floats2bfloat162_rn(tot.acc[d].x * inv, tot.acc[d].y * inv);
-          o[d] = *reinterpret_cast<uint32_t*>(&t);
-        }
-        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.out) + CU.row) + 2 * l8;
-        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-      }
+      if (grp == 0) q8_write_out(reinterpret_cast<unsigned char*>(p.out) + CU.row, tot, l8);
       begin = true;
     }
     if (++stage == kStages) { stage = 0; parity ^= 1u; }
@@ -467,6 +511,8 @@ cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st
   count_launch();
   return cudaGetLastError();
 }
+
+cudaError_t launch_decode_q8(const DecodeParams& p, cudaStream_t st) { return launch_decode_format<Q8Slots>(p, st); }
 
 int q8_slot_bytes() { return kQ8SlotBytes; }
 

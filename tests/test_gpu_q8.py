@@ -68,6 +68,10 @@ def _run(cfg, n_layers, seqs, steps, form, sample=None):
             out = cache.append_decode_layers(0, ks, vs, qs)
         else:
             out = torch.stack([cache.append_decode(l, ks[l], vs[l], qs[l]) for l in range(n_layers)])
+            if t == n0 + steps:
+                # attention alone over the store the fused call left behind: same shares, same codes, same bits
+                for l in range(n_layers):
+                    assert torch.equal(cache.decode_attn(l, qs[l]), out[l])
         out = out.float().cpu().numpy().astype(np.float64)
         assert np.isfinite(out).all()
         for (l, s, h) in sample:
@@ -93,19 +97,48 @@ def test_q8_tiny_every_step(form):
     _run(cfg, 2, [0, 1], cfg.n_img - cfg.n0, form)
 
 
-def test_q8_janus7b_slice():
+@pytest.mark.parametrize("form", ["layers", "per_layer"])
+def test_q8_janus7b_slice(form):
     cfg = wl.CONFIGS["janus7b"]
     rng = np.random.default_rng(2)
     sample = [(int(rng.integers(0, 3)), int(rng.integers(0, 4)), int(rng.integers(0, 32))) for _ in range(12)]
-    _run(cfg, 3, [0, 1, 2, 3], 70, "layers", sample)        # past one turn of the 64-slot rings
+    _run(cfg, 3, [0, 1, 2, 3], 70, form, sample)            # past one turn of the 64-slot rings
 
 
-def test_q8_janus7b_launch_size_sampled_pairs():
-    """The launch the benchmark's 8-bit leg times: 30 layers x 64 sequences x 32 heads in one launch."""
+@pytest.mark.parametrize("form", ["layers", "per_layer"])
+def test_q8_janus7b_launch_size_sampled_pairs(form):
+    """The launches the benchmark's 8-bit leg times: 30 layers x 64 sequences x 32 heads, in one launch and as one
+    launch per layer (every share boundary of the full-size layer cuts a head)."""
     cfg = wl.CONFIGS["janus7b"]
     rng = np.random.default_rng(6)
     sample = [(l, int(rng.integers(0, 64)), int(rng.integers(0, 32))) for l in (0, 9, 17, 29) for _ in range(2)]
-    _run(cfg, cfg.n_layers, list(range(cfg.n_seqs)), 3, "layers", sample)
+    _run(cfg, cfg.n_layers, list(range(cfg.n_seqs)), 3, form, sample)
+
+
+def test_q8_every_pair_of_a_full_size_layer():
+    """One janus7b layer at full width (64 sequences: 1628 shares, most heads cut once, some crossing thread
+    blocks), every (sequence, head) of the per-layer form against the one-launch form, which cuts no head: the two
+    differ only in the order of the partial sums, far inside the tolerance of the parity tests."""
+    cfg = wl.CONFIGS["janus7b"]
+    dev = torch.device("cuda:0")
+    L, n0, S = cfg.prompt_len, cfg.n0, cfg.n_seqs
+    caches = []
+    q, k, v, _ = wl.gen_layer(cfg, 0, range(S), device=dev)
+    for _ in range(2):
+        cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1), device=dev)
+        cache.set_kv_format(1)
+        cache.set_head_labels(wl.sink_mask(cfg, 0)[None])
+        cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+        caches.append(cache)
+    for t in range(n0 + 1, n0 + 4):
+        args = (k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous(), q[:, :, t - 1].contiguous())
+        a = caches[0].append_decode(0, *args).float()
+        b = caches[1].append_decode_layers(0, *(x[None] for x in args))[0].float()
+        err = (a - b).abs()
+        assert err.max().item() <= MAX_ABS / 4 and err.mean().item() <= MEAN_ABS / 4, (t, err.max().item())
+    assert caches[0].device_status() == 0
+    for c in caches:
+        c.close()
 
 
 def test_q8_unsupported_calls_are_refused():
@@ -118,7 +151,6 @@ def test_q8_unsupported_calls_are_refused():
     lib, st = B.load(), torch.cuda.current_stream().cuda_stream
     before = B.kernel_launch_count()
     assert lib.ssd_append(cache._h, 0, x.data_ptr(), x.data_ptr(), st) == B.SSD_ERR_BAD_STATE
-    assert lib.ssd_decode_attn(cache._h, 0, x.data_ptr(), x.data_ptr(), st) == B.SSD_ERR_BAD_STATE
     assert lib.ssd_decode_attn_static(cache._h, 0, x.data_ptr(), x.data_ptr(), st) == B.SSD_ERR_BAD_STATE
     assert lib.ssd_cache_set_row_buffer(cache._h, 1) == B.SSD_ERR_BAD_STATE
     assert lib.ssd_cache_set_kv_format(cache._h, 2) == B.SSD_ERR_INVALID_ARG
