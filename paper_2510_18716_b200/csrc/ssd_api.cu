@@ -482,6 +482,7 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
   gp.n_seqs = g.n_seqs; gp.H = g.n_heads; gp.L = g.prompt_len; gp.M = g.sink_budget; gp.n0 = n0;
   gp.static_valid = select ? sv : 0;
   gp.seq_slots = c->seq_slots[layer];
+  gp.after_select = select ? 1 : 0;
   if ((c->kv_q8 ? launch_gather_q8(gp, c->max_slots(), st) : launch_gather(gp, c->max_slots(), st)) != cudaSuccess)
     return SSD_ERR_CUDA;
   c->t_img[layer] = n0;

@@ -4,18 +4,13 @@
 //   gather : copy prompt rows, selected rows and the newest ring rows into the slab
 // The scores themselves (QK^T, softmax, column sums) come from the tensor-core kernel.
 #include "ssd_internal.cuh"
+#include "ssd_device.cuh"
 
 namespace ssd {
 
 namespace {
 
 constexpr int kThreads = 256;
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
 // Selection among few candidates without a radix pass: candidate c is kept iff fewer than k
 // candidates come before it in the order (score descending, then position ascending); its rank is
@@ -48,6 +43,7 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
   __shared__ uint32_t s_gt[kThreads + 1], s_eq[kThreads + 1];
   const int pair = blockIdx.x;
   const int head = pair % p.H;
+  pdl_allow_successor();      // the gather that follows copies what does not depend on this kernel meanwhile
   if (!p.desc[head].w) return;
   const int tid = threadIdx.x;
   // the score row arrives in 4 * n_parts pieces (one per lane quadrant of every thread block that shared the
@@ -164,31 +160,41 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
 }
 
 // ----------------------------------------------------------------------------- gather
-// One warp per destination slot: lanes 0-15 copy the K row, lanes 16-31 the V row.
-__global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams p, int max_slots) {
+// One warp per destination slot, two slots at a time (both rows are on their way before the first is stored):
+// lanes 0-15 copy the K row, lanes 16-31 the V row.  Thread blocks (pair, y < gridDim.y - 1) share the slots that
+// do not depend on the selection (prompt, rings, everything of a spatial head); the blocks of the last y, which
+// are handed out after all the others, copy the static slots of semantic heads once the selection kernel has
+// completed.  Launched as that kernel's programmatic dependent, everything but those last blocks runs beside it.
+__global__ void __launch_bounds__(kThreads) ssd_gather_kernel(const GatherParams p) {
   const int pair = blockIdx.x;
   const int seq = pair / p.H, head = pair - seq * p.H;
   const HeadDesc d = p.desc[head];
-  const int cap = p.L + d.y + d.z;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int ctx = p.L + p.n0;
   uint4* dst0 = p.slab + ((size_t)seq * p.seq_slots + d.x) * kSlotU4;
   const uint4* src = (lane < 16 ? p.k_full : p.v_full) + (size_t)pair * ctx * 16 + (lane & 15);
-  for (int s = blockIdx.y * 8 + warp; s < cap; s += gridDim.y * 8) {
-    int pos = -1;
-    if (s < p.L) {
-      pos = s;
-    } else if (s < p.L + d.y) {
-      int mm = s - p.L;
-      if (d.w && mm < p.static_valid) {
-        int j = p.static_idx[(size_t)pair * p.M + mm];
-        if (j >= 0 && j < p.n0) pos = p.L + j;
-      }
-    } else {
-      int r = s - p.L - d.y;                       // ring slot r holds the newest j = r (mod cap)
-      if (p.n0 - 1 >= r && (p.sem_ring || !d.w)) pos = p.L + ((p.n0 - 1 - r) / d.z) * d.z + r;
-    }
-    if (pos >= 0) dst0[(size_t)s * kSlotU4 + lane] = src[(size_t)pos * 16];
+  const bool selected = blockIdx.y == gridDim.y - 1;
+  int s, end, stride;
+  if (selected) {
+    const bool work = d.w && p.static_valid > 0;
+    if (!work && pair != 0) return;
+    pdl_wait_predecessor();                        // (pair 0 waits in any case: the launch must not complete before
+    if (!work) return;                             // the selection has)
+    s = p.L + warp; end = p.L + p.static_valid; stride = 8;
+  } else {
+    s = blockIdx.y * 8 + warp; end = p.L + d.y + d.z; stride = (gridDim.y - 1) * 8;
+  }
+  for (; s < end; s += 2 * stride) {
+    const int s2 = s + stride;
+    const bool a = gather_slot_selected(p, d, s) == selected;
+    const bool b = s2 < end && gather_slot_selected(p, d, s2) == selected;
+    const int pa = a ? gather_source_row(p, d, pair, s) : -1;
+    const int pb = b ? gather_source_row(p, d, pair, s2) : -1;
+    uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
+    if (pa >= 0) ra = src[(size_t)pa * 16];
+    if (pb >= 0) rb = src[(size_t)pb * 16];
+    if (pa >= 0) dst0[(size_t)s * kSlotU4 + lane] = ra;
+    if (pb >= 0) dst0[(size_t)s2 * kSlotU4 + lane] = rb;
   }
 }
 
@@ -417,10 +423,20 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t st) {
 }
 
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st) {
-  dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
-  ssd_gather_kernel<<<grid, kThreads, 0, st>>>(p, max_slots);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.n_seqs * p.H, (max_slots + 63) / 64 + 1);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = st;
+  // Only behind the selection kernel may the launch start early: behind anything else (the caller's kernel that
+  // produced k_full, say) its first pass could read rows that are not written yet.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.after_select ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, ssd_gather_kernel, p);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_recompress_layers(const RecompressLayersParams& p, cudaStream_t st) {

@@ -120,7 +120,29 @@ struct GatherParams {
   int n_seqs, H, L, M, n0;
   int static_valid;
   int seq_slots;
+  int after_select;          // 1: launched as the programmatic dependent of the selection kernel: the slots that
+                             // do not hold selected tokens are copied while the selection may still be running
 };
+
+#if defined(__CUDACC__)
+// Does slot s of a head hold a token chosen by the selection (a static slot of a semantic head)?
+__device__ __forceinline__ bool gather_slot_selected(const GatherParams& p, const HeadDesc& d, int s) {
+  return d.w && s >= p.L && s < p.L + d.y;
+}
+// Row of k_full / v_full that belongs in slot s of a head; -1: the slot stays empty.
+__device__ __forceinline__ int gather_source_row(const GatherParams& p, const HeadDesc& d, int pair, int s) {
+  if (s < p.L) return s;
+  if (s < p.L + d.y) {
+    const int mm = s - p.L;
+    if (!d.w || mm >= p.static_valid) return -1;
+    const int j = p.static_idx[(size_t)pair * p.M + mm];
+    return (j >= 0 && j < p.n0) ? p.L + j : -1;
+  }
+  const int r = s - p.L - d.y;                   // ring slot r holds the newest j = r (mod capacity)
+  if (p.n0 - 1 >= r && (p.sem_ring || !d.w)) return p.L + ((p.n0 - 1 - r) / d.z) * d.z + r;
+  return -1;
+}
+#endif
 
 struct ScoreParams {
   const __nv_bfloat16* q_obs;  // [n_seqs, H, n_obs, 128]

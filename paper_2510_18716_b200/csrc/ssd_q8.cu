@@ -74,36 +74,45 @@ __global__ void __launch_bounds__(256) ssd_quantize_rows_kernel(const uint4* __r
 }
 
 // ----------------------------------------------------------------------------- gather into 272-byte slots
-// One warp per destination slot: lanes 0-15 quantise the K row, lanes 16-31 the V row.
-__global__ void __launch_bounds__(256) ssd_gather_q8_kernel(const GatherParams p, int max_slots) {
+// One warp per destination slot, two slots at a time: lanes 0-15 quantise the K row, lanes 16-31 the V row.
+// The work is shared out as in ssd_gather_kernel: the thread blocks of the last y copy the static slots of
+// semantic heads once the selection kernel has completed, all others what does not depend on the selection.
+__global__ void __launch_bounds__(256) ssd_gather_q8_kernel(const GatherParams p) {
   const int pair = blockIdx.x;
   const int seq = pair / p.H, head = pair - seq * p.H;
   const HeadDesc d = p.desc[head];
-  const int cap = p.L + d.y + d.z;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int ctx = p.L + p.n0;
   unsigned char* dst0 = reinterpret_cast<unsigned char*>(p.slab) + ((size_t)seq * p.seq_slots + d.x) * kQ8SlotBytes;
   const uint4* src = (lane < 16 ? p.k_full : p.v_full) + (size_t)pair * ctx * 16 + (lane & 15);
-  for (int s = blockIdx.y * 8 + warp; s < cap; s += gridDim.y * 8) {
-    int pos = -1;
-    if (s < p.L) {
-      pos = s;
-    } else if (s < p.L + d.y) {
-      const int mm = s - p.L;
-      if (d.w && mm < p.static_valid) {
-        const int j = p.static_idx[(size_t)pair * p.M + mm];
-        if (j >= 0 && j < p.n0) pos = p.L + j;
-      }
-    } else {
-      const int r = s - p.L - d.y;                 // ring slot r holds the newest j = r (mod cap)
-      if (p.n0 - 1 >= r && (p.sem_ring || !d.w)) pos = p.L + ((p.n0 - 1 - r) / d.z) * d.z + r;
-    }
-    if (pos < 0) continue;                         // the same for the whole warp
-    const uint4 raw = src[(size_t)pos * 16];
+  auto put = [&](int s, const uint4& raw) {        // the whole warp together (the row scale is a warp reduction)
     const float scale = row_scale16(raw);
     unsigned char* dst = dst0 + (size_t)s * kQ8SlotBytes;
     reinterpret_cast<uint2*>(dst)[lane] = quantize8(raw, scale);           // K codes at 0, V codes at 128
     if ((lane & 15) == 0) reinterpret_cast<float*>(dst + 256)[lane >> 4] = scale;
+  };
+  const bool selected = blockIdx.y == gridDim.y - 1;
+  int s, end, stride;
+  if (selected) {
+    const bool work = d.w && p.static_valid > 0;
+    if (!work && pair != 0) return;
+    pdl_wait_predecessor();                        // (pair 0 waits in any case: the launch must not complete before
+    if (!work) return;                             // the selection has)
+    s = p.L + warp; end = p.L + p.static_valid; stride = 8;
+  } else {
+    s = blockIdx.y * 8 + warp; end = p.L + d.y + d.z; stride = (gridDim.y - 1) * 8;
+  }
+  for (; s < end; s += 2 * stride) {
+    const int s2 = s + stride;
+    const bool a = gather_slot_selected(p, d, s) == selected;
+    const bool b = s2 < end && gather_slot_selected(p, d, s2) == selected;
+    const int pa = a ? gather_source_row(p, d, pair, s) : -1;               // the same for the whole warp
+    const int pb = b ? gather_source_row(p, d, pair, s2) : -1;
+    uint4 ra = make_uint4(0, 0, 0, 0), rb = ra;
+    if (pa >= 0) ra = src[(size_t)pa * 16];
+    if (pb >= 0) rb = src[(size_t)pb * 16];
+    if (pa >= 0) put(s, ra);
+    if (pb >= 0) put(s2, rb);
   }
 }
 
@@ -484,10 +493,18 @@ cudaError_t launch_quantize_rows(const void* rows, long long n_rows, void* codes
 }
 
 cudaError_t launch_gather_q8(const GatherParams& p, int max_slots, cudaStream_t st) {
-  dim3 grid(p.n_seqs * p.H, (max_slots + 63) / 64);
-  ssd_gather_q8_kernel<<<grid, 256, 0, st>>>(p, max_slots);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.n_seqs * p.H, (max_slots + 63) / 64 + 1);
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];                     // behind the selection kernel only (see launch_gather)
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = p.after_select ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, ssd_gather_q8_kernel, p);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st) {
