@@ -36,8 +36,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.41e6, "per_layer_of_step": 160.98e6,
-                  "sha256": "4a845e3ac2a81a26e8916864b946d0f3387db3a95adacbf34dc0522cc8e20692"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 162.80e6, "per_layer_of_step": 161.13e6,
+                  "sha256": "8bbb7c57590b461a32911d329cc0deb7535c16b7ef9c181ac65a694f342553b3"}
 
 
 def decode_traffic(cfg):
