@@ -53,8 +53,8 @@ static Regions plan_regions(const ssd_config& c) {
   r.status = off;    off = align_up(off + 132);   // status word, and at +128 the unit counter of the all-layers launch
   r.partial_bytes = (size_t)decode_max_workers() * 2 * kPartialFloats * 4;
   r.partial = off;   off = align_up(off + r.partial_bytes);
-  // scoring: a row per lane quadrant of every thread block that shares a pair's query blocks
-  r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4 * kScoreQuads * kScoreMaxParts;
+  // scoring: two rows (one per half of the query rows) for every thread block that shares a pair's query blocks
+  r.score_bytes = pairs_layer * (size_t)c.max_image_tokens * 4 * kScoreHalves * kScoreMaxParts;
   r.score = off;     off = align_up(off + r.score_bytes);
   r.staging = off;   off = align_up(off + (size_t)kHostSlots * kHostGroup * 4 * pairs_layer * kHeadDim * 2);
   // row-buffer mode (Algorithm 2): accumulated scores and the last decode's logits of the static and
@@ -452,13 +452,13 @@ int ssd_compress(ssd_cache* c, int32_t layer, const void* q_obs, const void* k_f
       sp.n_seqs = g.n_seqs; sp.H = g.n_heads; sp.L = g.prompt_len; sp.n0 = n0; sp.n_obs = n_obs;
       sp.scale_log2 = c->scale * 1.4426950408889634f;
       sp.n_parts = n_parts;
-      if (cudaMemsetAsync(c->d_score(), 0, (size_t)n_parts * g.n_seqs * g.n_heads * kScoreQuads * n0 * 4, st) != cudaSuccess ||
+      if (cudaMemsetAsync(c->d_score(), 0, (size_t)n_parts * g.n_seqs * g.n_heads * kScoreHalves * n0 * 4, st) != cudaSuccess ||
           launch_score(sp, st) != cudaSuccess) {
         cudaGetLastError();
         return SSD_ERR_CUDA;
       }
     } else {
-      if (cudaMemsetAsync(c->d_score(), 0, (size_t)g.n_seqs * g.n_heads * kScoreQuads * n0 * 4, st) != cudaSuccess) return SSD_ERR_CUDA;
+      if (cudaMemsetAsync(c->d_score(), 0, (size_t)g.n_seqs * g.n_heads * kScoreHalves * n0 * 4, st) != cudaSuccess) return SSD_ERR_CUDA;
     }
     SelectParams sl;
     sl.score = c->d_score();
@@ -1015,9 +1015,9 @@ int ssd_cache_get_compress_scores(ssd_cache* c, int32_t layer, float* score_host
   const ssd_config& g = c->cfg;
   if (layer < 0 || layer >= g.n_layers) return SSD_ERR_INVALID_ARG;
   if (c->score_layer != layer || c->score_n0 < 1) return SSD_ERR_BAD_STATE;
-  // a pair's score row is the first of its kScoreQuads rows (the selection has added the others into it)
+  // a pair's score row is the first of its kScoreHalves rows (the selection has added the others into it)
   if (cudaDeviceSynchronize() != cudaSuccess ||
-      cudaMemcpy2D(score_host, (size_t)c->score_n0 * 4, c->d_score(), (size_t)kScoreQuads * c->score_n0 * 4,
+      cudaMemcpy2D(score_host, (size_t)c->score_n0 * 4, c->d_score(), (size_t)kScoreHalves * c->score_n0 * 4,
                    (size_t)c->score_n0 * 4, (size_t)g.n_seqs * g.n_heads, cudaMemcpyDeviceToHost) != cudaSuccess) {
     cudaGetLastError();
     return SSD_ERR_CUDA;

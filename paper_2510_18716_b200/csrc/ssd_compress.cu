@@ -46,16 +46,16 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
   pdl_allow_successor();      // the gather that follows copies what does not depend on this kernel meanwhile
   if (!p.desc[head].w) return;
   const int tid = threadIdx.x;
-  // the score row arrives in 4 * n_parts pieces (one per lane quadrant of every thread block that shared the
-  // pair's query blocks): add them in a fixed order, so the row is reproducible bit for bit
-  float* row = p.score + (size_t)pair * kScoreQuads * p.n0;
+  // the score row arrives in 2 * n_parts pieces (one per half of the query rows, from every thread block that
+  // shared the pair's query blocks): add them in a fixed order, so the row is reproducible bit for bit
+  float* row = p.score + (size_t)pair * kScoreHalves * p.n0;
   {
-    const size_t stride = (size_t)gridDim.x * kScoreQuads * p.n0;
+    const size_t stride = (size_t)gridDim.x * kScoreHalves * p.n0;
     for (int i = tid; i < p.n0; i += kThreads) {
       float s = 0.f;
       for (int part = 0; part < p.n_parts; ++part) {
         const float* r = row + (size_t)part * stride + i;
-        s += (r[0] + r[p.n0]) + (r[2 * (size_t)p.n0] + r[3 * (size_t)p.n0]);
+        s += r[0] + r[p.n0];
       }
       row[i] = s;
     }

@@ -148,8 +148,8 @@ struct ScoreParams {
   const __nv_bfloat16* q_obs;  // [n_seqs, H, n_obs, 128]
   const __nv_bfloat16* k_full; // [n_seqs, H, L + n0, 128]
   const HeadDesc* desc;
-  float* score;                // [n_parts][n_seqs, H][4][n0], zero at launch: row (part, pair, quadrant) gets the
-                               // sums over the query rows of that lane quadrant in the query blocks of that part
+  float* score;                // [n_parts][n_seqs, H][2][n0], zero at launch: row (part, pair, half) gets the sums
+                               // over that half of the query rows of the query blocks of that part
   uint32_t* status;            // device status word (bit 2: a bounded wait of the scoring ran out)
   int n_seqs, H, L, n0, n_obs;
   int n_parts;                 // thread blocks that share the query blocks of one (sequence, head)
@@ -157,8 +157,8 @@ struct ScoreParams {
 };
 
 struct SelectParams {
-  float* score;                // [n_parts][n_seqs, H][4][n0]; a pair's 4 * n_parts rows are first added, in a
-                               // fixed order, into its row (part 0, quadrant 0), which is the pair's score row
+  float* score;                // [n_parts][n_seqs, H][2][n0]; a pair's 2 * n_parts rows are first added, in a
+                               // fixed order, into its row (part 0, half 0), which is the pair's score row
   int n_parts;
   const HeadDesc* desc;
   int32_t* static_idx;         // [n_seqs, H, M]
@@ -187,7 +187,7 @@ cudaError_t launch_append(const AppendParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_slots, cudaStream_t st);
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st);
 constexpr int kScoreMaxParts = 4;
-constexpr int kScoreQuads = 4;   // score rows a scoring thread block keeps per pair: one per TMEM lane quadrant
+constexpr int kScoreHalves = 2;  // score rows a scoring thread block keeps per pair: one per half of a block's queries
 int score_parts(int n_sem_pairs, int n_obs);   // thread blocks per (sequence, head) the scoring kernel should use
 cudaError_t launch_select(const SelectParams& p, cudaStream_t st);
 struct RecompressParams {

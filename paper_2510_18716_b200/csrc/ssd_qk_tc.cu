@@ -8,11 +8,18 @@
 // columns are touched: the prompt's share of the softmax cancels in the ratio.
 // Used by the sink scoring of ssd_compress (Algorithm 1, AttentionScores and running sum): per
 // block of 128 observed queries, a first sweep over the key tiles gives every row its maximum and
-// exp-sum, a second sweep recomputes the tiles, normalises, and adds the columns up.  The sum over
-// the 32 rows of a warp is a shuffle transpose-reduction; each TMEM lane quadrant keeps its own
-// score row in global memory (it stays in L2; every element belongs to one lane of one warp, which
-// adds to it with reductions that return nothing), and the selection adds the rows in a fixed order,
-// so scores are bitwise reproducible from run to run, which it relies on.
+// exp-sum; a second sweep recomputes the tiles TRANSPOSED (S^T = K_tile Q_tile^T: the operands swap
+// roles, the shared-memory tiles are the same), so that a TMEM lane is a key and a thread adds up its
+// key's normalised probabilities over the queries in its own registers: no exchange between lanes.
+// What a query's logits are normalised by, m + log2(exp-sum), then differs from column to column of a
+// thread's accumulator row; it is subtracted by the tensor core: one more MMA step per tile adds the
+// rank-one term 1 (a_1 + a_2 + a_3)^T, where a_1 + a_2 + a_3 is the three-term bf16 expansion of
+// -(m + log2 l) / scale of each query (exact to 2^-24), from two small operand tiles that the epilogue
+// warps write (no-swizzle K-major layout), so the exponent is one multiplication away from the accumulator.
+// The two warps that share a lane quadrant take one half of the queries each and keep a score row
+// each in global memory (it stays in L2; every element belongs to one lane of one warp, which adds
+// to it with reductions that return nothing), and the selection adds the rows in a fixed order, so
+// scores are bitwise reproducible from run to run, which it relies on.
 //
 // A CTA is a pipeline of three roles that meet only at mbarriers:
 //   warp 0, one lane   producer: TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the query tile
@@ -106,7 +113,7 @@ __device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, volatil
 
 // The barriers of a CTA's pipeline, one after another in shared memory; `base` is the address of the first.
 struct PipeBars {
-  uint64_t b[2 + 2 * kStages + 2 * kAccs];
+  uint64_t b[2 + 2 * kStages + 2 * kAccs + 1];
 };
 struct Pipe {
   uint32_t base;
@@ -116,6 +123,8 @@ struct Pipe {
   __device__ __forceinline__ uint32_t empty(int s) const { return base + 16 + 8 * (kStages + s); }
   __device__ __forceinline__ uint32_t acc_full(int a) const { return base + 16 + 8 * (2 * kStages + a); }
   __device__ __forceinline__ uint32_t acc_empty(int a) const { return base + 16 + 8 * (2 * kStages + kAccs + a); }
+  // scoring only: the normalisers of a query block are in their operand tile (one arrival per writing warp)
+  __device__ __forceinline__ uint32_t ext_full() const { return base + 16 + 8 * (2 * kStages + 2 * kAccs); }
 };
 __device__ __forceinline__ Pipe pipe_make(PipeBars& bars, bool init) {
   Pipe p;
@@ -131,6 +140,7 @@ __device__ __forceinline__ Pipe pipe_make(PipeBars& bars, bool init) {
       mbar_init(p.acc_full(a), 1);
       mbar_init(p.acc_empty(a), kEpiWarps);
     }
+    mbar_init(p.ext_full(), kEpiWarps / 2);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   return p;
@@ -178,6 +188,28 @@ __device__ __forceinline__ void mma_tile(uint32_t tmem_d, uint32_t a_s, uint32_t
         "}\n" ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc), "r"(accumulate)
         : "memory");
   }
+}
+// A 128 x 16 bf16 operand without swizzle, K-major, in the canonical layout of 8-row x 16-byte core matrices:
+// [group of 8 rows][half of the 16 elements][row in group][16 bytes], i.e. 256 bytes from one group of rows to
+// the next and 128 bytes between the two core matrices of a group along K.
+constexpr int kExtTileBytes = 128 * 16 * 2;
+constexpr int kExtBytes = 2 * kExtTileBytes;     // the tile of ones, then the tile of normalisers
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr) {
+  const uint32_t lo = ((addr >> 4) & 0x3fffu) | ((uint32_t)(128 >> 4) << 16);
+  const uint32_t hi = (uint32_t)(256 >> 4) | (1u << 14);
+  return ((uint64_t)hi << 32) | lo;
+}
+__device__ __forceinline__ uint32_t ext_row_offset(int row) { return (uint32_t)((row >> 3) * 256 + (row & 7) * 16); }
+// One thread: S[128 x 128] += A_ext B_ext^T, one step of 16 along K.
+__device__ __forceinline__ void mma_ext(uint32_t tmem_d, uint32_t a_s, uint32_t b_s) {
+  const uint64_t da = smem_desc_plain(a_s), db = smem_desc_plain(b_s);
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(tmem_d), "l"(da), "l"(db), "r"(kInstrDesc), "r"(1u)
+      : "memory");
 }
 // The barrier gets one arrival when every tcgen05.mma this thread has issued so far is complete.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -247,15 +279,27 @@ struct Issuer {
   Pipe p;
   volatile int* abort;
   uint32_t q_s, k_s, tmem;
+  uint32_t ext_s = 0;          // scoring: the tile of ones, then the tile of normalisers
   int t = 0, qn = 0;
   __device__ __forceinline__ void query_block() { pipe_wait(p.q_full(), qn & 1, abort); }
-  __device__ __forceinline__ void key_tile() {
+  // scoring: the block's normalisers are written (and visible to the tensor core)
+  __device__ __forceinline__ void normalisers() {
+    pipe_wait(p.ext_full(), qn & 1, abort);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  }
+  // transposed: the accumulator gets S^T (lanes = keys, columns = queries) instead of S
+  __device__ __forceinline__ void key_tile(bool transposed = false) {
     const int s = t % kStages, a = t % kAccs;
     pipe_wait(p.full(s), (t / kStages) & 1, abort);
     pipe_wait(p.acc_empty(a), ((t / kAccs) & 1) ^ 1, abort);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!*abort) {
-      mma_tile(tmem + a * kKeys, q_s, k_s + s * kTileBytes);
+      if (transposed) {
+        mma_tile(tmem + a * kKeys, k_s + s * kTileBytes, q_s);
+        mma_ext(tmem + a * kKeys, ext_s, ext_s + kExtTileBytes);        // minus every query's normaliser
+      } else {
+        mma_tile(tmem + a * kKeys, q_s, k_s + s * kTileBytes);
+      }
       mma_commit(p.empty(s));
       mma_commit(p.acc_full(a));
     }
@@ -444,21 +488,6 @@ ssd_classify_kernel(const ClassifyParams p, int n_row_blocks, const __grid_const
 }
 
 // ----------------------------------------------------------------------------- score
-// Sum over the 32 lanes of a warp of 32 values each: lane j returns the total of value j.
-__device__ __forceinline__ float warp_column_sums(float (&a)[32], int lane) {
-#pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) {
-    const bool up = (lane & s) != 0;
-#pragma unroll
-    for (int i = 0; i < s; ++i) {
-      const float keep = up ? a[i + s] : a[i];
-      const float send = up ? a[i] : a[i + s];
-      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-    }
-  }
-  return a[0];
-}
-
 // The tiles of a scoring CTA, in the order all three roles walk them: for every block of 128
 // observed queries, the key tiles of sweep 1 (from key 0) and then of sweep 2 (from the tile that
 // holds the first image key), both up to the context of the block's last row.
@@ -501,7 +530,11 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
 
   Pipe pipe;
-  const uint32_t q_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe), k_s = q_s + kTileBytes;
+  // the two small operand tiles of the normalisers come first, so that whatever the tensor core reads through
+  // their descriptors lies inside this thread block's own tiles
+  const uint32_t ext_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe);
+  const uint32_t q_s = ext_s + kExtBytes, k_s = q_s + kTileBytes;
+  unsigned char* ext_p = smem + (ext_s - smem_u32(smem));
   const uint32_t tmem = s_tmem;
 
   if (warp == 0) {
@@ -520,13 +553,14 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   } else if (warp == 1) {
     if (lane == 0) {
       Issuer is;
-      is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem;
+      is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem; is.ext_s = ext_s;
       for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
         if (block_owner(r0 / kRows, p.n_parts) != part) continue;
         const ScoreBlock b = score_block(p, r0);
         is.query_block();
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
-        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
+        is.normalisers();
+        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile(true);
         is.end_block();
       }
     }
@@ -535,8 +569,18 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
     const int rl = quad * 32 + lane;                     // row inside a block of queries
     Consumer co;
     co.p = pipe; co.abort = &s_abort; co.tmem_lane = tmem + ((uint32_t)(quad * 32) << 16); co.lane = lane;
-    // this quadrant's score row; the two warps of a quadrant own disjoint keys, a key always the same lane
-    float* my_score = p.score + ((((size_t)part * n_pairs + pair) * kScoreQuads) + quad) * p.n0;
+    // this warp's score row in sweep 2: one per half of a block's queries; a key always belongs to the same lane
+    float* my_score = p.score + ((((size_t)part * n_pairs + pair) * kScoreHalves) + half) * p.n0;
+
+    if (half == 0) {
+      // once: row rl of the tile of ones (1 in the three columns the normalisers use), and the upper half of
+      // row rl of the tile of normalisers, which stays zero
+      uint4* ones = reinterpret_cast<uint4*>(ext_p + ext_row_offset(rl));
+      ones[0] = make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u);
+      ones[8] = make_uint4(0u, 0u, 0u, 0u);
+      reinterpret_cast<uint4*>(ext_p + kExtTileBytes + ext_row_offset(rl))[8] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const float inv_scale = 1.f / p.scale_log2;
 
     int blk = 0;                           // blocks this part has done
     for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
@@ -586,37 +630,60 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
       }
       // the normaliser goes into the exponent: p = 2^(x - (m + log2 l)), one multiplication less per logit
       const float m_l = st.all > 0.f ? st.m + __log2f(st.all) : 1.0e30f;
+      if (half == 0) {
+        // -(m + log2 l) / scale as three bf16 terms (each remainder is exact in float32); rows that do not exist
+        // get a large negative number, their columns are not read
+        const float a = st.all > 0.f ? -m_l * inv_scale : -30000.f;
+        const __nv_bfloat16 a1 = __float2bfloat16_rn(a);
+        const float r1 = a - __bfloat162float(a1);
+        const __nv_bfloat16 a2 = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 a3 = __float2bfloat16_rn(r1 - __bfloat162float(a2));
+        const uint32_t w0 = (uint32_t)__bfloat16_as_ushort(a1) | ((uint32_t)__bfloat16_as_ushort(a2) << 16);
+        const uint32_t w1 = (uint32_t)__bfloat16_as_ushort(a3);
+        *reinterpret_cast<uint4*>(ext_p + kExtTileBytes + ext_row_offset(rl)) = make_uint4(w0, w1, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the tensor core reads it
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pipe.ext_full());
+      }
 
-      // sweep 2: normalised probabilities, column sums over the block's rows
+      // sweep 2, transposed tiles with the normalisers already subtracted: this thread is key k0 + rl of the tile
+      // and sums that key's probabilities over the queries of its half of the block (two groups of 32 columns)
+      const int row_ctx0 = p.L + t_first + r0;          // context of the block's first row; row r sees keys < row_ctx0 + r
+      const int n_rows = b.last - r0 + 1;               // rows of the block that exist
       for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) {
         const uint32_t acc = co.tile();
         bool released = false;
+        const int key_lo = k0 + quad * 32, key = key_lo + lane;
+        float total = 0.f;
 #pragma unroll 1
         for (int cb = 2 * half; cb < 2 * half + 2; ++cb) {
-          const int base = k0 + cb * 32;
-          if (base >= warp_ctx) break;
-          if (base + 32 <= p.L) continue;                 // prompt keys only: not scored
+          const int q0 = cb * 32;                         // first row of this group, inside the block
+          if (q0 >= n_rows) break;                        // the block ends before these rows
+          if (key_lo + 32 <= p.L) break;                  // prompt keys only: not scored
+          if (key_lo >= row_ctx0 + min(q0 + 31, n_rows - 1)) continue;   // no row of the group sees a key of this warp
           float v[32];
-          tmem_ld32(acc + cb * 32, v);
+          tmem_ld32(acc + q0, v);
           if (cb == 2 * half + 1) {
             co.release();
             released = true;
           }
-          if (warp_full && base + 32 <= lo_ctx) {
+          float sum[4] = {0.f, 0.f, 0.f, 0.f};            // four chains of eight additions, joined in a fixed order
+          if (q0 + 32 <= n_rows && key_lo + 32 <= row_ctx0 + q0) {      // every row exists and sees all 32 keys
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = ex2(fmaf(v[j], p.scale_log2, -m_l));
+            for (int j = 0; j < 32; ++j) sum[j & 3] += ex2(v[j] * p.scale_log2);
           } else {
-            const int nv = clamp32(ctx_r - base);
+            // row q0 + j sees this key iff key < row_ctx0 + q0 + j, and exists iff q0 + j < n_rows
+            const int j_lo = max(key - row_ctx0 - q0 + 1, 0), j_hi = min(n_rows - q0, 32);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = j < nv ? ex2(fmaf(v[j], p.scale_log2, -m_l)) : 0.f;
+            for (int j = 0; j < 32; ++j) sum[j & 3] += (j >= j_lo && j < j_hi) ? ex2(v[j] * p.scale_log2) : 0.f;
           }
-          const float col = warp_column_sums(v, lane);
-          const int key = base + lane;
-          // an addition that returns nothing, so nothing waits for it; this lane is the only one that ever
-          // adds to this element, and its additions arrive in program order: the sum is reproducible
-          if (key >= p.L && key < b.ctx_max) atomicAdd(my_score + (key - p.L), col);
+          total += (sum[0] + sum[1]) + (sum[2] + sum[3]);
         }
         if (!released) co.release();
+        // an addition that returns nothing, so nothing waits for it; this lane is the only one that ever
+        // adds to this element, and its additions arrive in program order: the sum is reproducible
+        if (key >= p.L && key < b.ctx_max) atomicAdd(my_score + (key - p.L), total);
       }
       ++blk;
     }
@@ -701,7 +768,7 @@ int score_parts(int n_sem_pairs, int n_obs) {
 }
 
 cudaError_t launch_score(const ScoreParams& p, cudaStream_t st) {
-  const size_t smem = (1 + kStages) * (size_t)kTileBytes + 1024;
+  const size_t smem = (1 + kStages) * (size_t)kTileBytes + kExtBytes + 1024;
   CUtensorMap tq, tk;
   const uint64_t pairs = (uint64_t)p.n_seqs * p.H;
   cudaError_t e = make_tile_map(&tq, p.q_obs, (uint64_t)p.n_obs, pairs);
