@@ -39,6 +39,7 @@
 #include <cuda.h>
 
 #include "ssd_internal.cuh"
+#include "ssd_device.cuh"
 
 namespace ssd {
 
@@ -54,47 +55,9 @@ constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kTcThreads = 64 + kEpiThreads;
 constexpr int kTmemCols = kAccs * kKeys;   // 256: a power of two, as the allocator wants
-constexpr float kNegBig = -1.0e30f;
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 static_assert(kHeadDim == 128, "two 64-element boxes per tile row");
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// ---- mbarriers; every wait is bounded and gives up at once when the CTA's abort flag is up
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
+// ---- every wait on an mbarrier is bounded and gives up at once when the CTA's abort flag is up
 __device__ __forceinline__ bool pipe_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
   if (*abort) return false;
   if (mbar_try_wait(bar, parity)) return true;
