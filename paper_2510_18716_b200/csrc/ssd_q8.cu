@@ -131,14 +131,18 @@ constexpr int kStages = SSD_Q8_STAGES;
 constexpr int kChunk = SSD_Q8_CHUNK;       // slots per stage: 6528 bytes per copy in steady state
 constexpr int kGroups = 4;                 // 8-lane groups of a warp; group g takes slots g, g + 4, ..
 constexpr int kPer = kChunk / kGroups;
-constexpr int kU = kPer % 4 == 0 ? 4 : (kPer % 3 == 0 ? 3 : 2);   // slots a group folds in at a time
+// slots a group folds in at a time, of the kPer it takes from a stage
+template <int kPer>
+struct FoldWidth {
+  static constexpr int value = kPer % 4 == 0 ? 4 : (kPer % 3 == 0 ? 3 : (kPer % 2 == 0 ? 2 : 1));
+};
 constexpr int kRowBytes = kHeadDim * 2;    // a bf16 row of q, k_new, v_new, out
 constexpr int kStageQ = kChunk * kQ8SlotBytes;            // where the query row sits in a stage
 constexpr int kStageNew = kStageQ + kRowBytes;            // and the new token's K and V rows (bf16, as they arrive)
 constexpr int kStageBytes = kStageNew + 2 * kRowBytes;
 constexpr int kRingBytes = kWarps * kStages * kStageBytes;
 constexpr int kQ8SmemBytes = kRingBytes + kWarps * kStages * 8 + kWarps * 4 * 4;
-static_assert(kPer % kU == 0 && kQ8SmemBytes <= 227 * 1024 && kStageBytes % 16 == 0, "stage rings");
+static_assert(kChunk % kGroups == 0 && kQ8SmemBytes <= 227 * 1024 && kStageBytes % 16 == 0, "stage rings");
 
 struct Q8Unit {
   const unsigned char* hbase;   // the head's first slot
@@ -180,12 +184,14 @@ __device__ __forceinline__ void widen4(uint32_t w, float2& lo, float2& hi) {
 
 // The rows of a stage as one lane holds them: slot 4*u + grp, 16 codes of K and of V (dimensions
 // [16*l8, 16*l8 + 16)) and the two row scales.
+template <int kPer>
 struct Q8Rows {
   uint4 k[kPer], v[kPer];
   float ks[kPer], vs[kPer];
 };
 
-__device__ __forceinline__ void q8_load_stage(const unsigned char* __restrict__ sb, int n, int grp, int l8, Q8Rows& r) {
+template <int kPer>
+__device__ __forceinline__ void q8_load_stage(const unsigned char* __restrict__ sb, int n, int grp, int l8, Q8Rows<kPer>& r) {
 #pragma unroll
   for (int u = 0; u < kPer; ++u) {
     const int slot = kGroups * u + grp;
@@ -228,7 +234,9 @@ __device__ __forceinline__ void q8_axpy16(float p, const uint4& v, float2 (&acc)
   }
 }
 
-__device__ __forceinline__ void q8_fold_stage(const Q8Rows& r, int n, int grp, const float2 (&q)[8], State& st) {
+template <int kPer>
+__device__ __forceinline__ void q8_fold_stage(const Q8Rows<kPer>& r, int n, int grp, const float2 (&q)[8], State& st) {
+  constexpr int kU = FoldWidth<kPer>::value;
 #pragma unroll
   for (int s = 0; s < kPer; s += kU) {
     if (kGroups * s >= n) break;
@@ -301,14 +309,15 @@ __device__ __forceinline__ void q8_write_out(unsigned char* out_row, const State
 }
 
 // The 272-byte slot format as the one-layer kernel sees it.
-#ifndef SSD_Q8_LAYER_WARPS
-#define SSD_Q8_LAYER_WARPS 11
-#endif
+// Two shapes.  15 streaming warps and the finisher: 512 threads keep 128 registers each, which stages of 16
+// slots fit; this instance is bound by instruction issue, and the extra warps pay on large layers.  11 warps
+// (384 threads, 168 registers) with stages of 24 slots: fewer, longer shares, better on small layers.
+template <int kWarpsT, int kChunkT>
 struct Q8Slots {
-  static constexpr int kWarps = SSD_Q8_LAYER_WARPS, kStages = ssd::kStages, kChunk = ssd::kChunk;
+  static constexpr int kWarps = kWarpsT, kStages = 2, kChunk = kChunkT;
   static constexpr int kSlot = kQ8SlotBytes;
   static constexpr int kNewBytes = 2 * kRowBytes;     // the newest token's bf16 rows travel behind the query row
-  using Rows = Q8Rows;
+  using Rows = Q8Rows<kChunk / kGroups>;
   static __device__ __forceinline__ void load_q(const unsigned char* qrow, int l8, float scale_log2, float2 (&q)[8]) {
     q8_load_q(qrow, l8, scale_log2, q);
   }
@@ -462,7 +471,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(co
                      const_cast<unsigned char*>(CU.hbase) + (size_t)CU.phys * kQ8SlotBytes, lane);
       }
     }
-    Q8Rows rows;
+    Q8Rows<kPer> rows;
     q8_load_stage(sb, n, grp, l8, rows);
     __syncwarp();          // every lane has its rows in registers: the stage may be refilled
     --ahead;
@@ -529,7 +538,12 @@ cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode_q8(const DecodeParams& p, cudaStream_t st) { return launch_decode_format<Q8Slots>(p, st); }
+cudaError_t launch_decode_q8(const DecodeParams& p, cudaStream_t st) {
+  // measured per-layer steps, ms (15 x 16 against 11 x 24): 308736 slots per layer 0.695 / 0.724, 209920 slots
+  // 0.553 / 0.565, 71680 slots 0.288 / 0.275
+  const long total = (long)p.view.cum[p.view.H] * p.view.n_seqs;
+  return total >= 131072 ? launch_decode_format<Q8Slots<15, 16>>(p, st) : launch_decode_format<Q8Slots<11, 24>>(p, st);
+}
 
 int q8_slot_bytes() { return kQ8SlotBytes; }
 

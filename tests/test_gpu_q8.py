@@ -118,7 +118,7 @@ def test_q8_janus7b_launch_size_sampled_pairs(form):
 def test_q8_every_pair_of_a_full_size_layer():
     """One janus7b layer at full width (64 sequences: 1628 shares, most heads cut once, some crossing thread
     blocks), every (sequence, head) of the per-layer form against the one-launch form, which cuts no head: the two
-    differ only in the order of the partial sums, far inside the tolerance of the parity tests."""
+    differ only in the order of the partial sums: at most one bf16 rounding step per element."""
     cfg = wl.CONFIGS["janus7b"]
     dev = torch.device("cuda:0")
     L, n0, S = cfg.prompt_len, cfg.n0, cfg.n_seqs
@@ -134,8 +134,11 @@ def test_q8_every_pair_of_a_full_size_layer():
         args = (k[:, :, L + t - 1].contiguous(), v[:, :, L + t - 1].contiguous(), q[:, :, t - 1].contiguous())
         a = caches[0].append_decode(0, *args).float()
         b = caches[1].append_decode_layers(0, *(x[None] for x in args))[0].float()
+        # bf16 outputs: the two orders of summation may round an element to neighbouring values (one unit in the last
+        # place, 2^-8 of its magnitude), nothing more
         err = (a - b).abs()
-        assert err.max().item() <= MAX_ABS / 4 and err.mean().item() <= MEAN_ABS / 4, (t, err.max().item())
+        assert bool((err <= torch.clamp(b.abs() * 2.0 ** -7, min=MAX_ABS / 4)).all()), (t, err.max().item())
+        assert err.mean().item() <= MEAN_ABS / 4, (t, err.mean().item())
     assert caches[0].device_status() == 0
     for c in caches:
         c.close()
