@@ -43,7 +43,7 @@ DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.26e6, "per_layer_of_st
 def decode_traffic(cfg):
     import hashlib
     h = hashlib.sha256()
-    for f in ("ssd_decode.cu", "ssd_decode_layer.cuh", "ssd_device.cuh", "ssd_plan.h", "ssd_internal.cuh"):
+    for f in ("ssd_decode.cu", "ssd_decode_layer.cuh", "ssd_decode_step.cuh", "ssd_device.cuh", "ssd_plan.h", "ssd_internal.cuh"):
         with open(os.path.join(ROOT, "paper_2510_18716_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     if h.hexdigest() != DECODE_TRAFFIC["sha256"] or not cfg.name.startswith(DECODE_TRAFFIC["workload"]):
@@ -638,7 +638,7 @@ def run_ours(args, cfg):
                                          "achieved": qbytes / (ms_q[False] * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
                                          "frac": qbytes / (ms_q[False] * 1e-3) / 1e9 / peak, "peak_kind": f"of {peak_kind}",
                                          "bytes_per_launch": qbytes / cfg.n_layers, "traffic": None}},
-              "roofline": {"bound": "hbm", "kernel": "ssd_decode_layers_q8_kernel", "achieved": qbytes / (ms_q[True] * 1e-3) / 1e9,
+              "roofline": {"bound": "hbm", "kernel": "ssd_decode_layers_kernel<Q8Slots<12, 24>>", "achieved": qbytes / (ms_q[True] * 1e-3) / 1e9,
                                       "peak": peak, "unit": "GB/s", "frac": qbytes / (ms_q[True] * 1e-3) / 1e9 / peak,
                                       "peak_kind": f"of {peak_kind}", "bytes_per_launch": qbytes, "traffic": None},
               "device_status": qcache.device_status()}

@@ -7,17 +7,17 @@
 // that appends it), so what later steps read does not depend on when they read it.
 //   ssd_quantize_rows_kernel   the quantiser on its own (parity of the codes, bit for bit)
 //   ssd_gather_q8_kernel       ssd_compress's gather, quantising on the way into the slab
-//   ssd_decode_layers_q8_kernel  fused append + decode attention of every layer in one launch: whole heads
-//                              handed out to warps from a counter, as in ssd_decode_layers_kernel; codes are
-//                              widened with cvt.rn.f16x2.e4m3x2 (exact), all arithmetic in float32, the row
-//                              scales applied to the logit and to the softmax weight
-//   ssd_decode_kernel<Q8Slots>   one layer per launch: the equal-shares kernel of ssd_decode_layer.cuh with the
-//                              arithmetic of this format (decode alone, or fused with the append)
+//   ssd_decode_layers_kernel<Q8Slots<12, 24>>   fused append + decode attention of every layer in one launch: the
+//                              kernel of ssd_decode_step.cuh (whole heads handed out to warps from a counter) with
+//                              the arithmetic of this format: codes are widened with cvt.rn.f16x2.e4m3x2 (exact), all
+//                              arithmetic in float32, the row scales applied to the logit and to the softmax weight
+//   ssd_decode_kernel<Q8Slots<..>>   one layer per launch: the equal-shares kernel of ssd_decode_layer.cuh with the
+//                              same arithmetic (decode alone, or fused with the append)
 #include <cuda_fp16.h>
 
 #include <atomic>
 
-#include "ssd_decode_layer.cuh"
+#include "ssd_decode_step.cuh"
 
 namespace ssd {
 
@@ -118,60 +118,20 @@ __global__ void __launch_bounds__(256) ssd_gather_q8_kernel(const GatherParams p
 
 // ----------------------------------------------------------------------------- decode over 272-byte slots
 #ifndef SSD_Q8_WARPS
-#define SSD_Q8_WARPS 12
-#endif
-#ifndef SSD_Q8_STAGES
-#define SSD_Q8_STAGES 2
+#define SSD_Q8_WARPS 12           // the one-launch step: streaming warps per CTA ...
 #endif
 #ifndef SSD_Q8_CHUNK
-#define SSD_Q8_CHUNK 24
+#define SSD_Q8_CHUNK 24           // ... and slots per stage (6528 bytes per copy in steady state); 2 stages
 #endif
-constexpr int kWarps = SSD_Q8_WARPS;       // streaming warps per CTA, each an independent worker
-constexpr int kStages = SSD_Q8_STAGES;
-constexpr int kChunk = SSD_Q8_CHUNK;       // slots per stage: 6528 bytes per copy in steady state
 constexpr int kGroups = 4;                 // 8-lane groups of a warp; group g takes slots g, g + 4, ..
-constexpr int kPer = kChunk / kGroups;
+
 // slots a group folds in at a time, of the kPer it takes from a stage
 template <int kPer>
 struct FoldWidth {
   static constexpr int value = kPer % 4 == 0 ? 4 : (kPer % 3 == 0 ? 3 : (kPer % 2 == 0 ? 2 : 1));
 };
 constexpr int kRowBytes = kHeadDim * 2;    // a bf16 row of q, k_new, v_new, out
-constexpr int kStageQ = kChunk * kQ8SlotBytes;            // where the query row sits in a stage
-constexpr int kStageNew = kStageQ + kRowBytes;            // and the new token's K and V rows (bf16, as they arrive)
-constexpr int kStageBytes = kStageNew + 2 * kRowBytes;
-constexpr int kRingBytes = kWarps * kStages * kStageBytes;
-constexpr int kQ8SmemBytes = kRingBytes + kWarps * kStages * 8 + kWarps * 4 * 4;
-static_assert(kChunk % kGroups == 0 && kQ8SmemBytes <= 227 * 1024 && kStageBytes % 16 == 0, "stage rings");
 
-struct Q8Unit {
-  const unsigned char* hbase;   // the head's first slot
-  size_t row;                   // byte offset of the head's row in q, k_new, v_new and out
-  int vh;                       // slots that hold a token
-  int pv, sv;                   // of which prompt slots and static slots (the rest is the ring)
-  int y;                        // static capacity
-  int fresh, phys;              // valid-slot index of the token being appended, and its slot in the head
-  int contig;
-};
-
-__device__ __forceinline__ void q8_unit_load(const DecodeLayersParams& p, int u, Q8Unit& U) {
-  const int pairs = p.n_seqs * p.H;
-  const int layer = u / pairs, pair = u - layer * pairs;
-  const int seq = pair / p.H, head = pair - seq * p.H;
-  const LayerState& ls = p.layer[layer];
-  const HeadDesc d = __ldg(ls.desc + head);
-  const int r = ls.new_j % d.z;
-  U.pv = ls.prompt_valid;
-  U.sv = d.w ? ls.static_valid : 0;
-  U.y = d.y;
-  U.vh = U.pv + U.sv + (ls.t_img < d.z ? ls.t_img : d.z);
-  U.fresh = U.pv + U.sv + r;
-  U.phys = p.L + d.y + r;
-  U.contig = (U.pv == p.L && U.sv == d.y) ? 1 : 0;
-  U.hbase = reinterpret_cast<const unsigned char*>(p.slab) +
-            ((size_t)ls.first_slot + (size_t)seq * ls.seq_slots + d.x) * kQ8SlotBytes;
-  U.row = ((size_t)layer * pairs + pair) * kRowBytes;
-}
 
 // 4 codes (one 32-bit word) -> 4 floats, exactly
 __device__ __forceinline__ void widen4(uint32_t w, float2& lo, float2& hi) {
@@ -317,6 +277,8 @@ struct Q8Slots {
   static constexpr int kWarps = kWarpsT, kStages = 2, kChunk = kChunkT;
   static constexpr int kSlot = kQ8SlotBytes;
   static constexpr int kNewBytes = 2 * kRowBytes;     // the newest token's bf16 rows travel behind the query row
+  static constexpr bool kScores = false;              // no row-buffer modes in this format
+  static_assert(!kScores, "the one-launch step of this format keeps no score rows");
   using Rows = Q8Rows<kChunk / kGroups>;
   static __device__ __forceinline__ void load_q(const unsigned char* qrow, int l8, float scale_log2, float2 (&q)[8]) {
     q8_load_q(qrow, l8, scale_log2, q);
@@ -342,154 +304,6 @@ struct Q8Slots {
   }
 };
 
-// One warp streams a whole head; heads (units, in the order layer, sequence, head) come from a global counter, the
-// next one asked for while the current one streams; its copy pipeline runs on across unit boundaries; the unit
-// ids travel from the warp's producer side to its consumer side through a 4-entry shared-memory FIFO.
-__global__ void __launch_bounds__(kWarps * 32, 1) ssd_decode_layers_q8_kernel(const __grid_constant__ DecodeLayersParams p) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int grp = lane >> 3, l8 = lane & 7;
-  const uint32_t FULL = 0xffffffffu;
-  unsigned char* ring = smem + (size_t)warp * kStages * kStageBytes;
-  const uint32_t ring_s = smem_u32(ring);
-  const uint32_t bar0 = smem_u32(smem + kRingBytes) + (uint32_t)warp * kStages * 8;
-  volatile int* fifo = reinterpret_cast<volatile int*>(smem + kRingBytes + kWarps * kStages * 8) + warp * 4;
-  if (lane == 0) {
-#pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
-    mbar_init_fence();
-  }
-  __syncwarp();
-  const int n_units = p.n_layers * p.n_seqs * p.H;
-
-  int raw_next = 0;
-  auto ask = [&]() {
-    if (lane == 0) raw_next = (int)atomicAdd(p.work, 1u);
-  };
-  ask();
-  int u = __shfl_sync(FULL, raw_next, 0);
-  if (u >= n_units) return;
-  ask();
-
-  Q8Unit PU, CU;               // the producer's and the consumer's current head
-  int pi = 0, ci = 0;          // and their positions in it
-  int produced = 0, consumed = 0, ahead = 0;
-  bool feeding = true;
-  q8_unit_load(p, u, PU);
-  if (lane == 0) fifo[0] = u;
-  produced = 1;
-  __syncwarp();
-
-  // Lane 0 starts the copies of the producer's next chunk into `stage`; every lane advances.
-  auto issue = [&](int stage) {
-    const int n = PU.vh - pi < kChunk ? PU.vh - pi : kChunk;
-    if (lane == 0) {
-      const bool begin = pi == 0;
-      const uint32_t dst = ring_s + (uint32_t)stage * kStageBytes, bar = bar0 + 8 * stage;
-      const bool has_fresh = PU.fresh >= pi && PU.fresh < pi + n;
-      // order the warp's reads (and the writes of a quantised row) of this stage before the asynchronous writes
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_expect_tx(bar, (uint32_t)(n * kQ8SlotBytes + (begin ? kRowBytes : 0) + (has_fresh ? 2 * kRowBytes : 0)));
-      if (PU.contig) {
-        bulk_g2s(dst, PU.hbase + (size_t)pi * kQ8SlotBytes, (uint32_t)n * kQ8SlotBytes, bar);
-      } else {
-        const int l0[3] = {0, PU.pv, PU.pv + PU.sv};          // logical start of each run
-        const int l1[3] = {PU.pv, PU.pv + PU.sv, PU.vh};      // and end
-        const int p0[3] = {0, p.L, p.L + PU.y};               // physical start
-#pragma unroll
-        for (int r = 0; r < 3; ++r) {
-          const int lo = pi > l0[r] ? pi : l0[r], hi = pi + n < l1[r] ? pi + n : l1[r];
-          if (hi > lo)
-            bulk_g2s(dst + (uint32_t)(lo - pi) * kQ8SlotBytes, PU.hbase + (size_t)(p0[r] + lo - l0[r]) * kQ8SlotBytes,
-                     (uint32_t)(hi - lo) * kQ8SlotBytes, bar);
-        }
-      }
-      // the slot of the token being appended holds stale codes: its rows come from the caller, unquantised
-      if (has_fresh) {
-        bulk_g2s(dst + kStageNew, p.k_new + PU.row, kRowBytes, bar);
-        bulk_g2s(dst + kStageNew + kRowBytes, p.v_new + PU.row, kRowBytes, bar);
-      }
-      if (begin) bulk_g2s(dst + kStageQ, p.q + PU.row, kRowBytes, bar);
-    }
-    pi += n;
-    ++ahead;
-    if (pi == PU.vh) {                   // on to the unit asked for earlier, and ask for the one after
-      const int nu = __shfl_sync(FULL, raw_next, 0);
-      if (nu < n_units) {
-        ask();
-        q8_unit_load(p, nu, PU);
-        pi = 0;
-        if (lane == 0) fifo[produced & 3] = nu;
-        ++produced;
-        __syncwarp();
-      } else {
-        feeding = false;
-      }
-    }
-  };
-
-#pragma unroll 1
-  for (int s = 0; s < kStages && feeding; ++s) issue(s);
-
-  int stage = 0;
-  uint32_t parity = 0;
-  float2 q[8];
-  State st;
-  bool begin = true;
-
-#pragma unroll 1
-  for (;;) {
-    if (begin) {
-      if (consumed == produced) break;
-      q8_unit_load(p, fifo[consumed & 3], CU);
-      ++consumed;
-      ci = 0;
-    }
-    const int n = CU.vh - ci < kChunk ? CU.vh - ci : kChunk;
-    if (!mbar_wait(bar0 + 8 * stage, parity)) {
-      // give up: flag it, let the copies still in flight land (bounded), and leave
-      if (lane == 0) atomicOr(p.status, 1u);
-      for (int k = 0; k < ahead; ++k) {
-        mbar_wait(bar0 + 8 * stage, parity);
-        if (++stage == kStages) { stage = 0; parity ^= 1u; }
-      }
-      return;
-    }
-    unsigned char* sb = ring + (size_t)stage * kStageBytes;
-    if (begin) {
-      // the lane's 16 dimensions of the query, widened and scaled
-      q8_load_q(sb + kStageQ, l8, p.scale_log2, q);
-      state_init(st);
-      begin = false;
-    }
-    {
-      // the chunk that carries the newest token: quantise its rows (lanes 0-15 the K row, 16-31 the V row), put the
-      // slot in its place in the stage and in the slab; later steps read what this step has attended to
-      const int s_new = CU.fresh - ci;
-      if (s_new >= 0 && s_new < n) {
-        q8_store_new(sb + s_new * kQ8SlotBytes, sb + kStageNew,
-                     const_cast<unsigned char*>(CU.hbase) + (size_t)CU.phys * kQ8SlotBytes, lane);
-      }
-    }
-    Q8Rows<kPer> rows;
-    q8_load_stage(sb, n, grp, l8, rows);
-    __syncwarp();          // every lane has its rows in registers: the stage may be refilled
-    --ahead;
-    if (feeding) issue(stage);
-    q8_fold_stage(rows, n, grp, q, st);
-    ci += n;
-    if (ci == CU.vh) {
-      // the head is complete: merge the four groups and write the output row (lane l8 of group 0 holds
-      // dimensions [16 * l8, 16 * l8 + 16))
-      State tot = st;
-      state_merge_lane(tot, 8);
-      state_merge_lane(tot, 16);
-      if (grp == 0) q8_write_out(reinterpret_cast<unsigned char*>(p.out) + CU.row, tot, l8);
-      begin = true;
-    }
-    if (++stage == kStages) { stage = 0; parity ^= 1u; }
-  }
-}
 
 }  // namespace
 
@@ -517,25 +331,7 @@ cudaError_t launch_gather_q8(const GatherParams& p, int max_slots, cudaStream_t 
 }
 
 cudaError_t launch_decode_layers_q8(const DecodeLayersParams& p, cudaStream_t st) {
-  static std::atomic<int> n_sm[64] = {};   // 0 = this device is not set up yet
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  const bool cached = dev >= 0 && dev < 64;
-  int sms = cached ? n_sm[dev].load(std::memory_order_acquire) : 0;
-  if (sms == 0) {
-    e = cudaFuncSetAttribute(ssd_decode_layers_q8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQ8SmemBytes);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    if (cached) n_sm[dev].store(sms, std::memory_order_release);
-  }
-  const long units = (long)p.n_layers * p.n_seqs * p.H;
-  if (units < 1 || units > 0x3fffffffL || p.n_layers > kMaxLayersPerLaunch) return cudaErrorInvalidValue;
-  const long want = (units + kWarps - 1) / kWarps;
-  const int grid = (int)(want < sms ? want : sms);
-  ssd_decode_layers_q8_kernel<<<grid, kWarps * 32, kQ8SmemBytes, st>>>(p);
-  count_launch();
-  return cudaGetLastError();
+  return launch_decode_step_format<Q8Slots<SSD_Q8_WARPS, SSD_Q8_CHUNK>>(p, st);
 }
 
 cudaError_t launch_decode_q8(const DecodeParams& p, cudaStream_t st) {
