@@ -36,8 +36,8 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # 4 layers; every layer moves the same bytes, so a launch over n layers moves n times that).
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
-DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.26e6, "per_layer_of_step": 160.96e6,
-                  "sha256": "4d8dca45d7bdaa9eeaabb48a6c36630c5e5d75d177d958c341564d048e6368e3"}
+DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.34e6, "per_layer_of_step": 160.74e6,
+                  "sha256": "4812782dac66f0d623d75ed785ee201fe14e4eecc0eb194fef413b2ef52e37f3"}
 
 
 def decode_traffic(cfg):
