@@ -33,6 +33,60 @@ __device__ __forceinline__ void rank_select(const uint32_t* bits, const int* pos
   }
 }
 
+// Radix-select helpers shared by the selection and the re-selection: one digit of 8 bits per pass.
+// hist[b] += candidates of this thread's value with digit b; lanes of a warp that hold the same digit add once
+// (scores of one head share their leading digits, so most of a warp lands in one or two bins).
+__device__ __forceinline__ void hist_add(uint32_t* hist, bool take, uint32_t digit) {
+  const unsigned active = __ballot_sync(0xffffffffu, take);
+  if (!take) return;
+  const unsigned same = __match_any_sync(active, digit);
+  if ((int)(threadIdx.x & 31) == __ffs(same) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(same));
+}
+// Run by warp 0 after a pass: the highest bin b with (candidates in bins > b) < need <= (candidates in bins >= b);
+// returns it and takes the candidates above it off `need`.  Lane l owns bins [8l, 8l + 8).
+__device__ __forceinline__ int pick_bin(const uint32_t* hist, uint32_t& need, int lane) {
+  uint32_t own[8], t = 0u;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { own[j] = hist[8 * lane + j]; t += own[j]; }
+  uint32_t incl = t;                                   // sum over lanes >= this one
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t o = __shfl_down_sync(0xffffffffu, incl, off);
+    if (lane + off < 32) incl += o;
+  }
+  const unsigned ok = __ballot_sync(0xffffffffu, incl >= need);
+  const int owner = ok ? 31 - __clz(ok) : 0;          // (never empty: need <= the candidates that are left)
+  int bin = 0;
+  uint32_t left = need;
+  if (lane == owner) {
+    uint32_t cum = incl - t;                           // candidates in the bins of higher lanes
+    bin = 8 * lane + 7;
+    for (; bin > 8 * lane; --bin) {
+      if (cum + own[bin - 8 * lane] >= need) break;
+      cum += own[bin - 8 * lane];
+    }
+    left = need - cum;
+  }
+  need = __shfl_sync(0xffffffffu, left, owner);
+  return __shfl_sync(0xffffffffu, bin, owner);
+}
+// Exclusive prefix sums over the thread block of two counters per thread (kThreads = 8 warps); s_w: 2 x 8 words.
+__device__ __forceinline__ void block_prefix2(uint32_t& a, uint32_t& b, uint32_t (*s_w)[8]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t ia = a, ib = b;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t oa = __shfl_up_sync(0xffffffffu, ia, off), ob = __shfl_up_sync(0xffffffffu, ib, off);
+    if (lane >= off) { ia += oa; ib += ob; }
+  }
+  if (lane == 31) { s_w[0][warp] = ia; s_w[1][warp] = ib; }
+  __syncthreads();
+  uint32_t ba = 0u, bb = 0u;
+  for (int w = 0; w < warp; ++w) { ba += s_w[0][w]; bb += s_w[1][w]; }
+  a = ba + ia - a;
+  b = bb + ib - b;
+}
+
 // ----------------------------------------------------------------------------- select
 // One CTA per (sequence, semantic head): radix-select the k-th largest score (scores are
 // non-negative floats, so their bit patterns order like unsigned integers), then emit, in
@@ -40,7 +94,7 @@ __device__ __forceinline__ void rank_select(const uint32_t* bits, const int* pos
 __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams p) {
   __shared__ uint32_t s_hist[256];
   __shared__ uint32_t s_prefix, s_need;
-  __shared__ uint32_t s_gt[kThreads + 1], s_eq[kThreads + 1];
+  __shared__ uint32_t s_scan[2][8];
   const int pair = blockIdx.x;
   const int head = pair % p.H;
   pdl_allow_successor();      // the gather that follows copies what does not depend on this kernel meanwhile
@@ -100,20 +154,19 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
     __syncthreads();
     const uint32_t prefix = s_prefix;
     const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-    for (int i = tid; i < n; i += kThreads) {
-      uint32_t b = sc[i];
-      if ((b & mask) == prefix) atomicAdd(&s_hist[(b >> shift) & 255u], 1u);
+    for (int i0 = 0; i0 < n; i0 += kThreads) {         // every thread takes part in every round (warp votes inside)
+      const int i = i0 + tid;
+      const uint32_t b = i < n ? sc[i] : 0u;
+      hist_add(s_hist, i < n && (b & mask) == prefix, (b >> shift) & 255u);
     }
     __syncthreads();
-    if (tid == 0) {
-      uint32_t need = s_need, cum = 0u;
-      int bin = 255;
-      for (; bin > 0; --bin) {
-        if (cum + s_hist[bin] >= need) break;
-        cum += s_hist[bin];
+    if (tid < 32) {
+      uint32_t need = s_need;
+      const int bin = pick_bin(s_hist, need, tid);
+      if (tid == 0) {
+        s_need = need;
+        s_prefix = prefix | ((uint32_t)bin << shift);
       }
-      s_need = need - cum;
-      s_prefix = prefix | ((uint32_t)bin << shift);
     }
     __syncthreads();
   }
@@ -129,18 +182,8 @@ __global__ void __launch_bounds__(kThreads) ssd_select_kernel(const SelectParams
     cg += v > thr;
     ce += v == thr;
   }
-  s_gt[tid + 1] = cg;
-  s_eq[tid + 1] = ce;
-  if (tid == 0) { s_gt[0] = 0u; s_eq[0] = 0u; }
-  __syncthreads();
-  if (tid == 0) {
-    for (int i = 1; i <= kThreads; ++i) {
-      s_gt[i] += s_gt[i - 1];
-      s_eq[i] += s_eq[i - 1];
-    }
-  }
-  __syncthreads();
-  uint32_t g_before = s_gt[tid], e_before = s_eq[tid];
+  uint32_t g_before = cg, e_before = ce;          // candidates above / equal to the threshold in earlier segments
+  block_prefix2(g_before, e_before, s_scan);
   float* acc = acc_row;
   for (int i = a; i < b; ++i) {
     uint32_t v = sc[i];
@@ -252,20 +295,19 @@ __device__ __forceinline__ void recompress_pair(const RecompressParams& p, int p
     __syncthreads();
     const uint32_t prefix = s_prefix;
     const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-    for (int i = tid; i < n; i += kThreads) {
-      const uint32_t b = bits[i];
-      if ((b & mask) == prefix) atomicAdd(&s_hist[(b >> shift) & 255u], 1u);
+    for (int i0 = 0; i0 < n; i0 += kThreads) {
+      const int i = i0 + tid;
+      const uint32_t b = i < n ? bits[i] : 0u;
+      hist_add(s_hist, i < n && (b & mask) == prefix, (b >> shift) & 255u);
     }
     __syncthreads();
-    if (tid == 0) {
-      uint32_t need = s_need, cum = 0u;
-      int bin = 255;
-      for (; bin > 0; --bin) {
-        if (cum + s_hist[bin] >= need) break;
-        cum += s_hist[bin];
+    if (tid < 32) {
+      uint32_t need = s_need;
+      const int bin = pick_bin(s_hist, need, tid);
+      if (tid == 0) {
+        s_need = need;
+        s_prefix = prefix | ((uint32_t)bin << shift);
       }
-      s_need = need - cum;
-      s_prefix = prefix | ((uint32_t)bin << shift);
     }
     __syncthreads();
   }
