@@ -250,19 +250,22 @@ struct Issuer {
     pipe_wait(p.ext_full(), qn & 1, abort);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
-  // transposed: the accumulator gets S^T (lanes = keys, columns = queries) instead of S
-  __device__ __forceinline__ void key_tile(bool transposed = false) {
+  // transposed: the accumulator gets S^T (lanes = keys, columns = queries) instead of S, minus every query's
+  // normaliser.  first: the block's first such tile; its eight steps over the head dimension do not need the
+  // normalisers and are issued before the wait for them, so the tensor core works while the epilogue warps finish
+  // the first sweep.
+  __device__ __forceinline__ void key_tile(bool transposed = false, bool first = false) {
     const int s = t % kStages, a = t % kAccs;
     pipe_wait(p.full(s), (t / kStages) & 1, abort);
     pipe_wait(p.acc_empty(a), ((t / kAccs) & 1) ^ 1, abort);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!*abort) {
-      if (transposed) {
-        mma_tile(tmem + a * kKeys, k_s + s * kTileBytes, q_s);
-        mma_ext(tmem + a * kKeys, ext_s, ext_s + kExtTileBytes);        // minus every query's normaliser
-      } else {
-        mma_tile(tmem + a * kKeys, q_s, k_s + s * kTileBytes);
-      }
+      if (transposed) mma_tile(tmem + a * kKeys, k_s + s * kTileBytes, q_s);
+      else mma_tile(tmem + a * kKeys, q_s, k_s + s * kTileBytes);
+    }
+    if (first) normalisers();
+    if (!*abort) {
+      if (transposed) mma_ext(tmem + a * kKeys, ext_s, ext_s + kExtTileBytes);
       mma_commit(p.empty(s));
       mma_commit(p.acc_full(a));
     }
@@ -522,8 +525,7 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
         const ScoreBlock b = score_block(p, r0);
         is.query_block();
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
-        is.normalisers();
-        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile(true);
+        for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile(true, k0 == b.k_first2);
         is.end_block();
       }
     }
