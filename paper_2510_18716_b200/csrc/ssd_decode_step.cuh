@@ -1,18 +1,21 @@
+// A whole decode step (every layer's fused append + attention) in ONE launch, written once for every slot
+// format (the policy class F of ssd_decode_layer.cuh).
+//
+// With all layers in one launch there are tens of thousands of heads to go round, so no head needs to
+// be cut: the unit of work is one whole head of one (layer, sequence), units are handed out in stream
+// order from a global counter to whichever warp asks next (warps on slower SMs simply take fewer), and a
+// head is finished in the registers of the warp that streamed it.  No partials, no mailboxes, no
+// finisher, no barrier after start-up.  A warp's copy pipeline runs on across unit boundaries: the next
+// unit is claimed while the current one streams, and its first chunks are in flight before the current
+// head's arithmetic ends.  In the row-buffer modes (formats with F::kScores) the warp that streamed a
+// semantic head also adds the step's attention weights to the head's scores (Algorithm 2) or, with a
+// buffer of one token, re-selects on the spot (kEvict: Algorithm 1 taken literally).
 #pragma once
 
 #include "ssd_decode_layer.cuh"
 
 namespace ssd {
 
-// A whole decode step (every layer's fused append + attention) in ONE launch, written once for every slot format
-// (the policy class F of ssd_decode_layer.cuh).
-// Fused append + decode of every layer.  With all layers in one launch there are tens of thousands
-// of heads to go round, so no head needs to be cut: the unit of work is one whole head of one
-// (layer, sequence), units are handed out in stream order from a global counter to whichever warp
-// asks next (warps on slower SMs simply take fewer), and a head is finished in the registers of the
-// warp that streamed it.  No partials, no mailboxes, no finisher, no barrier after start-up.  A
-// warp's copy pipeline runs on across unit boundaries: the next unit is claimed while the current
-// one streams, and its first chunks are in flight before the current head's arithmetic ends.
 struct Unit {
   const unsigned char* hbase;   // the head's first slot
   size_t row;                   // byte offset of the head's row in q, k_new, v_new (and out)
