@@ -387,6 +387,30 @@ def test_compress_scores_elementwise(name, layer, n_seqs):
     cache.close()
 
 
+def test_compress_scores_with_large_logits():
+    """Queries eight times larger (an exact scaling in bf16): row maxima of several hundred in base-2 units, so
+    the normalisers the second sweep subtracts are large numbers and most probabilities underflow.  The score rows
+    must still match the oracle element by element and contain nothing that is not a finite non-negative number."""
+    cfg = wl.CONFIGS["janus1b"]
+    dev = torch.device("cuda:0")
+    L, n0, M, R, H, layer, n_seqs = cfg.prompt_len, cfg.n0, cfg.sink_budget, cfg.sink_recent, cfg.n_heads, 3, 2
+    labels = wl.sink_mask(cfg, layer)
+    cache = B.SsdCache(B.config_from_workload(cfg, n_layers=1, n_seqs=n_seqs), device=dev)
+    cache.set_head_labels(labels)
+    q, k, v, _ = wl.gen_layer(cfg, layer, list(range(n_seqs)), device=dev)
+    q = (q.float() * 8.0).to(torch.bfloat16)
+    cache.compress(0, q[:, :, :n0].contiguous(), k[:, :, : L + n0].contiguous(), v[:, :, : L + n0].contiguous(), n0)
+    got = cache.get_compress_scores(0, n0)
+    assert cache.device_status() == 0
+    sem = labels[None, :].repeat(n_seqs, 0).astype(np.uint8)
+    want, _, _ = oracle.select_batch(wl.to_u16(q[:, :, :n0]), wl.to_u16(k[:, :, : L + n0]), sem, L, n0, M, R)
+    for h in range(H):
+        if labels[h]:
+            assert np.isfinite(got[:, h]).all() and (got[:, h] >= 0).all()
+            assert np.allclose(got[:, h], want[:, h], rtol=2e-4, atol=1e-7), (h, np.abs(got[:, h] - want[:, h]).max())
+    cache.close()
+
+
 def test_exact_ties_on_the_radix_path_select_the_lowest_indices():
     """Algorithm 1, IndicesOfTopM with the lowest-index tie rule, where the selection radix-selects the
     threshold (more than 1024 candidates): with no observed step every score is zero, all candidates tie,
