@@ -110,6 +110,10 @@ __device__ __forceinline__ Pipe pipe_make(PipeBars& bars, bool init) {
 }
 
 // ---- operand tiles
+// Bring a tensor map (a kernel parameter) towards the TMA unit before its first use.
+__device__ __forceinline__ void prefetch_map(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 // One box of a tile: rows [y, y + 128) x elements [x, x + 64) of unit z of a [units, rows, 128] bf16
 // tensor.  x is 0 or 64 (128 bytes), so the copy starts on the boundary the TMA unit wants.
 __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
@@ -375,6 +379,10 @@ ssd_classify_kernel(const ClassifyParams p, int n_row_blocks, const __grid_const
   const int last_row = min(r0 + kRows, p.N) - 1;
   const int n_tiles = last_row / kKeys + 1;   // keys 0 .. last_row
 
+  if (tid == 0) {                      // while the thread block sets itself up
+    prefetch_map(&tq);
+    prefetch_map(&tk);
+  }
   Pipe pipe;
   const uint32_t q_s = cta_setup(smem, s_bars, &s_tmem, &s_abort, pipe), k_s = q_s + kTileBytes;
   const uint32_t tmem = s_tmem;
@@ -495,6 +503,10 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
 
+  if (tid == 0) {                      // while the thread block sets itself up
+    prefetch_map(&tq);
+    prefetch_map(&tk);
+  }
   Pipe pipe;
   // the two small operand tiles of the normalisers come first, so that whatever the tensor core reads through
   // their descriptors lies inside this thread block's own tiles
