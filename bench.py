@@ -288,8 +288,9 @@ def one_time_rooflines(cfg, S, compress_ms, noscore_ms):
     peak, and select + gather as a copy against the HBM peak."""
     L, n0, H = cfg.prompt_len, cfg.n0, cfg.n_heads
     tiles = 0
-    for r0 in range(0, n0, 128):
-        ctx = L + min(r0 + 128, n0)
+    nb = -(-n0 // 128)
+    for bi in range(nb):                       # blocks of 128 observed queries, aligned to the end (the first is the short one)
+        ctx = L + n0 - (nb - 1 - bi) * 128
         tiles += -(-ctx // 128) + -(-(ctx - (L // 128) * 128) // 128)
     pairs = S * cfg.n_sink_heads
     flops = tiles * 2 * 128 ** 3 * pairs

@@ -468,10 +468,15 @@ ssd_classify_kernel(const ClassifyParams p, int n_row_blocks, const __grid_const
 struct ScoreBlock {
   int r0, last, ctx_max, k_first2;
 };
-__device__ __forceinline__ ScoreBlock score_block(const ScoreParams& p, int r0) {
+// Block bi of n_blocks.  The blocks are aligned to the END of the observed queries: when their number is not a
+// multiple of 128 it is the FIRST block that is short (rows [0, n_obs mod 128) of the tile loaded at row 0; the
+// rows behind them belong to the next block and are left out like rows that do not exist), so the ragged block is
+// the one with the shortest context and the fewest key tiles, not the one with the most.
+__device__ __forceinline__ ScoreBlock score_block(const ScoreParams& p, int bi, int n_blocks) {
   ScoreBlock b;
-  b.r0 = r0;
-  b.last = min(r0 + kRows, p.n_obs) - 1;
+  const int r_end = p.n_obs - (n_blocks - 1 - bi) * kRows;
+  b.r0 = max(r_end - kRows, 0);
+  b.last = r_end - 1;
   b.ctx_max = p.L + (p.n0 - p.n_obs + 1) + b.last;   // keys [0, ctx_max) are visible to the block's last row
   b.k_first2 = (p.L / kKeys) * kKeys;
   return b;
@@ -502,6 +507,7 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
   if (!p.desc[head].w) return;            // before any tensor-memory allocation
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t_first = p.n0 - p.n_obs + 1;  // image step of observed row 0
+  const int n_blocks = (p.n_obs + kRows - 1) / kRows;
 
   if (tid == 0) {                      // while the thread block sets itself up
     prefetch_map(&tq);
@@ -519,10 +525,10 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
     if (lane == 0) {
       Producer pr;
       pr.p = pipe; pr.abort = &s_abort; pr.q_s = q_s; pr.k_s = k_s; pr.tq = &tq; pr.tk = &tk;
-      for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
-        if (block_owner(r0 / kRows, p.n_parts) != part) continue;
-        const ScoreBlock b = score_block(p, r0);
-        pr.query_block(r0, pair);
+      for (int bi = 0; bi < n_blocks; ++bi) {
+        if (block_owner(bi, p.n_parts) != part) continue;
+        const ScoreBlock b = score_block(p, bi, n_blocks);
+        pr.query_block(b.r0, pair);
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) pr.key_tile(k0, pair);
         for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) pr.key_tile(k0, pair);
       }
@@ -532,9 +538,9 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
     if (lane == 0) {
       Issuer is;
       is.p = pipe; is.abort = &s_abort; is.q_s = q_s; is.k_s = k_s; is.tmem = tmem; is.ext_s = ext_s;
-      for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
-        if (block_owner(r0 / kRows, p.n_parts) != part) continue;
-        const ScoreBlock b = score_block(p, r0);
+      for (int bi = 0; bi < n_blocks; ++bi) {
+        if (block_owner(bi, p.n_parts) != part) continue;
+        const ScoreBlock b = score_block(p, bi, n_blocks);
         is.query_block();
         for (int k0 = 0; k0 < b.ctx_max; k0 += kKeys) is.key_tile();
         for (int k0 = b.k_first2; k0 < b.ctx_max; k0 += kKeys) is.key_tile(true, k0 == b.k_first2);
@@ -560,11 +566,12 @@ ssd_score_kernel(const ScoreParams p, const __grid_constant__ CUtensorMap tq, co
     const float inv_scale = 1.f / p.scale_log2;
 
     int blk = 0;                           // blocks this part has done
-    for (int r0 = 0; r0 < p.n_obs; r0 += kRows) {
-      if (block_owner(r0 / kRows, p.n_parts) != part) continue;
-      const ScoreBlock b = score_block(p, r0);
+    for (int bi = 0; bi < n_blocks; ++bi) {
+      if (block_owner(bi, p.n_parts) != part) continue;
+      const ScoreBlock b = score_block(p, bi, n_blocks);
+      const int r0 = b.r0;
       const int row = r0 + rl;
-      const int ctx_r = row < p.n_obs ? p.L + t_first + row : 0;          // keys [0, ctx_r) are visible
+      const int ctx_r = row <= b.last ? p.L + t_first + row : 0;          // keys [0, ctx_r) are visible (none to rows left out)
       const int lo_row = r0 + quad * 32;
       const bool warp_full = lo_row + 31 <= b.last;                       // all 32 rows of the warp exist
       const int lo_ctx = p.L + t_first + lo_row;                          // context of the warp's first row
